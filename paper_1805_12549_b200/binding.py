@@ -1,0 +1,246 @@
+"""Thin ctypes binding of the cgconv C ABI (include/cgconv.h).
+
+Argument marshalling only: every step of the layer runs in the CUDA library.  Tensors are
+torch CUDA tensors (device memory and streams are torch's); their data pointers go straight
+through.  There is no CPU fallback: if the library cannot be loaded, importing fails loudly.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+from . import build as _build
+
+CG_OK = 0
+CG_F32, CG_BF16, CG_I8 = 0, 1, 2
+CG_ALGO_AUTO, CG_ALGO_DIRECT, CG_ALGO_TENSOR = 0, 1, 2
+CG_COND_AUTO, CG_COND_DENSE, CG_COND_SKIP_TILES, CG_COND_COMPACT = 0, 1, 2, 3
+
+EXPORTS = ("cg_conv_create", "cg_conv_workspace_bytes", "cg_conv_forward",
+           "cg_conv_host_staging_bytes", "cg_conv_forward_host", "cg_conv_partial_sums",
+           "cg_conv_stats", "cg_conv_launches_per_forward", "cg_conv_uses_tensor_cores",
+           "cg_conv_destroy", "cg_status_string")
+
+
+class CgConvDesc(C.Structure):
+    _fields_ = [(k, C.c_int32) for k in ("n", "h", "w", "c_in", "c_out", "kh", "kw", "stride",
+                                         "pad", "groups", "in_dtype", "out_dtype")] + \
+               [("bn_eps", C.c_float)] + \
+               [(k, C.c_int32) for k in ("relu", "has_residual", "requant_shift", "algo",
+                                         "cond_mode")]
+
+
+class CgBnParams(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k in ("gamma", "beta", "mean_base", "var_base", "mean_full",
+                                          "var_full", "gate_mean", "gate_var", "q_gate_thr",
+                                          "q_mul_base", "q_mul_full", "q_off_base", "q_off_full")]
+
+
+class CgStats(C.Structure):
+    _fields_ = [(k, C.c_int64) for k in ("calls", "outputs", "active", "dense_macs", "gated_macs",
+                                         "executed_macs", "tiles_total", "tiles_skipped",
+                                         "rows_total", "rows_active")] + \
+               [("device_status", C.c_int32), ("device_site", C.c_int32)]
+
+
+_lib = None
+
+
+def lib():
+    """Load libcgconv.so (building it first if the sources are newer)."""
+    global _lib
+    if _lib is None:
+        path = _build.build()
+        L = C.CDLL(path)
+        L.cg_conv_create.restype = C.c_int
+        L.cg_conv_create.argtypes = [C.POINTER(C.c_void_p), C.POINTER(CgConvDesc)]
+        L.cg_conv_workspace_bytes.restype = C.c_size_t
+        L.cg_conv_workspace_bytes.argtypes = [C.c_void_p]
+        L.cg_conv_forward.restype = C.c_int
+        L.cg_conv_forward.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                      C.POINTER(CgBnParams), C.c_void_p, C.c_void_p, C.c_void_p,
+                                      C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.cg_conv_host_staging_bytes.restype = C.c_size_t
+        L.cg_conv_host_staging_bytes.argtypes = [C.c_void_p]
+        L.cg_conv_forward_host.restype = C.c_int
+        L.cg_conv_forward_host.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                           C.POINTER(CgBnParams), C.c_void_p, C.c_void_p,
+                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                           C.c_void_p]
+        L.cg_conv_partial_sums.restype = C.c_int
+        L.cg_conv_partial_sums.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                           C.c_void_p]
+        L.cg_conv_stats.restype = C.c_int
+        L.cg_conv_stats.argtypes = [C.c_void_p, C.POINTER(CgStats), C.c_void_p]
+        L.cg_conv_launches_per_forward.restype = C.c_int
+        L.cg_conv_launches_per_forward.argtypes = [C.c_void_p]
+        L.cg_conv_uses_tensor_cores.restype = C.c_int
+        L.cg_conv_uses_tensor_cores.argtypes = [C.c_void_p]
+        L.cg_conv_destroy.restype = None
+        L.cg_conv_destroy.argtypes = [C.c_void_p]
+        L.cg_status_string.restype = C.c_char_p
+        L.cg_status_string.argtypes = [C.c_int]
+        _lib = L
+    return _lib
+
+
+class CgError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {lib().cg_status_string(status).decode()} (status {status})")
+
+
+def _check(status: int, where: str):
+    if status != CG_OK:
+        raise CgError(status, where)
+
+
+_TORCH_DTYPE = {CG_F32: torch.float32, CG_BF16: torch.bfloat16, CG_I8: torch.int8}
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+@dataclass
+class Stats:
+    calls: int
+    outputs: int
+    active: int
+    dense_macs: int
+    gated_macs: int
+    executed_macs: int
+    tiles_total: int
+    tiles_skipped: int
+    rows_total: int
+    rows_active: int
+    device_status: int
+    device_site: int
+
+    @property
+    def density(self):
+        return self.active / max(self.outputs, 1)
+
+
+def cg_conv_create(desc: CgConvDesc) -> C.c_void_p:
+    h = C.c_void_p()
+    _check(lib().cg_conv_create(C.byref(h), C.byref(desc)), "cg_conv_create")
+    return h
+
+
+def cg_conv_destroy(h):
+    lib().cg_conv_destroy(h)
+
+
+def cg_conv_workspace_bytes(h) -> int:
+    return int(lib().cg_conv_workspace_bytes(h))
+
+
+def make_bn(params: dict) -> CgBnParams:
+    """dict of torch CUDA tensors (missing/None -> NULL) -> cg_bn_params."""
+    bn = CgBnParams()
+    for k, _ in CgBnParams._fields_:
+        t = params.get(k)
+        setattr(bn, k, None if t is None else t.data_ptr())
+    return bn
+
+
+def cg_conv_forward(h, x, w_base, w_cond, bn: CgBnParams, delta, residual, y, mask_out,
+                    workspace=None, stream=None):
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().cg_conv_forward(h, _ptr(x), _ptr(w_base), _ptr(w_cond), C.byref(bn), _ptr(delta),
+                                 _ptr(residual), _ptr(y), _ptr(mask_out), _ptr(workspace),
+                                 ws_bytes, _stream_ptr(stream)), "cg_conv_forward")
+
+
+def cg_conv_host_staging_bytes(h) -> int:
+    return int(lib().cg_conv_host_staging_bytes(h))
+
+
+def cg_conv_forward_host(h, x_host, w_base, w_cond, bn: CgBnParams, delta, residual_host, y_host,
+                         mask_host, staging, stream=None):
+    _check(lib().cg_conv_forward_host(h, _ptr(x_host), _ptr(w_base), _ptr(w_cond), C.byref(bn),
+                                      _ptr(delta), _ptr(residual_host), _ptr(y_host),
+                                      _ptr(mask_host), _ptr(staging),
+                                      staging.numel() * staging.element_size(),
+                                      _stream_ptr(stream)), "cg_conv_forward_host")
+
+
+def cg_conv_partial_sums(h, x, w_base, p_out, stream=None):
+    _check(lib().cg_conv_partial_sums(h, _ptr(x), _ptr(w_base), _ptr(p_out), _stream_ptr(stream)),
+           "cg_conv_partial_sums")
+
+
+def cg_conv_stats(h, stream=None, check=True) -> Stats:
+    st = CgStats()
+    rc = lib().cg_conv_stats(h, C.byref(st), _stream_ptr(stream))
+    out = Stats(*[getattr(st, k) for k, _ in CgStats._fields_])
+    if check:
+        _check(rc, f"cg_conv_stats (device site {out.device_site})")
+    return out
+
+
+def cg_conv_launches_per_forward(h) -> int:
+    return int(lib().cg_conv_launches_per_forward(h))
+
+
+def cg_conv_uses_tensor_cores(h) -> bool:
+    return bool(lib().cg_conv_uses_tensor_cores(h))
+
+
+class GatedConv:
+    """Convenience owner of one handle plus its workspace (still argument marshalling only)."""
+
+    def __init__(self, n, h, w, c_in, c_out, *, k=3, stride=1, pad=1, groups=4, dtype=CG_BF16,
+                 bn_eps=1e-5, relu=True, has_residual=False, requant_shift=0,
+                 algo=CG_ALGO_AUTO, cond_mode=CG_COND_AUTO, device="cuda"):
+        self.desc = CgConvDesc(n, h, w, c_in, c_out, k, k, stride, pad, groups, dtype, dtype,
+                               bn_eps, int(relu), int(has_residual), requant_shift, algo, cond_mode)
+        self.handle = cg_conv_create(self.desc)
+        self.dtype = dtype
+        self.ho = (h + 2 * pad - k) // stride + 1
+        self.wo = (w + 2 * pad - k) // stride + 1
+        self.m = n * self.ho * self.wo
+        self.c_out = c_out
+        self.words = (c_out + 31) // 32
+        self.device = device
+        nbytes = cg_conv_workspace_bytes(self.handle)
+        self.workspace = torch.empty(max(nbytes, 1), dtype=torch.uint8, device=device) \
+            if nbytes else None
+
+    def alloc_outputs(self):
+        y = torch.empty((self.desc.n, self.ho, self.wo, self.c_out), dtype=_TORCH_DTYPE[self.dtype],
+                        device=self.device)
+        mask = torch.empty((self.m, self.words), dtype=torch.int32, device=self.device)
+        return y, mask
+
+    def forward(self, x, w_base, w_cond, bn: CgBnParams, delta, y, mask=None, residual=None,
+                stream=None):
+        cg_conv_forward(self.handle, x, w_base, w_cond, bn, delta, residual, y, mask,
+                        self.workspace, stream)
+
+    def stats(self, stream=None, check=True) -> Stats:
+        return cg_conv_stats(self.handle, stream, check)
+
+    @property
+    def uses_tensor_cores(self):
+        return cg_conv_uses_tensor_cores(self.handle)
+
+    def close(self):
+        if self.handle is not None:
+            cg_conv_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

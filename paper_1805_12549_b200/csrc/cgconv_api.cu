@@ -1,0 +1,251 @@
+// Host side of the cgconv C ABI (include/cgconv.h): argument checks, kernel selection,
+// counters.  No kernel lives here.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+#include "tc_conv.cuh"
+
+struct cg_conv_s {
+  cg_conv_desc desc;
+  cg::LayerDims L;
+  int use_tc;
+  cg::TcPlan plan;
+  int device;
+  unsigned long long* counters;   // device, cg::CNT_SLOTS entries
+  long long calls;
+  cg::TcMaps maps;                // tensor maps cached for the last set of pointers
+};
+
+namespace {
+
+size_t elem_bytes(int dt) { return dt == CG_F32 ? 4 : (dt == CG_BF16 ? 2 : 1); }
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+cg_status check_desc(const cg_conv_desc* d) {
+  if (!d) return CG_ERR_INVALID_ARG;
+  if (d->n <= 0 || d->h <= 0 || d->w <= 0 || d->c_in <= 0 || d->c_out <= 0) return CG_ERR_INVALID_ARG;
+  if (d->kh <= 0 || d->kw <= 0 || d->stride <= 0 || d->pad < 0) return CG_ERR_INVALID_ARG;
+  if (d->kh != d->kw) return CG_ERR_INVALID_ARG;
+  if (d->groups <= 0 || d->c_in % d->groups != 0) return CG_ERR_INVALID_ARG;
+  if ((d->h + 2 * d->pad - d->kh) < 0 || (d->w + 2 * d->pad - d->kw) < 0) return CG_ERR_INVALID_ARG;
+  if (d->in_dtype != CG_F32 && d->in_dtype != CG_BF16 && d->in_dtype != CG_I8) return CG_ERR_INVALID_ARG;
+  if (d->out_dtype != d->in_dtype) return CG_ERR_INVALID_ARG;
+  if (d->in_dtype == CG_I8 && (d->requant_shift < 1 || d->requant_shift > 31)) return CG_ERR_INVALID_ARG;
+  if (d->in_dtype == CG_I8 && d->has_residual) return CG_ERR_INVALID_ARG;
+  if (!(d->bn_eps >= 0.f)) return CG_ERR_INVALID_ARG;
+  if (d->algo < CG_ALGO_AUTO || d->algo > CG_ALGO_TENSOR) return CG_ERR_INVALID_ARG;
+  if (d->cond_mode < CG_COND_AUTO || d->cond_mode > CG_COND_COMPACT) return CG_ERR_INVALID_ARG;
+  return CG_OK;
+}
+
+cg::LayerDims make_dims(const cg_conv_desc& d) {
+  cg::LayerDims L;
+  L.n = d.n; L.h = d.h; L.w = d.w; L.c_in = d.c_in; L.c_out = d.c_out;
+  L.kh = d.kh; L.kw = d.kw; L.stride = d.stride; L.pad = d.pad;
+  L.groups = d.groups; L.c_p = d.c_in / d.groups; L.c_r = d.c_in - L.c_p;
+  L.ho = (d.h + 2 * d.pad - d.kh) / d.stride + 1;
+  L.wo = (d.w + 2 * d.pad - d.kw) / d.stride + 1;
+  L.m = (long long)d.n * L.ho * L.wo;
+  L.words = (d.c_out + 31) / 32;
+  L.eps = d.bn_eps; L.relu = d.relu ? 1 : 0; L.has_residual = d.has_residual ? 1 : 0;
+  L.shift = d.requant_shift;
+  return L;
+}
+
+cg_status check_bn(const cg_conv_s* h, const cg_bn_params* bn, const float* delta) {
+  if (!bn) return CG_ERR_INVALID_ARG;
+  if (h->desc.in_dtype == CG_I8) {
+    if (!bn->q_gate_thr || !bn->q_mul_base || !bn->q_mul_full || !bn->q_off_base || !bn->q_off_full)
+      return CG_ERR_INVALID_ARG;
+  } else {
+    if (!bn->gamma || !bn->beta || !bn->mean_base || !bn->var_base || !bn->mean_full || !bn->var_full)
+      return CG_ERR_INVALID_ARG;
+    if ((bn->gate_mean == nullptr) != (bn->gate_var == nullptr)) return CG_ERR_INVALID_ARG;
+    if (!delta) return CG_ERR_INVALID_ARG;
+  }
+  return CG_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* cg_status_string(cg_status s) {
+  switch (s) {
+    case CG_OK: return "ok";
+    case CG_ERR_INVALID_ARG: return "invalid argument";
+    case CG_ERR_UNSUPPORTED: return "layer not supported by the requested kernels";
+    case CG_ERR_ALIGNMENT: return "tensor pointer not sufficiently aligned";
+    case CG_ERR_WORKSPACE: return "workspace missing or too small";
+    case CG_ERR_CUDA: return "CUDA call failed";
+    case CG_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel expired";
+    case CG_ERR_DEVICE_BOUNDS: return "a kernel-side range check failed";
+  }
+  return "unknown status";
+}
+
+cg_status cg_conv_create(cg_conv_t* out, const cg_conv_desc* desc) {
+  if (!out) return CG_ERR_INVALID_ARG;
+  const cg_status st = check_desc(desc);
+  if (st != CG_OK) return st;
+  cg_conv_s* h = new (std::nothrow) cg_conv_s();
+  if (!h) return CG_ERR_INVALID_ARG;
+  h->desc = *desc;
+  h->L = make_dims(*desc);
+  h->calls = 0;
+  h->counters = nullptr;
+  std::memset(&h->maps, 0, sizeof(h->maps));
+  const bool tc_ok = cg::tc_plan(h->L, desc->in_dtype, desc->cond_mode, &h->plan);
+  if (desc->algo == CG_ALGO_TENSOR && !tc_ok) { delete h; return CG_ERR_UNSUPPORTED; }
+  h->use_tc = (desc->algo != CG_ALGO_DIRECT) && tc_ok;
+  if (cudaGetDevice(&h->device) != cudaSuccess) { delete h; return CG_ERR_CUDA; }
+  if (h->use_tc && !cg::tc_device_ok(h->device)) {
+    if (desc->algo == CG_ALGO_TENSOR) { delete h; return CG_ERR_UNSUPPORTED; }
+    h->use_tc = 0;
+  }
+  if (cudaMalloc(&h->counters, cg::CNT_SLOTS * sizeof(unsigned long long)) != cudaSuccess) {
+    delete h; return CG_ERR_CUDA;
+  }
+  if (cudaMemset(h->counters, 0, cg::CNT_SLOTS * sizeof(unsigned long long)) != cudaSuccess) {
+    cudaFree(h->counters); delete h; return CG_ERR_CUDA;
+  }
+  *out = h;
+  return CG_OK;
+}
+
+void cg_conv_destroy(cg_conv_t h) {
+  if (!h) return;
+  if (h->counters) cudaFree(h->counters);
+  delete h;
+}
+
+size_t cg_conv_workspace_bytes(cg_conv_t h) {
+  if (!h) return 0;
+  return h->use_tc ? cg::tc_workspace_bytes(h->L, h->plan) : 0;
+}
+
+int cg_conv_launches_per_forward(cg_conv_t h) { return h ? 1 : 0; }
+
+int cg_conv_uses_tensor_cores(cg_conv_t h) { return h ? h->use_tc : 0; }
+
+cg_status cg_conv_forward(cg_conv_t h, const void* x, const void* w_base, const void* w_cond,
+                          const cg_bn_params* bn, const float* delta, const void* residual,
+                          void* y, uint32_t* mask_out, void* workspace, size_t workspace_bytes,
+                          void* cuda_stream) {
+  if (!h || !x || !w_base || !y) return CG_ERR_INVALID_ARG;
+  if (!w_cond && h->L.c_r > 0) return CG_ERR_INVALID_ARG;
+  cg_status st = check_bn(h, bn, delta);
+  if (st != CG_OK) return st;
+  if ((residual != nullptr) != (h->desc.has_residual != 0)) return CG_ERR_INVALID_ARG;
+  if (!aligned(x, 16) || !aligned(w_base, 16) || (w_cond && !aligned(w_cond, 16)) ||
+      !aligned(y, 16) || (residual && !aligned(residual, 16)) || (mask_out && !aligned(mask_out, 4)))
+    return CG_ERR_ALIGNMENT;
+  const size_t need = cg_conv_workspace_bytes(h);
+  if (need > 0 && (!workspace || workspace_bytes < need)) return CG_ERR_WORKSPACE;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  int err;
+  if (h->use_tc) {
+    err = cg::launch_tc(h->L, h->plan, h->desc.in_dtype, &h->maps, x, w_base, w_cond, *bn, delta,
+                        residual, y, mask_out, workspace, h->counters, stream);
+  } else {
+    err = cg::launch_direct(h->L, h->desc.in_dtype, x, w_base, w_cond, *bn, delta, residual, y,
+                            mask_out, nullptr, 0, h->counters, stream);
+  }
+  if (err != 0) return CG_ERR_CUDA;
+  h->calls += 1;
+  return CG_OK;
+}
+
+size_t cg_conv_host_staging_bytes(cg_conv_t h) {
+  if (!h) return 0;
+  const size_t eb = elem_bytes(h->desc.in_dtype), ob = elem_bytes(h->desc.out_dtype);
+  size_t total = align_up((size_t)h->L.n * h->L.h * h->L.w * h->L.c_in * eb, 256);
+  total += align_up((size_t)h->L.m * h->L.c_out * ob, 256);                     // y
+  total += align_up((size_t)h->L.m * h->L.words * 4, 256);                      // mask
+  if (h->desc.has_residual) total += align_up((size_t)h->L.m * h->L.c_out * ob, 256);
+  total += align_up(cg_conv_workspace_bytes(h), 256);
+  return total;
+}
+
+cg_status cg_conv_forward_host(cg_conv_t h, const void* x_host, const void* w_base,
+                               const void* w_cond, const cg_bn_params* bn, const float* delta,
+                               const void* residual_host, void* y_host, uint32_t* mask_host,
+                               void* staging, size_t staging_bytes, void* cuda_stream) {
+  if (!h || !x_host || !y_host || !staging) return CG_ERR_INVALID_ARG;
+  if (staging_bytes < cg_conv_host_staging_bytes(h)) return CG_ERR_WORKSPACE;
+  if (!aligned(staging, 256)) return CG_ERR_ALIGNMENT;
+  if ((residual_host != nullptr) != (h->desc.has_residual != 0)) return CG_ERR_INVALID_ARG;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const size_t eb = elem_bytes(h->desc.in_dtype), ob = elem_bytes(h->desc.out_dtype);
+  const size_t x_bytes = (size_t)h->L.n * h->L.h * h->L.w * h->L.c_in * eb;
+  const size_t y_bytes = (size_t)h->L.m * h->L.c_out * ob;
+  const size_t m_bytes = (size_t)h->L.m * h->L.words * 4;
+  char* p = static_cast<char*>(staging);
+  void* x_dev = p; p += align_up(x_bytes, 256);
+  void* y_dev = p; p += align_up(y_bytes, 256);
+  uint32_t* m_dev = reinterpret_cast<uint32_t*>(p); p += align_up(m_bytes, 256);
+  void* r_dev = nullptr;
+  if (h->desc.has_residual) { r_dev = p; p += align_up(y_bytes, 256); }
+  void* ws = p;
+  if (cudaMemcpyAsync(x_dev, x_host, x_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+    return CG_ERR_CUDA;
+  if (r_dev && cudaMemcpyAsync(r_dev, residual_host, y_bytes, cudaMemcpyHostToDevice, stream) !=
+                   cudaSuccess)
+    return CG_ERR_CUDA;
+  const cg_status st = cg_conv_forward(h, x_dev, w_base, w_cond, bn, delta, r_dev, y_dev,
+                                       mask_host ? m_dev : nullptr, ws,
+                                       cg_conv_workspace_bytes(h), cuda_stream);
+  if (st != CG_OK) return st;
+  if (cudaMemcpyAsync(y_host, y_dev, y_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+    return CG_ERR_CUDA;
+  if (mask_host &&
+      cudaMemcpyAsync(mask_host, m_dev, m_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+    return CG_ERR_CUDA;
+  return CG_OK;
+}
+
+cg_status cg_conv_partial_sums(cg_conv_t h, const void* x, const void* w_base, void* p_out,
+                               void* cuda_stream) {
+  if (!h || !x || !w_base || !p_out) return CG_ERR_INVALID_ARG;
+  if (!aligned(x, 16) || !aligned(w_base, 16) || !aligned(p_out, 4)) return CG_ERR_ALIGNMENT;
+  cg_bn_params none;
+  std::memset(&none, 0, sizeof(none));
+  const int err = cg::launch_direct(h->L, h->desc.in_dtype, x, w_base, nullptr, none, nullptr,
+                                    nullptr, nullptr, nullptr, p_out, 1, h->counters,
+                                    reinterpret_cast<cudaStream_t>(cuda_stream));
+  return err == 0 ? CG_OK : CG_ERR_CUDA;
+}
+
+cg_status cg_conv_stats(cg_conv_t h, cg_stats* out, void* cuda_stream) {
+  if (!h || !out) return CG_ERR_INVALID_ARG;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  unsigned long long c[cg::CNT_SLOTS];
+  if (cudaMemcpyAsync(c, h->counters, sizeof(c), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+    return CG_ERR_CUDA;
+  if (cudaMemsetAsync(h->counters, 0, sizeof(c), stream) != cudaSuccess) return CG_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return CG_ERR_CUDA;
+  const cg::LayerDims& L = h->L;
+  const long long k2 = (long long)L.kh * L.kw;
+  std::memset(out, 0, sizeof(*out));
+  out->calls = h->calls;
+  out->outputs = h->calls * L.m * L.c_out;
+  out->active = (int64_t)c[cg::CNT_ACTIVE];
+  out->dense_macs = out->outputs * k2 * L.c_in;
+  out->gated_macs = k2 * ((long long)L.c_p * out->outputs + (long long)L.c_r * out->active);
+  out->executed_macs = k2 * L.c_p * out->outputs + (int64_t)c[cg::CNT_EXEC_MACS];
+  out->tiles_total = (int64_t)c[cg::CNT_TILES_TOTAL];
+  out->tiles_skipped = (int64_t)c[cg::CNT_TILES_SKIPPED];
+  out->rows_total = (int64_t)c[cg::CNT_ROWS_TOTAL];
+  out->rows_active = (int64_t)c[cg::CNT_ROWS_ACTIVE];
+  out->device_status = (int32_t)c[cg::CNT_STATUS];
+  out->device_site = (int32_t)c[cg::CNT_SITE];
+  h->calls = 0;
+  return out->device_status ? (cg_status)out->device_status : CG_OK;
+}
+
+}  // extern "C"

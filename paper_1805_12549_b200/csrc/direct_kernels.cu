@@ -1,0 +1,230 @@
+// CUDA-core direct convolution of the channel-gated layer: the path for fp32 layers and for
+// every shape the tensor-core path does not take.
+//
+// One warp owns one (pixel row m, 32-channel block q): lane = output channel.  Each lane runs
+// the base-path sum (Section 3.1), takes the gate decision (Eq. 2/3), runs the conditional-path
+// sum only if its own gate fired (Eq. 1), applies the path's batch norm and ReLU, and the
+// warp's ballot is the mask word.  Floating-point sums run in the order (r, s, c_in) with
+// separately rounded multiply and add, so results do not depend on the launch shape.
+#include "common.cuh"
+
+namespace cg {
+namespace {
+
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+  static __device__ __forceinline__ float ld(const float* p) { return *p; }
+};
+template <> struct Elem<__nv_bfloat16> {
+  static __device__ __forceinline__ float ld(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+};
+
+__device__ __forceinline__ void st_out(float* p, float v) { *p = v; }
+__device__ __forceinline__ void st_out(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+// Sum over taps and channels [c_lo, c_lo + cw) of one output activation.
+template <typename T>
+__device__ __forceinline__ float conv_point(const LayerDims& L, const T* __restrict__ x,
+                                            const T* __restrict__ w, int n, int ho, int wo, int co,
+                                            int c_lo, int cw) {
+  float acc = 0.f;
+  for (int r = 0; r < L.kh; ++r) {
+    const int hi = ho * L.stride + r - L.pad;
+    if (hi < 0 || hi >= L.h) continue;
+    for (int s = 0; s < L.kw; ++s) {
+      const int wi = wo * L.stride + s - L.pad;
+      if (wi < 0 || wi >= L.w) continue;
+      const T* xp = x + (((long long)n * L.h + hi) * L.w + wi) * L.c_in + c_lo;
+      const T* wp = w + (((long long)co * L.kh + r) * L.kw + s) * cw;
+      for (int ci = 0; ci < cw; ++ci)
+        acc = __fadd_rn(acc, __fmul_rn(Elem<T>::ld(xp + ci), Elem<T>::ld(wp + ci)));
+    }
+  }
+  return acc;
+}
+
+__device__ __forceinline__ int conv_point_i8(const LayerDims& L, const int8_t* __restrict__ x,
+                                             const int8_t* __restrict__ w, int n, int ho, int wo,
+                                             int co, int c_lo, int cw) {
+  int acc = 0;
+  for (int r = 0; r < L.kh; ++r) {
+    const int hi = ho * L.stride + r - L.pad;
+    if (hi < 0 || hi >= L.h) continue;
+    for (int s = 0; s < L.kw; ++s) {
+      const int wi = wo * L.stride + s - L.pad;
+      if (wi < 0 || wi >= L.w) continue;
+      const int8_t* xp = x + (((long long)n * L.h + hi) * L.w + wi) * L.c_in + c_lo;
+      const int8_t* wp = w + (((long long)co * L.kh + r) * L.kw + s) * cw;
+      for (int ci = 0; ci < cw; ++ci) acc += (int)xp[ci] * (int)wp[ci];
+    }
+  }
+  return acc;
+}
+
+constexpr int kThreads = 256;
+
+template <typename TIn, typename TOut>
+__global__ void __launch_bounds__(kThreads)
+direct_gated_conv_kernel(LayerDims L, const TIn* __restrict__ x, const TIn* __restrict__ w_base,
+                         const TIn* __restrict__ w_cond, cg_bn_params bn,
+                         const float* __restrict__ delta, const TOut* __restrict__ residual,
+                         TOut* __restrict__ y, uint32_t* __restrict__ mask,
+                         float* __restrict__ p_out, int base_only,
+                         unsigned long long* __restrict__ counters) {
+  extern __shared__ float s_consts[];   // 5 * c_out: t, a1, b1, a2, b2
+  __shared__ unsigned long long s_active;
+  float* s_t = s_consts;
+  float* s_a1 = s_t + L.c_out;
+  float* s_b1 = s_a1 + L.c_out;
+  float* s_a2 = s_b1 + L.c_out;
+  float* s_b2 = s_a2 + L.c_out;
+  if (threadIdx.x == 0) s_active = 0ull;
+  if (!base_only) {
+    for (int c = threadIdx.x; c < L.c_out; c += blockDim.x) {
+      const ChannelConsts k = fold_channel(bn, delta, L.eps, c);
+      s_t[c] = k.t; s_a1[c] = k.a1; s_b1[c] = k.b1; s_a2[c] = k.a2; s_b2[c] = k.b2;
+    }
+  }
+  __syncthreads();
+
+  const int lane = threadIdx.x & 31;
+  const long long warps = (long long)gridDim.x * (blockDim.x >> 5);
+  const long long warp0 = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const long long items = L.m * L.words;
+  unsigned long long my_active = 0;
+  for (long long it = warp0; it < items; it += warps) {
+    const long long m = it / L.words;
+    const int q = (int)(it - m * L.words);
+    const int co = q * 32 + lane;
+    const bool valid = co < L.c_out;
+    const int wo = (int)(m % L.wo);
+    const int ho = (int)((m / L.wo) % L.ho);
+    const int n = (int)(m / ((long long)L.wo * L.ho));
+    bool fire = false;
+    if (valid) {
+      const float p = conv_point<TIn>(L, x, w_base, n, ho, wo, co, 0, L.c_p);
+      if (base_only) {
+        p_out[m * L.c_out + co] = p;
+      } else {
+        fire = (p >= s_t[co]);   // NaN compares false
+        float v;
+        if (fire) {
+          const float r = conv_point<TIn>(L, x, w_cond, n, ho, wo, co, L.c_p, L.c_r);
+          v = __fadd_rn(__fmul_rn(s_a2[co], __fadd_rn(p, r)), s_b2[co]);
+        } else {
+          v = __fadd_rn(__fmul_rn(s_a1[co], p), s_b1[co]);
+        }
+        if (residual) v = __fadd_rn(v, (float)residual[m * L.c_out + co]);
+        if (L.relu) v = (v > 0.f) ? v : 0.f;
+        st_out(y + m * L.c_out + co, v);
+      }
+    }
+    if (!base_only) {
+      const unsigned word = __ballot_sync(0xffffffffu, fire);
+      if (lane == 0) {
+        if (mask) mask[it] = word;
+        my_active += __popc(word);
+      }
+    }
+  }
+  if (!base_only) {
+    if (lane == 0 && my_active) atomicAdd(&s_active, my_active);
+    __syncthreads();
+    if (threadIdx.x == 0 && s_active) {
+      atomicAdd(&counters[CNT_ACTIVE], s_active);
+      atomicAdd(&counters[CNT_EXEC_MACS],
+                s_active * (unsigned long long)(L.kh * L.kw * L.c_r));
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kThreads)
+direct_gated_conv_i8_kernel(LayerDims L, const int8_t* __restrict__ x,
+                            const int8_t* __restrict__ w_base, const int8_t* __restrict__ w_cond,
+                            cg_bn_params bn, int8_t* __restrict__ y, uint32_t* __restrict__ mask,
+                            int* __restrict__ p_out, int base_only,
+                            unsigned long long* __restrict__ counters) {
+  __shared__ unsigned long long s_active;
+  if (threadIdx.x == 0) s_active = 0ull;
+  __syncthreads();
+  const int lane = threadIdx.x & 31;
+  const long long warps = (long long)gridDim.x * (blockDim.x >> 5);
+  const long long warp0 = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const long long items = L.m * L.words;
+  unsigned long long my_active = 0;
+  for (long long it = warp0; it < items; it += warps) {
+    const long long m = it / L.words;
+    const int q = (int)(it - m * L.words);
+    const int co = q * 32 + lane;
+    const bool valid = co < L.c_out;
+    const int wo = (int)(m % L.wo);
+    const int ho = (int)((m / L.wo) % L.ho);
+    const int n = (int)(m / ((long long)L.wo * L.ho));
+    bool fire = false;
+    if (valid) {
+      const int p = conv_point_i8(L, x, w_base, n, ho, wo, co, 0, L.c_p);
+      if (base_only) {
+        p_out[m * L.c_out + co] = p;
+      } else {
+        fire = (p >= bn.q_gate_thr[co]);
+        long long acc = p;
+        if (fire) acc += conv_point_i8(L, x, w_cond, n, ho, wo, co, L.c_p, L.c_r);
+        const bool full = fire;
+        const long long mul = full ? bn.q_mul_full[co] : bn.q_mul_base[co];
+        const long long off = full ? bn.q_off_full[co] : bn.q_off_base[co];
+        long long qv = (acc * mul + off + (1ll << (L.shift - 1))) >> L.shift;
+        const long long lo = L.relu ? 0 : -128;
+        qv = qv < lo ? lo : (qv > 127 ? 127 : qv);
+        y[m * L.c_out + co] = (int8_t)qv;
+      }
+    }
+    if (!base_only) {
+      const unsigned word = __ballot_sync(0xffffffffu, fire);
+      if (lane == 0) {
+        if (mask) mask[it] = word;
+        my_active += __popc(word);
+      }
+    }
+  }
+  if (!base_only) {
+    if (lane == 0 && my_active) atomicAdd(&s_active, my_active);
+    __syncthreads();
+    if (threadIdx.x == 0 && s_active) {
+      atomicAdd(&counters[CNT_ACTIVE], s_active);
+      atomicAdd(&counters[CNT_EXEC_MACS],
+                s_active * (unsigned long long)(L.kh * L.kw * L.c_r));
+    }
+  }
+}
+
+}  // namespace
+
+int launch_direct(const LayerDims& L, int in_dtype, const void* x, const void* w_base,
+                  const void* w_cond, const cg_bn_params& bn, const float* delta,
+                  const void* residual, void* y, uint32_t* mask, void* p_out, int base_only,
+                  unsigned long long* counters, cudaStream_t stream) {
+  const long long items = L.m * L.words;
+  if (items == 0) return 0;
+  const int warps_per_block = kThreads / 32;
+  long long blocks = (items + warps_per_block - 1) / warps_per_block;
+  const long long cap = 148ll * 8 * 8;
+  if (blocks > cap) blocks = cap;
+  const size_t smem = (size_t)5 * L.c_out * sizeof(float);
+  if (in_dtype == CG_F32) {
+    direct_gated_conv_kernel<float, float><<<(unsigned)blocks, kThreads, smem, stream>>>(
+        L, (const float*)x, (const float*)w_base, (const float*)w_cond, bn, delta,
+        (const float*)residual, (float*)y, mask, (float*)p_out, base_only, counters);
+  } else if (in_dtype == CG_BF16) {
+    direct_gated_conv_kernel<__nv_bfloat16, __nv_bfloat16><<<(unsigned)blocks, kThreads, smem, stream>>>(
+        L, (const __nv_bfloat16*)x, (const __nv_bfloat16*)w_base, (const __nv_bfloat16*)w_cond, bn,
+        delta, (const __nv_bfloat16*)residual, (__nv_bfloat16*)y, mask, (float*)p_out, base_only,
+        counters);
+  } else {
+    direct_gated_conv_i8_kernel<<<(unsigned)blocks, kThreads, 0, stream>>>(
+        L, (const int8_t*)x, (const int8_t*)w_base, (const int8_t*)w_cond, bn, (int8_t*)y, mask,
+        (int*)p_out, base_only, counters);
+  }
+  return (int)cudaGetLastError();
+}
+
+}  // namespace cg

@@ -1,0 +1,49 @@
+// Tensor-core (tcgen05) path of the channel-gated layer: plan, tensor maps, launcher.
+#pragma once
+
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace cg {
+
+// Tiling of one layer for the shifted-window implicit GEMM (see tc_conv.cu).
+struct TcPlan {
+  int valid;
+  int elem_bytes;       // 2 (bf16) or 1 (int8)
+  int ck;               // channels per 128-byte (bf16) patch row = one K chunk
+  int images_mode;      // 0: a tile is `r` output rows of one image; 1: `ni` whole images
+  int wp;               // patch row pitch in pixels: w + pad (rows share their zero columns)
+  int r;                // output rows per tile (rows mode)
+  int ni;               // images per tile (images mode), else 1
+  int ip;               // image pitch in patch pixels: (h + pad) * wp
+  int tiles_per_image;  // rows mode
+  int tiles_m, tiles_n, nt;
+  int chunks;           // c_in / ck patch buffers, all resident
+  int base_chunks;      // chunks that hold base-path channels
+  int box_h;            // patch box rows: r + 2*pad (rows mode) or h + pad (images mode)
+  int box_pixels;       // wp * box_h * ni
+  int patch_rows;       // rows allocated per patch buffer
+  int patch_bytes;
+  int out_box_h;        // y store box rows
+  int stage_rows;       // rows of the y staging tile
+  int stages;           // depth of the weight-tile ring
+  int base_tiles, cond_tiles;   // weight tiles per phase
+  int cond_mode;
+  unsigned off_a, off_b, off_y, off_consts, off_bar, smem_bytes;
+};
+
+struct TcMaps {
+  const void* key[4];   // x, w_base, w_cond, y the maps below were encoded for
+  CUtensorMap x, wb, wc, y;
+};
+
+bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan);
+bool tc_device_ok(int device);
+size_t tc_workspace_bytes(const LayerDims& L, const TcPlan& plan);
+int launch_tc(const LayerDims& L, const TcPlan& plan, int in_dtype, TcMaps* maps, const void* x,
+              const void* w_base, const void* w_cond, const cg_bn_params& bn, const float* delta,
+              const void* residual, void* y, uint32_t* mask, void* workspace,
+              unsigned long long* counters, cudaStream_t stream);
+
+}  // namespace cg

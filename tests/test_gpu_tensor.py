@@ -1,0 +1,101 @@
+"""GPU parity of the tcgen05 tensor-core path against the oracle.
+
+bf16 bar: masks equal except where the oracle's normalised partial sum lies within 1e-3 of
+Delta (that count is printed); outputs within 2e-2 + 1e-2*|ref| wherever the masks agree."""
+import numpy as np
+import pytest
+
+from oracle import oracle as O
+from tests import cases as K
+
+pytestmark = pytest.mark.gpu
+
+TENSOR = 2
+DENSE, SKIP = 1, 2
+
+# (shape, why): several tiles, ragged last tiles, every tiling mode
+SHAPES = [
+    (O.Shape(2, 56, 56, 64, 64, groups=4), "rows mode, 2 rows per tile, c_p = 16"),
+    (O.Shape(3, 28, 28, 128, 128, groups=4), "rows mode, c_p = 32, two chunks"),
+    (O.Shape(3, 14, 14, 256, 256, groups=4), "rows mode 7+7, c_p = 64, two column tiles"),
+    (O.Shape(5, 7, 7, 512, 512, groups=4), "two images per tile, odd batch, c_p = 128"),
+    (O.Shape(2, 32, 32, 64, 64, groups=4), "CIFAR 32x32"),
+    (O.Shape(2, 16, 16, 128, 128, groups=4), "CIFAR 16x16"),
+    (O.Shape(3, 8, 8, 256, 256, groups=4), "one 8x8 image per tile"),
+    (O.Shape(7, 4, 4, 512, 512, groups=4), "five 4x4 images per tile, ragged"),
+    (O.Shape(2, 28, 28, 128, 128, groups=8), "G = 8, c_p = 16"),
+    (O.Shape(2, 14, 14, 256, 64, groups=8), "G = 8, c_p = 32, c_out != c_in"),
+    (O.Shape(2, 13, 11, 64, 192, groups=2), "odd extents, G = 2, three column tiles of 64"),
+    (O.Shape(2, 9, 9, 64, 64, kh=1, kw=1, pad=0, groups=4), "1x1 kernel"),
+]
+
+
+def _run(c, cond_mode=0):
+    ref = K.run_oracle(c)
+    g = K.GpuCase(c, algo=TENSOR, cond_mode=cond_mode)
+    assert g.conv.uses_tensor_cores
+    y, mask, st = g.run()
+    exempt = K.compare(c, ref, y, mask, st)
+    g.close()
+    return ref, st, exempt
+
+
+@pytest.mark.parametrize("s,why", SHAPES, ids=[w for _, w in SHAPES])
+def test_parity_at_30_percent(s, why):
+    c = K.make_float_case("tc30", s, "bf16", density=0.3)
+    ref, st, exempt = _run(c)
+    print(f"{why}: density {st.density:.3f}, near-tie mismatches {exempt}, "
+          f"blocks skipped {st.tiles_skipped}/{st.tiles_total}")
+    assert abs(st.density - ref.density) < 2e-3
+    assert 0.2 < st.density < 0.4
+
+
+@pytest.mark.parametrize("s,why", SHAPES[:4], ids=[w for _, w in SHAPES[:4]])
+@pytest.mark.parametrize("dv", [-K.INF, K.INF])
+def test_delta_limits(s, why, dv):
+    """All gates open: the ordinary layer.  All gates shut: base path only, every block skipped."""
+    c = K.make_float_case("tclim", s, "bf16", delta=dv)
+    ref, st, exempt = _run(c)
+    assert exempt == 0
+    if dv < 0:
+        assert st.active == st.outputs and st.tiles_skipped == 0
+    else:
+        assert st.active == 0 and st.tiles_skipped == st.tiles_total
+
+
+@pytest.mark.parametrize("s,why", SHAPES[:4], ids=[w for _, w in SHAPES[:4]])
+def test_dense_mode_matches_skip_mode(s, why):
+    c = K.make_float_case("tcdense", s, "bf16", density=0.1, rho=0.7)
+    ref, st_d, _ = _run(c, cond_mode=DENSE)
+    _, st_s, _ = _run(c, cond_mode=SKIP)
+    assert st_d.active == st_s.active
+    assert st_d.tiles_skipped == 0
+    assert st_s.executed_macs <= st_d.executed_macs
+
+
+def test_idle_tiles_are_skipped():
+    """A blank image gives P = 0 below every (positive) threshold: its tiles skip the
+    conditional path entirely; clustered gates leave most pixel rows idle elsewhere."""
+    s = O.Shape(2, 56, 56, 64, 64, groups=4)
+    c = K.make_float_case("tcskip", s, "bf16", density=0.02, rho=0.95)
+    c.x[1] = 0.0
+    t = O.fold_params(s, c.bn, c.delta)["t"]
+    assert (t > 0).all()
+    ref, st, _ = _run(c, cond_mode=SKIP)
+    assert st.tiles_total == 56 and st.tiles_skipped >= 28
+    assert st.rows_active < st.rows_total // 2
+    assert st.rows_total == s.m
+    k2 = 9
+    assert st.executed_macs == 128 * 64 * k2 * (s.c_p * 56 + s.c_r * (56 - st.tiles_skipped))
+
+
+def test_two_calls_accumulate_and_are_deterministic():
+    s = O.Shape(2, 28, 28, 128, 128, groups=4)
+    c = K.make_float_case("tcdet", s, "bf16", density=0.3)
+    g = K.GpuCase(c, algo=TENSOR)
+    y1, m1, st1 = g.run()
+    y2, m2, st2 = g.run()
+    np.testing.assert_array_equal(y1.view(np.uint32), y2.view(np.uint32))
+    np.testing.assert_array_equal(m1, m2)
+    assert st1.active == st2.active and st1.calls == st2.calls == 1
+    g.close()

@@ -1,0 +1,95 @@
+"""CPU-side checks of the C-ABI library: it loads without a GPU, exports every symbol the
+header declares, and rejects bad descriptions before touching CUDA."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_1805_12549_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "cgconv.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(cg_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = B.lib()
+    names = _declared_symbols()
+    assert set(B.EXPORTS) <= set(names)
+    assert len(names) >= 11
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_status_strings():
+    lib = B.lib()
+    seen = {lib.cg_status_string(i) for i in range(8)}
+    assert len(seen) == 8
+    assert lib.cg_status_string(0) == b"ok"
+
+
+def _desc(**kw):
+    base = dict(n=2, h=8, w=8, c_in=16, c_out=16, kh=3, kw=3, stride=1, pad=1, groups=4,
+                in_dtype=B.CG_F32, out_dtype=B.CG_F32, bn_eps=1e-5, relu=1, has_residual=0,
+                requant_shift=0, algo=0, cond_mode=0)
+    base.update(kw)
+    return B.CgConvDesc(**base)
+
+
+@pytest.mark.parametrize("kw", [dict(n=0), dict(c_in=15), dict(kh=3, kw=5), dict(groups=0),
+                                dict(stride=0), dict(pad=-1), dict(in_dtype=7, out_dtype=7),
+                                dict(out_dtype=B.CG_BF16), dict(h=1, w=1, pad=0),
+                                dict(in_dtype=B.CG_I8, out_dtype=B.CG_I8, requant_shift=0),
+                                dict(in_dtype=B.CG_I8, out_dtype=B.CG_I8, requant_shift=32),
+                                dict(bn_eps=-1.0), dict(algo=9), dict(cond_mode=-1)])
+def test_create_rejects_bad_descriptions(kw):
+    h = C.c_void_p()
+    d = _desc(**kw)
+    assert B.lib().cg_conv_create(C.byref(h), C.byref(d)) == 1      # CG_ERR_INVALID_ARG
+    assert not h.value
+
+
+def test_create_null_arguments():
+    d = _desc()
+    assert B.lib().cg_conv_create(None, C.byref(d)) == 1
+    h = C.c_void_p()
+    assert B.lib().cg_conv_create(C.byref(h), None) == 1
+
+
+def test_tensor_algo_rejects_ineligible_layers():
+    h = C.c_void_p()
+    for kw in (dict(algo=B.CG_ALGO_TENSOR),                                  # fp32
+               dict(algo=B.CG_ALGO_TENSOR, in_dtype=B.CG_BF16, out_dtype=B.CG_BF16, c_in=24,
+                    c_out=16)):                                              # c_p = 6 channels
+        d = _desc(**kw)
+        assert B.lib().cg_conv_create(C.byref(h), C.byref(d)) == 2           # CG_ERR_UNSUPPORTED
+
+
+def test_null_handle_calls_are_safe():
+    lib = B.lib()
+    assert lib.cg_conv_workspace_bytes(None) == 0
+    assert lib.cg_conv_host_staging_bytes(None) == 0
+    assert lib.cg_conv_launches_per_forward(None) == 0
+    assert lib.cg_conv_uses_tensor_cores(None) == 0
+    lib.cg_conv_destroy(None)
+    st = B.CgStats()
+    assert lib.cg_conv_stats(None, C.byref(st), None) == 1
+    bn = B.CgBnParams()
+    assert lib.cg_conv_forward(None, None, None, None, C.byref(bn), None, None, None, None, None,
+                               0, None) == 1
+
+
+def test_create_without_a_device_reports_cuda_error():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    h = C.c_void_p()
+    d = _desc()
+    assert B.lib().cg_conv_create(C.byref(h), C.byref(d)) == 5               # CG_ERR_CUDA
+    with pytest.raises(B.CgError):
+        B.cg_conv_create(d)
