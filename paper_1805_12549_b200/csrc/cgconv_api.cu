@@ -14,7 +14,6 @@ struct cg_conv_s {
   cg::TcPlan plan;
   int device;
   unsigned long long* counters;   // device, cg::CNT_SLOTS entries
-  long long calls;
   cg::TcMaps maps;                // tensor maps cached for the last set of pointers
 };
 
@@ -97,7 +96,6 @@ cg_status cg_conv_create(cg_conv_t* out, const cg_conv_desc* desc) {
   if (!h) return CG_ERR_INVALID_ARG;
   h->desc = *desc;
   h->L = make_dims(*desc);
-  h->calls = 0;
   h->counters = nullptr;
   std::memset(&h->maps, 0, sizeof(h->maps));
   const bool tc_ok = cg::tc_plan(h->L, desc->in_dtype, desc->cond_mode, &h->plan);
@@ -157,7 +155,6 @@ cg_status cg_conv_forward(cg_conv_t h, const void* x, const void* w_base, const 
                             mask_out, nullptr, 0, h->counters, stream);
   }
   if (err != 0) return CG_ERR_CUDA;
-  h->calls += 1;
   return CG_OK;
 }
 
@@ -232,19 +229,20 @@ cg_status cg_conv_stats(cg_conv_t h, cg_stats* out, void* cuda_stream) {
   const cg::LayerDims& L = h->L;
   const long long k2 = (long long)L.kh * L.kw;
   std::memset(out, 0, sizeof(*out));
-  out->calls = h->calls;
-  out->outputs = h->calls * L.m * L.c_out;
+  out->calls = (int64_t)c[cg::CNT_CALLS];
+  out->outputs = out->calls * L.m * L.c_out;
   out->active = (int64_t)c[cg::CNT_ACTIVE];
   out->dense_macs = out->outputs * k2 * L.c_in;
   out->gated_macs = k2 * ((long long)L.c_p * out->outputs + (long long)L.c_r * out->active);
-  out->executed_macs = k2 * L.c_p * out->outputs + (int64_t)c[cg::CNT_EXEC_MACS];
+  // the tensor-core kernels count every MMA they issue (base path included, at tile
+  // granularity); the direct kernels execute exactly the method's count
+  out->executed_macs = h->use_tc ? (int64_t)c[cg::CNT_EXEC_MACS] : out->gated_macs;
   out->tiles_total = (int64_t)c[cg::CNT_TILES_TOTAL];
   out->tiles_skipped = (int64_t)c[cg::CNT_TILES_SKIPPED];
   out->rows_total = (int64_t)c[cg::CNT_ROWS_TOTAL];
   out->rows_active = (int64_t)c[cg::CNT_ROWS_ACTIVE];
   out->device_status = (int32_t)c[cg::CNT_STATUS];
   out->device_site = (int32_t)c[cg::CNT_SITE];
-  h->calls = 0;
   return out->device_status ? (cg_status)out->device_status : CG_OK;
 }
 

@@ -31,6 +31,7 @@ enum CounterSlot {
   CNT_ROWS_ACTIVE = 5,
   CNT_STATUS = 6,   // first non-zero cg_status reported by a kernel
   CNT_SITE = 7,     // id of the wait/check that reported it
+  CNT_CALLS = 8,    // forward passes executed (counted on the device: graph replays count)
   CNT_SLOTS = 16
 };
 

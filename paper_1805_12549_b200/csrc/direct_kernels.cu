@@ -130,10 +130,9 @@ direct_gated_conv_kernel(LayerDims L, const TIn* __restrict__ x, const TIn* __re
   if (!base_only) {
     if (lane == 0 && my_active) atomicAdd(&s_active, my_active);
     __syncthreads();
+    if (threadIdx.x == 0 && blockIdx.x == 0) atomicAdd(&counters[CNT_CALLS], 1ull);
     if (threadIdx.x == 0 && s_active) {
       atomicAdd(&counters[CNT_ACTIVE], s_active);
-      atomicAdd(&counters[CNT_EXEC_MACS],
-                s_active * (unsigned long long)(L.kh * L.kw * L.c_r));
     }
   }
 }
@@ -189,10 +188,9 @@ direct_gated_conv_i8_kernel(LayerDims L, const int8_t* __restrict__ x,
   if (!base_only) {
     if (lane == 0 && my_active) atomicAdd(&s_active, my_active);
     __syncthreads();
+    if (threadIdx.x == 0 && blockIdx.x == 0) atomicAdd(&counters[CNT_CALLS], 1ull);
     if (threadIdx.x == 0 && s_active) {
       atomicAdd(&counters[CNT_ACTIVE], s_active);
-      atomicAdd(&counters[CNT_EXEC_MACS],
-                s_active * (unsigned long long)(L.kh * L.kw * L.c_r));
     }
   }
 }

@@ -428,6 +428,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       // counters of this tile
       const uint32_t blocks = dense ? kAllBlocks : sh->blk_active;
       const unsigned long long k_p = (unsigned long long)taps * L.c_p, k_r = (unsigned long long)taps * L.c_r;
+      if (blockIdx.x == 0) atomicAdd(&prm.counters[CNT_CALLS], 1ull);
       atomicAdd(&prm.counters[CNT_ACTIVE], (unsigned long long)sh->n_active);
       atomicAdd(&prm.counters[CNT_TILES_TOTAL], (unsigned long long)kBlocks);
       atomicAdd(&prm.counters[CNT_TILES_SKIPPED], (unsigned long long)(kBlocks - __popc(blocks)));
@@ -571,37 +572,45 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
   (void)in_dtype; (void)residual; (void)workspace;
   if (!P.valid) return (int)cudaErrorInvalidValue;
   const void* wc_key = w_cond ? w_cond : w_base;
-  if (maps->key[0] != x || maps->key[1] != w_base || maps->key[2] != wc_key || maps->key[3] != y) {
+  TcMapSet* ms = nullptr;
+  for (int i = 0; i < TcMaps::kEntries; ++i) {
+    TcMapSet* c = &maps->set[i];
+    if (c->key[0] == x && c->key[1] == w_base && c->key[2] == wc_key && c->key[3] == y) { ms = c; break; }
+  }
+  if (!ms) {
+    ms = &maps->set[maps->next];
+    maps->next = (maps->next + 1) % TcMaps::kEntries;
+    ms->key[0] = nullptr;
     const int taps = L.kh * L.kw;
     {
       cuuint64_t dims[4] = {(cuuint64_t)L.c_in, (cuuint64_t)L.w, (cuuint64_t)L.h, (cuuint64_t)L.n};
       cuuint64_t str[3] = {(cuuint64_t)L.c_in * 2, (cuuint64_t)L.w * L.c_in * 2,
                            (cuuint64_t)L.h * L.w * L.c_in * 2};
       cuuint32_t box[4] = {64, (cuuint32_t)P.wp, (cuuint32_t)P.box_h, (cuuint32_t)P.ni};
-      if (!encode(&maps->x, const_cast<void*>(x), 4, dims, str, box)) return (int)cudaErrorInvalidValue;
+      if (!encode(&ms->x, const_cast<void*>(x), 4, dims, str, box)) return (int)cudaErrorInvalidValue;
     }
     {
       cuuint64_t dims[2] = {(cuuint64_t)taps * L.c_p, (cuuint64_t)L.c_out};
       cuuint64_t str[1] = {(cuuint64_t)taps * L.c_p * 2};
       cuuint32_t box[2] = {64, (cuuint32_t)P.nt};
-      if (!encode(&maps->wb, const_cast<void*>(w_base), 2, dims, str, box)) return (int)cudaErrorInvalidValue;
+      if (!encode(&ms->wb, const_cast<void*>(w_base), 2, dims, str, box)) return (int)cudaErrorInvalidValue;
     }
     if (L.c_r > 0) {
       cuuint64_t dims[2] = {(cuuint64_t)taps * L.c_r, (cuuint64_t)L.c_out};
       cuuint64_t str[1] = {(cuuint64_t)taps * L.c_r * 2};
       cuuint32_t box[2] = {64, (cuuint32_t)P.nt};
-      if (!encode(&maps->wc, const_cast<void*>(w_cond), 2, dims, str, box)) return (int)cudaErrorInvalidValue;
+      if (!encode(&ms->wc, const_cast<void*>(w_cond), 2, dims, str, box)) return (int)cudaErrorInvalidValue;
     } else {
-      maps->wc = maps->wb;
+      ms->wc = ms->wb;
     }
     {
       cuuint64_t dims[4] = {(cuuint64_t)L.c_out, (cuuint64_t)L.wo, (cuuint64_t)L.ho, (cuuint64_t)L.n};
       cuuint64_t str[3] = {(cuuint64_t)L.c_out * 2, (cuuint64_t)L.wo * L.c_out * 2,
                            (cuuint64_t)L.ho * L.wo * L.c_out * 2};
       cuuint32_t box[4] = {64, (cuuint32_t)P.wp, (cuuint32_t)P.out_box_h, (cuuint32_t)P.ni};
-      if (!encode(&maps->y, y, 4, dims, str, box)) return (int)cudaErrorInvalidValue;
+      if (!encode(&ms->y, y, 4, dims, str, box)) return (int)cudaErrorInvalidValue;
     }
-    maps->key[0] = x; maps->key[1] = w_base; maps->key[2] = wc_key; maps->key[3] = y;
+    ms->key[0] = x; ms->key[1] = w_base; ms->key[2] = wc_key; ms->key[3] = y;
   }
   TcParams prm;
   prm.L = L; prm.P = P; prm.bn = bn; prm.delta = delta; prm.mask = mask; prm.counters = counters;
@@ -614,7 +623,7 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
       if (e != cudaSuccess) return (int)e;
       attr128 = true;
     }
-    tc_gated_conv_kernel<128><<<grid, kThreads, P.smem_bytes, stream>>>(maps->x, maps->wb, maps->wc, maps->y, prm);
+    tc_gated_conv_kernel<128><<<grid, kThreads, P.smem_bytes, stream>>>(ms->x, ms->wb, ms->wc, ms->y, prm);
   } else {
     static bool attr64 = false;
     if (!attr64) {
@@ -622,7 +631,7 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
       if (e != cudaSuccess) return (int)e;
       attr64 = true;
     }
-    tc_gated_conv_kernel<64><<<grid, kThreads, P.smem_bytes, stream>>>(maps->x, maps->wb, maps->wc, maps->y, prm);
+    tc_gated_conv_kernel<64><<<grid, kThreads, P.smem_bytes, stream>>>(ms->x, ms->wb, ms->wc, ms->y, prm);
   }
   return (int)cudaGetLastError();
 }

@@ -33,9 +33,17 @@ struct TcPlan {
   unsigned off_a, off_b, off_y, off_consts, off_bar, smem_bytes;
 };
 
-struct TcMaps {
+struct TcMapSet {
   const void* key[4];   // x, w_base, w_cond, y the maps below were encoded for
   CUtensorMap x, wb, wc, y;
+};
+
+// Small cache of encoded tensor maps, so that callers that rotate a few buffers do not pay
+// four cuTensorMapEncodeTiled calls per forward.
+struct TcMaps {
+  static constexpr int kEntries = 8;
+  TcMapSet set[kEntries];
+  int next;
 };
 
 bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan);
