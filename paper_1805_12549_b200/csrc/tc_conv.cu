@@ -1,25 +1,33 @@
-// Channel-gated convolution on tcgen05 tensor cores: one fused kernel per layer.
+// Channel-gated convolution on tcgen05 tensor cores: one persistent fused kernel per layer.
 //
-// "Shifted-window" implicit GEMM (stride-1, k = 2*pad+1 convolutions).  A CTA owns a tile of up
-// to 128 output pixels that are whole image rows (or whole small images) and NT output
+// "Shifted-window" implicit GEMM (stride-1, k = 2*pad+1 convolutions).  A job is a tile of up
+// to 128 output pixels that are whole image rows (or whole small images) times NT output
 // channels.  The input patch of the tile -- the rows it needs plus the zero padding, which TMA
-// out-of-bounds fill provides -- is loaded ONCE per 64-channel chunk into shared memory as
+// out-of-bounds fill provides -- is loaded once per 64-channel chunk into shared memory as
 // [pixel][64 channels] rows of 128 bytes (128-byte swizzle).  Rows are laid out with pitch
 // W+pad, so that the right padding of one image row is the left padding of the next; then the
-// A operand of filter tap (r,s) is simply the same buffer read from row r*(W+pad)+s onwards:
-// output pixel i reads patch pixel i + r*(W+pad) + s.  Nine MMAs per K-slice reuse one patch;
-// only the weights stream through a TMA ring.
+// A operand of filter tap (r,s) is the same buffer read from row r*(W+pad)+s onwards: output
+// pixel i reads patch pixel i + r*(W+pad) + s.  All k*k taps reuse one patch load.
 //
-// Per tile, following the paper's block (Section 3.1, Eq. 1-3, Section 4):
+// Per job, following the paper's block (Section 3.1, Eq. 1-3, Section 4):
 //   1. base path   P = W_p * x_p : MMAs over the base channels, fp32 accumulator in TMEM;
-//   2. gate        d = (P >= t[c]) read from TMEM by the epilogue warps -> mask words, counts,
-//                  y_base = f(BN1(P)) staged in shared memory;
-//   3. conditional R = W_r * x_r accumulated ONTO P in the same TMEM columns, only for the
-//                  64-channel column blocks in which a gate fired (whole tile skipped if none);
-//   4. combine     where d = 1 the staged value is replaced by f(BN2(P+R)); one TMA store.
+//   2. gate        d = (P >= t[c]) read from TMEM by the epilogue warps -> mask words, counts;
+//   3. conditional R = W_r * x_r into a second TMEM accumulator, only for the 64-channel column
+//                  blocks in which a gate fired; its patch chunks and weight tiles are not even
+//                  loaded for tiles where none fired;
+//   4. combine     y = f(BN1(P)) where d = 0, f(BN2(P+R)) where d = 1, staged in shared memory
+//                  and written by one TMA store per 64 channels.
 //
-// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM), warps 2-5 = epilogue.
-// Every mbarrier wait is bounded; on expiry the CTA records CG_ERR_DEVICE_TIMEOUT and leaves.
+// The CTA is persistent (one per SM) and software-pipelined over its jobs:
+//   MMA issue order      base(0) | base(1) cond(0) | base(2) cond(1) | ...
+//   epilogue order       gate(0) | gate(1) combine(0) | gate(2) combine(1) | ...
+// so the tensor pipe works on the next tile's base path while the gate of the current tile is
+// being evaluated.  TMEM holds two job slots of (P, R) accumulators: 4*NT columns.
+// Weights stay resident in shared memory when they fit, otherwise they stream through a ring.
+//
+// Warp roles: 0 = patch (A) producer, 1 = MMA issuer (owns TMEM), 2 = weight (B) producer,
+// 3-10 = epilogue.  Every mbarrier wait is bounded; on expiry the CTA records
+// CG_ERR_DEVICE_TIMEOUT with the id of the wait and leaves.
 #include <cstring>
 
 #include "ptx.cuh"
@@ -29,9 +37,12 @@ namespace cg {
 
 namespace {
 
-constexpr int kThreads = 192;
-constexpr int kBM = 128;            // MMA M: patch rows per tile
-constexpr int kSpinLimit = 1 << 22; // try_wait polls before a wait gives up
+constexpr int kThreads = 352;       // 3 single-role warps + 8 epilogue warps
+constexpr int kEpiThread0 = 96;     // first epilogue thread
+constexpr int kEpiThreads = 256;
+constexpr int kBM = 128;            // MMA M: patch rows per job
+constexpr int kSpinLimit = 1 << 21; // try_wait polls (each up to ~2 us) before a wait gives up
+constexpr int kMaxWTiles = 192;     // weight tiles per job, both phases
 
 struct TcParams {
   LayerDims L;
@@ -42,68 +53,241 @@ struct TcParams {
   unsigned long long* counters;
 };
 
-// One weight tile of the ring: 64 K-elements of NT output channels.
+// One weight tile: 64 K-elements of NT output channels.
 struct WTile {
   int x;        // K coordinate in the weight matrix
-  int chunk;    // patch buffer it multiplies
-  int t0, ntap; // filter taps covered
-  int a_k0;     // first 16-element K step inside the patch row
-  int nks;      // K steps per tap
-  int b_step;   // K steps between consecutive taps inside the weight tile
+  int chunk;    // input-channel chunk (64 channels) it multiplies
 };
 
+// Weight tiles in the order the MMA issuer consumes them.  Base path: chunk-major, one tile
+// per tap when c_p >= 64; when c_p < 64 a tile covers 64/c_p taps of chunk 0.  Conditional
+// path: chunk-major, one tile per tap; when c_p < 64 chunk 0 comes first with the K slices
+// behind the base channels.
 __device__ __forceinline__ WTile base_tile(const LayerDims& L, int bt) {
   const int taps = L.kh * L.kw;
-  WTile w;
   if (L.c_p >= 64) {
     const int q = bt / taps, t = bt - q * taps;
-    w = {t * L.c_p + 64 * q, q, t, 1, 0, 4, 0};
-  } else {
-    const int tpt = 64 / L.c_p;
-    const int t0 = bt * tpt;
-    w = {bt * 64, 0, t0, min(tpt, taps - t0), 0, L.c_p / 16, L.c_p / 16};
+    return {t * L.c_p + 64 * q, q};
   }
-  return w;
+  return {bt * 64, 0};
 }
 
 __device__ __forceinline__ WTile cond_tile(const LayerDims& L, int bt) {
   const int taps = L.kh * L.kw;
-  WTile w;
   if (L.c_p >= 64) {
     const int q = L.c_p / 64 + bt / taps, t = bt % taps;
-    w = {t * L.c_r + 64 * q - L.c_p, q, t, 1, 0, 4, 0};
-  } else if (bt < taps) {
-    w = {bt * L.c_r, 0, bt, 1, L.c_p / 16, 4 - L.c_p / 16, 0};
-  } else {
-    const int b2 = bt - taps;
-    const int q = 1 + b2 / taps, t = b2 % taps;
-    w = {t * L.c_r + 64 * q - L.c_p, q, t, 1, 0, 4, 0};
+    return {t * L.c_r + 64 * q - L.c_p, q};
   }
-  return w;
+  if (bt < taps) return {bt * L.c_r, 0};
+  const int b2 = bt - taps;
+  const int q = 1 + b2 / taps, t = b2 % taps;
+  return {t * L.c_r + 64 * q - L.c_p, q};
 }
 
 struct Shared {
-  uint64_t a_full[8];
-  uint64_t b_full[8];
-  uint64_t b_empty[8];
-  uint64_t base_done, gate_done, cond_done;
+  uint64_t a_full[8], a_empty[8];
+  uint64_t b_full[8], b_empty[8];
+  uint64_t w_ready;
+  uint64_t base_done[2], gate_done[2], cond_done[2], acc_free[2];
   uint32_t tmem_base;
-  uint32_t blk_active;      // bit b: a gate fired in column block b (64 channels)
   uint32_t abort_flag;
-  uint32_t n_active, n_rows_valid, n_rows_active;
+  uint32_t warp_blk[2][8];   // per job slot, per epilogue warp: column blocks with a firing gate
 };
 
-__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Shared* sh,
-                                         unsigned long long* counters, int site) {
+struct Ctx {
+  Shared* sh;
+  unsigned long long* counters;
+};
+
+// Bounded wait.  The first poll is inline; the loop lives in one out-of-line copy so that the
+// role loops stay small.  Each poll parks the thread in hardware for up to ~2 us, so the bound
+// is a few seconds; a CTA that already gave up elsewhere is noticed within a few polls.
+__device__ __noinline__ bool wait_bar_slow(Shared* sh, unsigned long long* counters, uint64_t* bar,
+                                           uint32_t parity, int site) {
   for (int i = 0; i < kSpinLimit; ++i) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
-    if ((i & 1023) == 1023 && *(volatile uint32_t*)&sh->abort_flag) return false;
+    if ((i & 15) == 15 && *(volatile uint32_t*)&sh->abort_flag) return false;
   }
   if (atomicCAS(&counters[CNT_STATUS], 0ull, (unsigned long long)CG_ERR_DEVICE_TIMEOUT) == 0ull)
     atomicExch(&counters[CNT_SITE], (unsigned long long)site);
   atomicExch(&sh->abort_flag, 1u);
   return false;
 }
+
+__device__ __forceinline__ bool wait_bar(const Ctx& cx, uint64_t* bar, uint32_t parity, int site) {
+  if (ptx::mbar_try_wait(bar, parity, 0u)) return true;
+  return wait_bar_slow(cx.sh, cx.counters, bar, parity, site);
+}
+
+__device__ __forceinline__ uint32_t slot_blocks(const Shared* sh, int slot) {
+  const volatile uint32_t* w = sh->warp_blk[slot];
+  return w[0] | w[1] | w[2] | w[3] | w[4] | w[5] | w[6] | w[7];
+}
+
+// MMA issue for one CTA.  The whole warp runs this code convergently and one lane's tcgen05
+// instructions are predicated on, so addresses stay warp-uniform and there is no branch between
+// two MMAs: for 3x3 kernels the taps and K steps are fully unrolled with immediate descriptor
+// offsets.  (The issuing lane cannot hide latency: every branch, instruction-cache miss or
+// dependent scalar instruction between two MMAs is tensor idle time.)  Weight tiles are
+// visited in the order base_tile()/cond_tile() enumerate them, which is the order the weight
+// producer loads them.
+template <int NT>
+struct MmaIssuer {
+  Shared* sh;
+  Ctx cx;
+  uint32_t issue;                        // 1 on the issuing lane
+  uint32_t desc_hi;                      // upper descriptor word (see ptx::smem_desc)
+  uint32_t a_base_lo, b_base_lo;         // lower descriptor words of the ring bases
+  uint32_t patch_lo, wtile_lo, row_lo;   // buffer sizes / one patch pixel row, in 16-byte units
+  int resident, na, nb, kp16, chunks, base_chunks, base_tiles, kh, kw;
+  int as, bs;                            // ring slots and the parities of their "full" barriers
+  uint32_t apar, bpar;
+  // per phase
+  uint32_t d_tmem, a_lo, b_lo, acc, blk_off_d, blk_off_b;
+  int a_held, b_held;
+  bool ok;
+
+  __device__ __forceinline__ void init(Shared* sh_, const Ctx& cx_, const uint8_t* s_a,
+                                       const uint8_t* s_b, const TcPlan& P, const LayerDims& L,
+                                       int lane) {
+    sh = sh_; cx = cx_;
+    issue = lane == 0 ? 1u : 0u;
+    // descriptor words: upper = 8-row groups 1024 bytes apart, 128-byte swizzle, version 1;
+    // lower = (address >> 4) | (1 << 16)
+    desc_hi = (uint32_t)(ptx::smem_desc(0, 1024, 2) >> 32);
+    a_base_lo = (ptx::smem_u32(s_a) >> 4) | 0x10000u;
+    b_base_lo = (ptx::smem_u32(s_b) >> 4) | 0x10000u;
+    patch_lo = (uint32_t)P.patch_bytes >> 4;
+    wtile_lo = (uint32_t)(NT * 128) >> 4;
+    row_lo = (uint32_t)P.wp * 8u;
+    resident = P.resident; na = P.na; nb = P.nb; kp16 = L.c_p / 16; chunks = P.chunks;
+    base_chunks = P.base_chunks; base_tiles = P.base_tiles; kh = L.kh; kw = L.kw;
+    as = 0; bs = 0; apar = 0; bpar = 0;
+    a_held = 0; b_held = 0; ok = true;
+  }
+  template <bool ALL>
+  __device__ __forceinline__ void mma(uint32_t al, uint32_t bl) {
+    const uint64_t da = ((uint64_t)desc_hi << 32) | al;
+    if (ALL)
+      ptx::umma_bf16_if(issue, d_tmem, da, ((uint64_t)desc_hi << 32) | bl, ptx::idesc_bf16(kBM, NT), acc);
+    else   // exactly one of the two 64-channel column blocks
+      ptx::umma_bf16_if(issue, d_tmem + blk_off_d, da, ((uint64_t)desc_hi << 32) | (bl + blk_off_b),
+                        ptx::idesc_bf16(kBM, 64), acc);
+    acc = 1u;
+  }
+  __device__ __forceinline__ void acquire_a() {
+    ok = ok && wait_bar(cx, &sh->a_full[as], apar, 7);
+    a_held = as;
+    a_lo = a_base_lo + (uint32_t)as * patch_lo;
+    if (++as == na) { as = 0; apar ^= 1; }
+  }
+  __device__ __forceinline__ void release_a() { ptx::umma_commit_if(issue, &sh->a_empty[a_held]); }
+  template <bool RES>
+  __device__ __forceinline__ void acquire_b() {
+    if (!RES) {
+      ok = ok && wait_bar(cx, &sh->b_full[bs], bpar, 8);
+      b_held = bs;
+      b_lo = b_base_lo + (uint32_t)bs * wtile_lo;
+      if (++bs == nb) { bs = 0; bpar ^= 1; }
+    }
+  }
+  template <bool RES>
+  __device__ __forceinline__ void release_b() {
+    if (RES) b_lo += wtile_lo;
+    else ptx::umma_commit_if(issue, &sh->b_empty[b_held]);
+  }
+  // K steps [KS0, KS1) of every tap of the next chunk in the ring, one weight tile per tap
+  template <bool RES, bool ALL, int KS0, int KS1>
+  __device__ __forceinline__ void chunk_taps() {
+    acquire_a();
+    if (kh == 3 && kw == 3) {
+#pragma unroll
+      for (int r = 0; r < 3; ++r) {
+#pragma unroll
+        for (int sx = 0; sx < 3; ++sx) {
+          acquire_b<RES>();
+          if (!ok) return;
+          const uint32_t a_t = a_lo + (uint32_t)r * row_lo + (uint32_t)sx * 8u;
+#pragma unroll
+          for (int ks = KS0; ks < KS1; ++ks) mma<ALL>(a_t + ks * 2, b_lo + (ks - KS0) * 2);
+          release_b<RES>();
+        }
+      }
+    } else {
+      uint32_t a_r = a_lo;
+      for (int r = 0; r < kh; ++r, a_r += row_lo) {
+        for (int sx = 0; sx < kw; ++sx) {
+          acquire_b<RES>();
+          if (!ok) return;
+          const uint32_t a_t = a_r + (uint32_t)sx * 8u;
+#pragma unroll
+          for (int ks = KS0; ks < KS1; ++ks) mma<ALL>(a_t + ks * 2, b_lo + (ks - KS0) * 2);
+          release_b<RES>();
+        }
+      }
+    }
+    release_a();
+  }
+  // base path when c_p < 64: the first KP K steps of chunk 0; a weight tile covers 4/KP taps
+  template <bool RES, bool ALL, int KP>
+  __device__ __forceinline__ void base_small() {
+    constexpr int TPT = 4 / KP;
+    acquire_a();
+    if (kh == 3 && kw == 3) {
+#pragma unroll
+      for (int t = 0; t < 9; ++t) {
+        if (t % TPT == 0) acquire_b<RES>();
+        if (!ok) return;
+        const uint32_t a_t = a_lo + (uint32_t)(t / 3) * row_lo + (uint32_t)(t % 3) * 8u;
+#pragma unroll
+        for (int ks = 0; ks < KP; ++ks) mma<ALL>(a_t + ks * 2, b_lo + ((t % TPT) * KP + ks) * 2);
+        if (t % TPT == TPT - 1 || t == 8) release_b<RES>();
+      }
+    } else {
+      int in_tile = 0;
+      uint32_t a_r = a_lo;
+      for (int r = 0; r < kh; ++r, a_r += row_lo) {
+        for (int sx = 0; sx < kw; ++sx) {
+          if (in_tile == 0) acquire_b<RES>();
+          if (!ok) return;
+          const uint32_t a_t = a_r + (uint32_t)sx * 8u;
+#pragma unroll
+          for (int ks = 0; ks < KP; ++ks) mma<ALL>(a_t + ks * 2, b_lo + (uint32_t)(in_tile * KP + ks) * 2u);
+          if (++in_tile == TPT) { release_b<RES>(); in_tile = 0; }
+        }
+      }
+      if (in_tile != 0) release_b<RES>();
+    }
+    release_a();
+  }
+  template <bool RES, bool ALL>
+  __device__ __forceinline__ void phase(bool cond) {
+    if (kp16 >= 4) {
+      const int q0 = cond ? base_chunks : 0, q1 = cond ? chunks : base_chunks;
+      for (int q = q0; q < q1 && ok; ++q) chunk_taps<RES, ALL, 0, 4>();
+    } else if (!cond) {
+      if (kp16 == 1) base_small<RES, ALL, 1>(); else base_small<RES, ALL, 2>();
+    } else {
+      // conditional channels of chunk 0 (K steps kp16..3), then the remaining chunks
+      if (kp16 == 1) chunk_taps<RES, ALL, 1, 4>(); else chunk_taps<RES, ALL, 2, 4>();
+      for (int q = 1; q < chunks && ok; ++q) chunk_taps<RES, ALL, 0, 4>();
+    }
+  }
+  // base or conditional MMAs of one job into the accumulator at d; `blocks` = column blocks to
+  // compute (all of them for the base path)
+  __device__ __forceinline__ bool run_phase(uint32_t d, bool cond, uint32_t blocks) {
+    constexpr uint32_t kAll = (1u << (NT / 64)) - 1u;
+    d_tmem = d;
+    acc = 0u;   // the first K step overwrites the accumulator
+    ok = true;
+    b_lo = b_base_lo + (cond ? (uint32_t)base_tiles * wtile_lo : 0u);   // resident tiles
+    blk_off_d = blocks == 2u ? 64u : 0u;
+    blk_off_b = blocks == 2u ? (64u * 128u / 16u) : 0u;
+    if (blocks == kAll) { if (resident) phase<true, true>(cond); else phase<false, true>(cond); }
+    else { if (resident) phase<true, false>(cond); else phase<false, false>(cond); }
+    return ok;
+  }
+};
 
 template <int NT>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -124,49 +308,65 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   float* s_b1 = s_a1 + NT;
   float* s_a2 = s_b1 + NT;
   float* s_b2 = s_a2 + NT;
+  uint32_t* s_mask = (uint32_t*)(smem + P.off_mask);       // [2][128][NT/32]
+  int* s_wx = (int*)(smem + P.off_tables);                 // [base_tiles + cond_tiles] K coordinates
   Shared* sh = (Shared*)(smem + P.off_bar);
+  const Ctx cx{sh, prm.counters};
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // jobs of this CTA: a fixed column tile, every `groups`-th row tile
   const int tile_n = blockIdx.x % P.tiles_n;
-  const int tile_m = blockIdx.x / P.tiles_n;
-  int n0, h0;
-  if (P.images_mode) { n0 = tile_m * P.ni; h0 = 0; }
-  else { n0 = tile_m / P.tiles_per_image; h0 = (tile_m - n0 * P.tiles_per_image) * P.r; }
+  const int group = blockIdx.x / P.tiles_n;
+  const int groups = gridDim.x / P.tiles_n;
+  const int jobs = group < P.tiles_m ? (P.tiles_m - group + groups - 1) / groups : 0;
   const int taps = L.kh * L.kw;
   const bool dense = (P.cond_mode == CG_COND_DENSE);
-  constexpr int kBlocks = NT / 64;                       // column blocks of the conditional path
+  const bool has_cond = P.cond_tiles > 0;
+  const int cond_first_chunk = L.c_p >= 64 ? P.base_chunks : 0;
+  constexpr int kBlocks = NT / 64;
   constexpr uint32_t kAllBlocks = (1u << kBlocks) - 1u;
-  const uint32_t b_tile_bytes = NT * 128;
+  constexpr int kWords = NT / 32;
+  const uint32_t w_tile_bytes = NT * 128;
+  const uint32_t patch_tx = (uint32_t)P.box_pixels * 128u;
+
+  auto job_origin = [&](int j, int& n0, int& h0) {
+    const int tile_m = group + j * groups;
+    if (P.images_mode) { n0 = tile_m * P.ni; h0 = 0; }
+    else { n0 = tile_m / P.tiles_per_image; h0 = (tile_m - n0 * P.tiles_per_image) * P.r; }
+  };
 
   // ---------------------------------------------------------------- setup
   if (threadIdx.x == 0) {
-    for (int i = 0; i < P.chunks; ++i) ptx::mbar_init(&sh->a_full[i], 1);
-    for (int i = 0; i < P.stages; ++i) { ptx::mbar_init(&sh->b_full[i], 1); ptx::mbar_init(&sh->b_empty[i], 1); }
-    ptx::mbar_init(&sh->base_done, 1);
-    ptx::mbar_init(&sh->gate_done, 128);
-    ptx::mbar_init(&sh->cond_done, 1);
-    sh->blk_active = 0; sh->abort_flag = 0; sh->n_active = 0; sh->n_rows_valid = 0; sh->n_rows_active = 0;
+    for (int i = 0; i < P.na; ++i) { ptx::mbar_init(&sh->a_full[i], 1); ptx::mbar_init(&sh->a_empty[i], 1); }
+    for (int i = 0; i < P.nb; ++i) { ptx::mbar_init(&sh->b_full[i], 1); ptx::mbar_init(&sh->b_empty[i], 1); }
+    ptx::mbar_init(&sh->w_ready, 1);
+    for (int i = 0; i < 2; ++i) {
+      ptx::mbar_init(&sh->base_done[i], 1);
+      ptx::mbar_init(&sh->gate_done[i], kEpiThreads);
+      ptx::mbar_init(&sh->cond_done[i], 1);
+      ptx::mbar_init(&sh->acc_free[i], kEpiThreads);
+    }
+    sh->abort_flag = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&map_x); ptx::prefetch_tensormap(&map_wb);
     ptx::prefetch_tensormap(&map_wc); ptx::prefetch_tensormap(&map_y);
   }
-  if (warp == 1) ptx::tmem_alloc(&sh->tmem_base, NT);
-  if (warp >= 2) {
-    // zero the patch rows behind the TMA box: they stand for the last row's right padding
+  if (warp == 1) ptx::tmem_alloc(&sh->tmem_base, 4 * NT);
+  if (warp >= 3) {
+    const int et = threadIdx.x - kEpiThread0;
+    // zero the rows behind the TMA box of every patch buffer: they stand for the right padding
+    // of the last patch row and are never written again
     const int tail0 = P.box_pixels * 128, tail1 = P.patch_rows * 128;
-    for (int q = 0; q < P.chunks; ++q) {
+    for (int q = 0; q < P.na; ++q) {
       uint8_t* base = s_a + (size_t)q * P.patch_bytes;
-      for (int o = tail0 + (threadIdx.x - 64) * 16; o < tail1; o += 128 * 16)
-        *(uint4*)(base + o) = make_uint4(0, 0, 0, 0);
+      for (int o = tail0 + et * 16; o < tail1; o += kEpiThreads * 16) *(uint4*)(base + o) = make_uint4(0, 0, 0, 0);
     }
-    for (int c = threadIdx.x - 64; c < NT; c += 128) {
-      const int cg_ = tile_n * NT + c;
-      if (cg_ < L.c_out) {
-        const ChannelConsts k = fold_channel(prm.bn, prm.delta, L.eps, cg_);
-        s_t[c] = k.t; s_a1[c] = k.a1; s_b1[c] = k.b1; s_a2[c] = k.a2; s_b2[c] = k.b2;
-      } else {
-        s_t[c] = __int_as_float(0x7f800000); s_a1[c] = 0.f; s_b1[c] = 0.f; s_a2[c] = 0.f; s_b2[c] = 0.f;
-      }
+    // K coordinate of every weight tile, for the weight producer
+    for (int bt = et; bt < P.base_tiles + P.cond_tiles; bt += kEpiThreads)
+      s_wx[bt] = (bt < P.base_tiles ? base_tile(L, bt) : cond_tile(L, bt - P.base_tiles)).x;
+    for (int c = et; c < NT; c += kEpiThreads) {
+      const ChannelConsts k = fold_channel(prm.bn, prm.delta, L.eps, tile_n * NT + c);
+      s_t[c] = k.t; s_a1[c] = k.a1; s_b1[c] = k.b1; s_a2[c] = k.a2; s_b2[c] = k.b2;
     }
     ptx::fence_proxy_async();
   }
@@ -176,273 +376,275 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   const uint32_t tmem = sh->tmem_base;
 
   if (warp == 0) {
-    // ============================================================ TMA producer
-    if (lane == 0) {
-      do {
-        const uint32_t patch_tx = (uint32_t)P.box_pixels * 128u;
-        for (int q = 0; q < P.base_chunks; ++q) {
-          ptx::mbar_expect_tx(&sh->a_full[q], patch_tx);
-          ptx::tma_load_4d(s_a + (size_t)q * P.patch_bytes, &map_x, &sh->a_full[q], q * 64, -L.pad,
+    // ============================================================ patch (A) producer
+    // Loads chunks in the order the MMA issuer consumes them: base(0) | base(1) cond(0) | ...
+    if (lane == 0 && jobs > 0) {
+      int as = 0;              // ring slot and the parity of its "empty" barrier
+      uint32_t apar = 1;
+      bool ok = true;
+      auto load_chunks = [&](int j, int q0, int q1) {
+        int n0, h0;
+        job_origin(j, n0, h0);
+        for (int q = q0; q < q1 && ok; ++q) {
+          ok = wait_bar(cx, &sh->a_empty[as], apar, 1);
+          if (!ok) return;
+          ptx::mbar_expect_tx(&sh->a_full[as], patch_tx);
+          ptx::tma_load_4d(s_a + (size_t)as * P.patch_bytes, &map_x, &sh->a_full[as], q * 64, -L.pad,
                            h0 - L.pad, n0);
+          if (++as == P.na) { as = 0; apar ^= 1; }
         }
-        if (dense) {
-          for (int q = P.base_chunks; q < P.chunks; ++q) {
-            ptx::mbar_expect_tx(&sh->a_full[q], patch_tx);
-            ptx::tma_load_4d(s_a + (size_t)q * P.patch_bytes, &map_x, &sh->a_full[q], q * 64,
-                             -L.pad, h0 - L.pad, n0);
+      };
+      for (int j = 0; j <= jobs && ok; ++j) {
+        if (j < jobs) load_chunks(j, 0, P.base_chunks);
+        if (j >= 1 && has_cond && ok) {
+          const int jj = j - 1;
+          uint32_t blocks = kAllBlocks;
+          if (!dense) {
+            ok = wait_bar(cx, &sh->gate_done[jj & 1], (jj >> 1) & 1, 2);
+            if (!ok) break;
+            blocks = slot_blocks(sh, jj & 1);
           }
+          if (blocks) load_chunks(jj, cond_first_chunk, P.chunks);
         }
-        int it = 0;
+      }
+    }
+    __syncwarp();
+  } else if (warp == 2) {
+    // ============================================================ weight (B) producer
+    if (lane == 0 && jobs > 0) {
+      if (P.resident) {
+        const uint32_t total = (uint32_t)(P.base_tiles + P.cond_tiles) * w_tile_bytes;
+        ptx::mbar_expect_tx(&sh->w_ready, total);
+        for (int bt = 0; bt < P.base_tiles + P.cond_tiles; ++bt)
+          ptx::tma_load_2d(s_b + (size_t)bt * w_tile_bytes, bt < P.base_tiles ? &map_wb : &map_wc,
+                           &sh->w_ready, s_wx[bt], tile_n * NT);
+      } else {
+        int bs = 0;            // ring slot and the parity of its "empty" barrier
+        uint32_t bpar = 1;
         bool ok = true;
-        for (int bt = 0; bt < P.base_tiles && ok; ++bt, ++it) {
-          const int s = it % P.stages;
-          ok = wait_bar(&sh->b_empty[s], ((it / P.stages) & 1) ^ 1, sh, prm.counters, 1);
-          if (!ok) break;
-          const WTile w = base_tile(L, bt);
-          ptx::mbar_expect_tx(&sh->b_full[s], b_tile_bytes);
-          ptx::tma_load_2d(s_b + (size_t)s * b_tile_bytes, &map_wb, &sh->b_full[s], w.x, tile_n * NT);
-        }
-        if (!ok || P.cond_tiles == 0) break;
-        uint32_t blocks = kAllBlocks;
-        if (!dense) {
-          if (!wait_bar(&sh->gate_done, 0, sh, prm.counters, 2)) break;
-          blocks = *(volatile uint32_t*)&sh->blk_active;
-          if (blocks == 0) break;
-          for (int q = P.base_chunks; q < P.chunks; ++q) {
-            ptx::mbar_expect_tx(&sh->a_full[q], patch_tx);
-            ptx::tma_load_4d(s_a + (size_t)q * P.patch_bytes, &map_x, &sh->a_full[q], q * 64,
-                             -L.pad, h0 - L.pad, n0);
+        auto load_tiles = [&](const CUtensorMap* map, int t0, int n) {
+          for (int bt = 0; bt < n && ok; ++bt) {
+            ok = wait_bar(cx, &sh->b_empty[bs], bpar, 3);
+            if (!ok) return;
+            ptx::mbar_expect_tx(&sh->b_full[bs], w_tile_bytes);
+            ptx::tma_load_2d(s_b + (size_t)bs * w_tile_bytes, map, &sh->b_full[bs], s_wx[t0 + bt],
+                             tile_n * NT);
+            if (++bs == P.nb) { bs = 0; bpar ^= 1; }
+          }
+        };
+        for (int j = 0; j <= jobs && ok; ++j) {
+          if (j < jobs) load_tiles(&map_wb, 0, P.base_tiles);
+          if (j >= 1 && has_cond && ok) {
+            const int jj = j - 1;
+            uint32_t blocks = kAllBlocks;
+            if (!dense) {
+              ok = wait_bar(cx, &sh->gate_done[jj & 1], (jj >> 1) & 1, 4);
+              if (!ok) break;
+              blocks = slot_blocks(sh, jj & 1);
+            }
+            if (blocks) load_tiles(&map_wc, P.base_tiles, P.cond_tiles);
           }
         }
-        for (int bt = 0; bt < P.cond_tiles && ok; ++bt, ++it) {
-          const int s = it % P.stages;
-          ok = wait_bar(&sh->b_empty[s], ((it / P.stages) & 1) ^ 1, sh, prm.counters, 3);
-          if (!ok) break;
-          const WTile w = cond_tile(L, bt);
-          ptx::mbar_expect_tx(&sh->b_full[s], b_tile_bytes);
-          ptx::tma_load_2d(s_b + (size_t)s * b_tile_bytes, &map_wc, &sh->b_full[s], w.x, tile_n * NT);
-        }
-      } while (0);
+      }
     }
     __syncwarp();
   } else if (warp == 1) {
     // ============================================================ MMA issuer
-    if (lane == 0) {
-      do {
-        const uint32_t a_base = ptx::smem_u32(s_a);
-        const uint32_t b_base = ptx::smem_u32(s_b);
-        int it = 0;
-        bool ok = true;
-        uint32_t chunk_ready = 0;
-        uint32_t first = 1;
-        for (int bt = 0; bt < P.base_tiles && ok; ++bt, ++it) {
-          const WTile w = base_tile(L, bt);
-          if (!((chunk_ready >> w.chunk) & 1u)) {
-            ok = wait_bar(&sh->a_full[w.chunk], 0, sh, prm.counters, 4);
-            if (!ok) break;
-            chunk_ready |= 1u << w.chunk;
-          }
-          const int s = it % P.stages;
-          ok = wait_bar(&sh->b_full[s], (it / P.stages) & 1, sh, prm.counters, 5);
+    if (jobs > 0) {
+      MmaIssuer<NT> mi;
+      mi.init(sh, cx, s_a, s_b, P, L, lane);
+      bool ok = true;
+      if (P.resident) ok = wait_bar(cx, &sh->w_ready, 0, 6);
+      for (int j = 0; j <= jobs && ok; ++j) {
+        if (j < jobs) {
+          ok = wait_bar(cx, &sh->acc_free[j & 1], ((j >> 1) & 1) ^ 1, 9);
           if (!ok) break;
           ptx::tc_fence_after();
-          const uint32_t a_chunk = a_base + (uint32_t)w.chunk * P.patch_bytes;
-          const uint32_t b_stage = b_base + (uint32_t)s * b_tile_bytes;
-          for (int j = 0; j < w.ntap; ++j) {
-            const int t = w.t0 + j;
-            const uint32_t shift = (uint32_t)((t / L.kw) * P.wp + (t % L.kw)) * 128u;
-            for (int ks = 0; ks < w.nks; ++ks) {
-              const uint64_t da = ptx::smem_desc(a_chunk + shift + (uint32_t)(w.a_k0 + ks) * 32u, 1024, 2);
-              const uint64_t db = ptx::smem_desc(b_stage + (uint32_t)(j * w.b_step + ks) * 32u, 1024, 2);
-              ptx::umma_bf16(tmem, da, db, ptx::idesc_bf16(kBM, NT), first ? 0u : 1u);
-              first = 0;
-            }
-          }
-          ptx::umma_commit(&sh->b_empty[s]);
-        }
-        if (!ok) break;
-        ptx::umma_commit(&sh->base_done);
-        if (P.cond_tiles == 0) break;
-        // P must have been read by the gate before R is accumulated onto it
-        if (!wait_bar(&sh->gate_done, 0, sh, prm.counters, 6)) break;
-        ptx::tc_fence_after();
-        const uint32_t blocks = dense ? kAllBlocks : *(volatile uint32_t*)&sh->blk_active;
-        if (blocks == 0) break;
-        for (int bt = 0; bt < P.cond_tiles && ok; ++bt, ++it) {
-          const WTile w = cond_tile(L, bt);
-          if (!((chunk_ready >> w.chunk) & 1u)) {
-            ok = wait_bar(&sh->a_full[w.chunk], 0, sh, prm.counters, 7);
-            if (!ok) break;
-            chunk_ready |= 1u << w.chunk;
-          }
-          const int s = it % P.stages;
-          ok = wait_bar(&sh->b_full[s], (it / P.stages) & 1, sh, prm.counters, 8);
+          ok = mi.run_phase(tmem + (uint32_t)((j & 1) * 2 * NT), false, kAllBlocks);
           if (!ok) break;
-          ptx::tc_fence_after();
-          const uint32_t a_chunk = a_base + (uint32_t)w.chunk * P.patch_bytes;
-          const uint32_t b_stage = b_base + (uint32_t)s * b_tile_bytes;
-          const int t = w.t0;
-          const uint32_t shift = (uint32_t)((t / L.kw) * P.wp + (t % L.kw)) * 128u;
-          for (int ks = 0; ks < w.nks; ++ks) {
-            const uint32_t a_addr = a_chunk + shift + (uint32_t)(w.a_k0 + ks) * 32u;
-            const uint32_t b_addr = b_stage + (uint32_t)ks * 32u;
-            if (blocks == kAllBlocks) {
-              ptx::umma_bf16(tmem, ptx::smem_desc(a_addr, 1024, 2), ptx::smem_desc(b_addr, 1024, 2),
-                             ptx::idesc_bf16(kBM, NT), 1u);
-            } else {
-#pragma unroll
-              for (int b = 0; b < kBlocks; ++b) {
-                if ((blocks >> b) & 1u)
-                  ptx::umma_bf16(tmem + b * 64, ptx::smem_desc(a_addr, 1024, 2),
-                                 ptx::smem_desc(b_addr + b * 64 * 128, 1024, 2),
-                                 ptx::idesc_bf16(kBM, 64), 1u);
-              }
-            }
-          }
-          ptx::umma_commit(&sh->b_empty[s]);
+          ptx::umma_commit_if(mi.issue, &sh->base_done[j & 1]);
         }
-        if (!ok) break;
-        ptx::umma_commit(&sh->cond_done);
-      } while (0);
+        if (j >= 1) {
+          const int jj = j - 1;
+          if (has_cond) {
+            uint32_t blocks = kAllBlocks;
+            if (!dense) {
+              ok = wait_bar(cx, &sh->gate_done[jj & 1], (jj >> 1) & 1, 10);
+              if (!ok) break;
+              blocks = slot_blocks(sh, jj & 1);
+            }
+            if (blocks) ok = mi.run_phase(tmem + (uint32_t)((jj & 1) * 2 * NT + NT), true, blocks);
+            if (!ok) break;
+          }
+          ptx::umma_commit_if(mi.issue, &sh->cond_done[jj & 1]);
+        }
+      }
     }
     __syncwarp();
   } else {
-    // ============================================================ epilogue (128 threads)
+    // ============================================================ epilogue (8 warps)
+    // Warps w and w+4 share a TMEM lane quadrant and split its 32-column blocks between them.
     const int quad = warp & 3;
+    const int half = (warp - 3) >> 2;
     const int row = quad * 32 + lane;                      // TMEM lane = patch row i
-    const int et = threadIdx.x - 64;
-    // which output pixel is row i?
+    const int et = threadIdx.x - kEpiThread0;
     const int n_loc = P.images_mode ? row / P.ip : 0;
     const int rem = P.images_mode ? row - n_loc * P.ip : row;
     const int h_loc = rem / P.wp;
     const int w_out = rem - h_loc * P.wp;
-    const int rows_here = P.images_mode ? L.h : min(P.r, L.h - h0);
-    const bool valid = (w_out < L.w) && (h_loc < rows_here) && (n_loc < P.ni) && (n0 + n_loc < L.n);
-    const long long m = ((long long)(n0 + n_loc) * L.ho + (h0 + h_loc)) * L.wo + w_out;
-    const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16);
-    uint32_t words[NT / 32];
-    bool alive = true;
-    do {
-      if (!wait_bar(&sh->base_done, 0, sh, prm.counters, 9)) { alive = false; break; }
+    const uint32_t t_lane = tmem + ((uint32_t)(quad * 32) << 16);
+    unsigned long long st_active = 0, st_rows_valid = 0, st_rows_active = 0;
+    unsigned long long st_blocks_run = 0;                  // et == 0
+    bool ok = true;
+
+    // gate of job j: P -> mask words (global + stash), block activity flags
+    auto gate_pass = [&](int j) {
+      const int slot = j & 1;
+      ok = wait_bar(cx, &sh->base_done[slot], (j >> 1) & 1, 11);
+      if (!ok) return;
       ptx::tc_fence_after();
-      uint32_t my_active = 0;
+      int n0, h0;
+      job_origin(j, n0, h0);
+      const int rows_here = P.images_mode ? L.h : min(P.r, L.h - h0);
+      const bool valid = (w_out < L.w) && (h_loc < rows_here) && (n_loc < P.ni) && (n0 + n_loc < L.n);
+      const long long m = ((long long)(n0 + n_loc) * L.ho + (h0 + h_loc)) * L.wo + w_out;
       uint32_t my_blocks = 0;
 #pragma unroll
-      for (int cb = 0; cb < NT / 32; ++cb) {
+      for (int cc = 0; cc < kWords / 2; ++cc) {
+        const int cb = cc * 2 + half;
         uint32_t r[32];
-        ptx::tmem_ld32(t_row + cb * 32, r);
+        ptx::tmem_ld32(t_lane + (uint32_t)(slot * 2 * NT + cb * 32), r);
         uint32_t word = 0;
-        uint32_t packed[16];
 #pragma unroll
-        for (int j = 0; j < 32; j += 2) {
-          const int c = cb * 32 + j;
-          const float p0 = __uint_as_float(r[j]), p1 = __uint_as_float(r[j + 1]);
-          word |= (p0 >= s_t[c] ? 1u : 0u) << j;
-          word |= (p1 >= s_t[c + 1] ? 1u : 0u) << (j + 1);
-          float v0 = __fadd_rn(__fmul_rn(s_a1[c], p0), s_b1[c]);
-          float v1 = __fadd_rn(__fmul_rn(s_a1[c + 1], p1), s_b1[c + 1]);
-          if (L.relu) { v0 = v0 > 0.f ? v0 : 0.f; v1 = v1 > 0.f ? v1 : 0.f; }
-          const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
-          packed[j >> 1] = *(const uint32_t*)&h2;
+        for (int q = 0; q < 8; ++q) {
+          const float4 t4 = *(const float4*)(s_t + cb * 32 + q * 4);
+          word |= (__uint_as_float(r[q * 4 + 0]) >= t4.x ? 1u : 0u) << (q * 4 + 0);
+          word |= (__uint_as_float(r[q * 4 + 1]) >= t4.y ? 1u : 0u) << (q * 4 + 1);
+          word |= (__uint_as_float(r[q * 4 + 2]) >= t4.z ? 1u : 0u) << (q * 4 + 2);
+          word |= (__uint_as_float(r[q * 4 + 3]) >= t4.w ? 1u : 0u) << (q * 4 + 3);
         }
         if (!valid) word = 0;
-        words[cb] = word;
-        my_active += __popc(word);
+        s_mask[(slot * 128 + row) * kWords + cb] = word;
+        st_active += __popc(word);
         if (word) my_blocks |= 1u << (cb >> 1);
-        if (valid && prm.mask) prm.mask[m * L.words + tile_n * (NT / 32) + cb] = word;
+        if (valid && prm.mask) prm.mask[m * L.words + tile_n * kWords + cb] = word;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) my_blocks |= __shfl_xor_sync(0xffffffffu, my_blocks, o);
+      if (lane == 0) sh->warp_blk[slot][warp - 3] = my_blocks;
+      if (half == 0) {
+        const uint32_t row_valid = __ballot_sync(0xffffffffu, valid);
+        if (lane == 0) st_rows_valid += __popc(row_valid);
+      }
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(&sh->gate_done[slot]);
+    };
+
+    // combine of job j: y = f(BN1(P)) or f(BN2(P+R)) by mask bit, staged and stored
+    auto combine_pass = [&](int j) {
+      const int slot = j & 1;
+      ok = wait_bar(cx, &sh->gate_done[slot], (j >> 1) & 1, 12);   // every warp's flags and words
+      if (!ok) return;
+      const uint32_t blocks = !has_cond ? 0u : (dense ? kAllBlocks : slot_blocks(sh, slot));
+      if (half == 0) {
+        uint32_t any = 0;
+#pragma unroll
+        for (int cb = 0; cb < kWords; ++cb) any |= s_mask[(slot * 128 + row) * kWords + cb];
+        const uint32_t row_active = __ballot_sync(0xffffffffu, any != 0);
+        if (lane == 0) st_rows_active += __popc(row_active);
+      }
+      ok = wait_bar(cx, &sh->cond_done[slot], (j >> 1) & 1, 13);
+      if (!ok) return;
+      ptx::tc_fence_after();
+      if (et == 0) {
+        ptx::tma_store_wait_read();   // the previous store has finished reading the staging tile
+        st_blocks_run += __popc(blocks);
+      }
+      ptx::named_bar_sync(1, kEpiThreads);
+#pragma unroll
+      for (int cc = 0; cc < kWords / 2; ++cc) {
+        const int cb = cc * 2 + half;
+        const uint32_t word = s_mask[(slot * 128 + row) * kWords + cb];
+        uint32_t p[32], rr[32];
+        ptx::tmem_ld32(t_lane + (uint32_t)(slot * 2 * NT + cb * 32), p);
+        const bool have_r = ((blocks >> (cb >> 1)) & 1u) && __ballot_sync(0xffffffffu, word != 0) != 0;
+        if (have_r) {
+          ptx::tmem_ld32(t_lane + (uint32_t)(slot * 2 * NT + NT + cb * 32), rr);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) rr[i] = 0u;
+        }
         uint8_t* st = s_y + (size_t)(cb >> 1) * P.stage_rows * 128 + (size_t)row * 128;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          const int c16 = (cb & 1) * 4 + q;
-          *(uint4*)(st + ((c16 ^ (row & 7)) << 4)) =
-              make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
-        }
-      }
-      // tile-level bookkeeping
-      const uint32_t row_active = __ballot_sync(0xffffffffu, my_active != 0);
-      const uint32_t row_valid = __ballot_sync(0xffffffffu, valid);
-      uint32_t wa = my_active, wb_ = my_blocks;
+          uint32_t packed[4];
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        wa += __shfl_xor_sync(0xffffffffu, wa, o);
-        wb_ |= __shfl_xor_sync(0xffffffffu, wb_, o);
-      }
-      if (lane == 0) {
-        if (wa) atomicAdd(&sh->n_active, wa);
-        if (wb_) atomicOr(&sh->blk_active, wb_);
-        atomicAdd(&sh->n_rows_valid, __popc(row_valid));
-        atomicAdd(&sh->n_rows_active, __popc(row_active));
+          for (int e = 0; e < 4; ++e) {
+            const int jx = q * 8 + e * 2;
+            const int c = cb * 32 + jx;
+            const float2 a1 = *(const float2*)(s_a1 + c), b1 = *(const float2*)(s_b1 + c);
+            const float2 a2 = *(const float2*)(s_a2 + c), b2 = *(const float2*)(s_b2 + c);
+            const bool f0 = (word >> jx) & 1u, f1 = (word >> (jx + 1)) & 1u;
+            const float p0 = __uint_as_float(p[jx]), p1 = __uint_as_float(p[jx + 1]);
+            // Eq. 1: the full sum P+R where the gate fired, the partial sum elsewhere; then the
+            // batch norm of that path (Section 4) as one multiply and one add
+            const float s0 = f0 ? __fadd_rn(p0, __uint_as_float(rr[jx])) : p0;
+            const float s1 = f1 ? __fadd_rn(p1, __uint_as_float(rr[jx + 1])) : p1;
+            float v0 = __fadd_rn(__fmul_rn(f0 ? a2.x : a1.x, s0), f0 ? b2.x : b1.x);
+            float v1 = __fadd_rn(__fmul_rn(f1 ? a2.y : a1.y, s1), f1 ? b2.y : b1.y);
+            if (L.relu) { v0 = v0 > 0.f ? v0 : 0.f; v1 = v1 > 0.f ? v1 : 0.f; }
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
+            packed[e] = *(const uint32_t*)&h2;
+          }
+          const int c16 = (cb & 1) * 4 + q;
+          *(uint4*)(st + ((c16 ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        }
       }
       ptx::tc_fence_before();
-      ptx::mbar_arrive(&sh->gate_done);
-      if (P.cond_tiles > 0) {
-        // every epilogue thread needs the tile-wide block mask
-        if (!wait_bar(&sh->gate_done, 0, sh, prm.counters, 10)) { alive = false; break; }
-        const uint32_t blocks = dense ? kAllBlocks : *(volatile uint32_t*)&sh->blk_active;
-        if (blocks != 0) {
-          if (!wait_bar(&sh->cond_done, 0, sh, prm.counters, 11)) { alive = false; break; }
-          ptx::tc_fence_after();
+      ptx::mbar_arrive(&sh->acc_free[slot]);
+      ptx::fence_proxy_async();
+      ptx::named_bar_sync(1, kEpiThreads);
+      if (et == 0) {
+        int n0, h0;
+        job_origin(j, n0, h0);
 #pragma unroll
-          for (int cb = 0; cb < NT / 32; ++cb) {
-            const uint32_t word = words[cb];
-            if (__ballot_sync(0xffffffffu, word != 0) == 0) continue;   // warp-uniform: tcgen05.ld is .aligned
-            uint32_t r[32];
-            ptx::tmem_ld32(t_row + cb * 32, r);
-            uint8_t* st = s_y + (size_t)(cb >> 1) * P.stage_rows * 128 + (size_t)row * 128;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const int c16 = (cb & 1) * 4 + q;
-              uint4* slot = (uint4*)(st + ((c16 ^ (row & 7)) << 4));
-              uint4 cur = *slot;
-              uint32_t* cw = (uint32_t*)&cur;
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const int j = q * 8 + e * 2;
-                const int c = cb * 32 + j;
-                float v0 = __fadd_rn(__fmul_rn(s_a2[c], __uint_as_float(r[j])), s_b2[c]);
-                float v1 = __fadd_rn(__fmul_rn(s_a2[c + 1], __uint_as_float(r[j + 1])), s_b2[c + 1]);
-                if (L.relu) { v0 = v0 > 0.f ? v0 : 0.f; v1 = v1 > 0.f ? v1 : 0.f; }
-                const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
-                const uint32_t nv = *(const uint32_t*)&h2;
-                const uint32_t sel = (((word >> j) & 1u) ? 0x0000ffffu : 0u) |
-                                     (((word >> (j + 1)) & 1u) ? 0xffff0000u : 0u);
-                cw[e] = (cw[e] & ~sel) | (nv & sel);
-              }
-              *slot = cur;
-            }
-          }
-        }
+        for (int b = 0; b < kBlocks; ++b)
+          ptx::tma_store_4d(&map_y, s_y + (size_t)b * P.stage_rows * 128, tile_n * NT + b * 64, 0, h0, n0);
+        ptx::tma_store_commit();
       }
-    } while (0);
-    // staged tile -> global: one TMA store per 64-channel block
-    ptx::fence_proxy_async();
-    ptx::named_bar_sync(1, 128);
-    if (et == 0 && alive && !*(volatile uint32_t*)&sh->abort_flag) {
+    };
+
+    for (int j = 0; j < jobs && ok; ++j) {
+      gate_pass(j);
+      if (j >= 1 && ok) combine_pass(j - 1);
+    }
+    if (jobs > 0 && ok) combine_pass(jobs - 1);
+    if (et == 0) ptx::tma_store_wait_all();
+
+    // counters of this CTA
 #pragma unroll
-      for (int b = 0; b < kBlocks; ++b) {
-        if (tile_n * NT + b * 64 < L.c_out)
-          ptx::tma_store_4d(&map_y, s_y + (size_t)b * P.stage_rows * 128, tile_n * NT + b * 64, 0,
-                            h0, n0);
+    for (int o = 16; o > 0; o >>= 1) st_active += __shfl_xor_sync(0xffffffffu, st_active, o);
+    if (lane == 0 && ok) {
+      atomicAdd(&prm.counters[CNT_ACTIVE], st_active);
+      if (half == 0) {
+        atomicAdd(&prm.counters[CNT_ROWS_TOTAL], st_rows_valid);
+        atomicAdd(&prm.counters[CNT_ROWS_ACTIVE], st_rows_active);
       }
-      ptx::tma_store_commit();
-      // counters of this tile
-      const uint32_t blocks = dense ? kAllBlocks : sh->blk_active;
+    }
+    if (et == 0 && ok) {
       const unsigned long long k_p = (unsigned long long)taps * L.c_p, k_r = (unsigned long long)taps * L.c_r;
       if (blockIdx.x == 0) atomicAdd(&prm.counters[CNT_CALLS], 1ull);
-      atomicAdd(&prm.counters[CNT_ACTIVE], (unsigned long long)sh->n_active);
-      atomicAdd(&prm.counters[CNT_TILES_TOTAL], (unsigned long long)kBlocks);
-      atomicAdd(&prm.counters[CNT_TILES_SKIPPED], (unsigned long long)(kBlocks - __popc(blocks)));
-      atomicAdd(&prm.counters[CNT_ROWS_TOTAL], (unsigned long long)sh->n_rows_valid);
-      atomicAdd(&prm.counters[CNT_ROWS_ACTIVE], (unsigned long long)sh->n_rows_active);
+      atomicAdd(&prm.counters[CNT_TILES_TOTAL], (unsigned long long)kBlocks * jobs);
+      atomicAdd(&prm.counters[CNT_TILES_SKIPPED],
+                has_cond ? (unsigned long long)kBlocks * jobs - st_blocks_run : 0ull);
       atomicAdd(&prm.counters[CNT_EXEC_MACS],
-                (unsigned long long)kBM * NT * k_p + (unsigned long long)kBM * 64ull * __popc(blocks) * k_r);
-      ptx::tma_store_wait_all();
+                (unsigned long long)kBM * NT * k_p * jobs + (unsigned long long)kBM * 64ull * st_blocks_run * k_r);
     }
   }
   // ---------------------------------------------------------------- teardown
   ptx::tc_fence_before();
   __syncthreads();
-  if (warp == 1) ptx::tmem_dealloc(tmem, NT);
+  if (warp == 1) ptx::tmem_dealloc(tmem, 4 * NT);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -477,6 +679,17 @@ bool encode(CUtensorMap* map, void* base, int rank, const cuuint64_t* dims,
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+int sm_count() {
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+      sms = 148;
+  }
+  return sms;
+}
+
 }  // namespace
 
 bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
@@ -486,7 +699,7 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
   if (in_dtype != CG_BF16) return false;
   if (L.has_residual) return false;
   if (L.stride != 1 || L.kh != L.kw || L.kh != 2 * L.pad + 1) return false;
-  if (L.c_in % 64 != 0 || L.c_in / 64 > 8) return false;
+  if (L.c_in % 64 != 0) return false;
   if (!(L.c_p == 16 || L.c_p == 32 || L.c_p % 64 == 0)) return false;
   if (L.c_out % 64 != 0) return false;
   if (L.w + L.pad > kBM) return false;
@@ -534,25 +747,47 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
   P.stage_rows = (int)align_up((size_t)max(kBM, P.wp * P.out_box_h * P.ni), 8);
   P.cond_mode = cond_mode == CG_COND_AUTO ? CG_COND_SKIP_TILES : cond_mode;
   if (P.cond_mode == CG_COND_COMPACT) P.cond_mode = CG_COND_SKIP_TILES;
-  // widest column tile (<= 128) whose buffers fit in shared memory
+  if (P.base_tiles + P.cond_tiles > kMaxWTiles) return false;
+  // shared-memory layout: [weights: resident tiles or ring][patch ring][y staging][consts]
+  // [mask stash][tile coordinates][barriers]; widest column tile first, resident weights if
+  // they fit next to at least two patch buffers
   const size_t limit = 227 * 1024 - 1024;
   for (int nt = 128; nt >= 64; nt >>= 1) {
     if (L.c_out % nt != 0) continue;
-    for (int stages = 4; stages >= 2; --stages) {
-      size_t off = 0;
-      P.off_a = (unsigned)off; off += (size_t)P.chunks * P.patch_bytes;
-      P.off_b = (unsigned)off; off += (size_t)stages * nt * 128;
-      P.off_y = (unsigned)off; off += align_up((size_t)(nt / 64) * P.stage_rows * 128, 1024);
-      P.off_consts = (unsigned)off; off += align_up((size_t)5 * nt * 4, 128);
-      P.off_bar = (unsigned)off; off += align_up(sizeof(Shared), 128);
-      if (off <= limit) {
-        P.nt = nt; P.stages = stages; P.tiles_n = L.c_out / nt;
-        P.smem_bytes = (unsigned)(off + 1024);
-        P.valid = 1;
-        *plan = P;
-        return true;
+    const size_t fixed = align_up((size_t)(nt / 64) * P.stage_rows * 128, 1024) +
+                         align_up((size_t)5 * nt * 4, 128) +
+                         align_up((size_t)2 * 128 * (nt / 32) * 4, 128) +
+                         align_up((size_t)kMaxWTiles * 4, 128) + align_up(sizeof(Shared), 128);
+    const size_t w_tile = (size_t)nt * 128;
+    const size_t w_all = (size_t)(P.base_tiles + P.cond_tiles) * w_tile;
+    int na = 0, nb = 0, resident = 0;
+    if (fixed + w_all + 2 * (size_t)P.patch_bytes <= limit) {
+      resident = 1;
+      na = (int)((limit - fixed - w_all) / P.patch_bytes);
+      if (na > 4) na = 4;
+    } else {
+      bool found = false;
+      for (nb = 6; nb >= 3 && !found; --nb) {
+        if (fixed + nb * w_tile + 2 * (size_t)P.patch_bytes > limit) continue;
+        na = (int)((limit - fixed - nb * w_tile) / P.patch_bytes);
+        if (na > 4) na = 4;
+        if (na >= 3 || nb == 3) { found = true; break; }
       }
+      if (!found || na < 2) continue;
     }
+    size_t off = 0;
+    P.off_b = (unsigned)off; off += resident ? w_all : nb * w_tile;
+    P.off_a = (unsigned)off; off += (size_t)na * P.patch_bytes;
+    P.off_y = (unsigned)off; off += align_up((size_t)(nt / 64) * P.stage_rows * 128, 1024);
+    P.off_consts = (unsigned)off; off += align_up((size_t)5 * nt * 4, 128);
+    P.off_mask = (unsigned)off; off += align_up((size_t)2 * 128 * (nt / 32) * 4, 128);
+    P.off_tables = (unsigned)off; off += align_up((size_t)kMaxWTiles * 4, 128);
+    P.off_bar = (unsigned)off; off += align_up(sizeof(Shared), 128);
+    P.nt = nt; P.na = na; P.nb = nb; P.resident = resident; P.tiles_n = L.c_out / nt;
+    P.smem_bytes = (unsigned)(off + 1024);
+    P.valid = 1;
+    *plan = P;
+    return true;
   }
   return false;
 }
@@ -614,7 +849,11 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
   }
   TcParams prm;
   prm.L = L; prm.P = P; prm.bn = bn; prm.delta = delta; prm.mask = mask; prm.counters = counters;
-  const unsigned grid = (unsigned)(P.tiles_m * P.tiles_n);
+  // persistent grid: one CTA per SM, a multiple of the number of column tiles
+  const int sms = sm_count();
+  int grid = sms - sms % P.tiles_n;
+  if (grid < P.tiles_n) grid = P.tiles_n;
+  if (grid > P.tiles_m * P.tiles_n) grid = P.tiles_m * P.tiles_n;
   cudaError_t e;
   if (P.nt == 128) {
     static bool attr128 = false;

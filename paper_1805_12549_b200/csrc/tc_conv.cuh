@@ -19,18 +19,20 @@ struct TcPlan {
   int ip;               // image pitch in patch pixels: (h + pad) * wp
   int tiles_per_image;  // rows mode
   int tiles_m, tiles_n, nt;
-  int chunks;           // c_in / ck patch buffers, all resident
+  int chunks;           // c_in / ck input-channel chunks
   int base_chunks;      // chunks that hold base-path channels
+  int na;               // patch buffers in the ring
+  int nb;               // weight-tile ring depth (0 when the weights are resident)
+  int resident;         // 1: all weight tiles of a column tile stay in shared memory
   int box_h;            // patch box rows: r + 2*pad (rows mode) or h + pad (images mode)
   int box_pixels;       // wp * box_h * ni
   int patch_rows;       // rows allocated per patch buffer
   int patch_bytes;
   int out_box_h;        // y store box rows
   int stage_rows;       // rows of the y staging tile
-  int stages;           // depth of the weight-tile ring
   int base_tiles, cond_tiles;   // weight tiles per phase
   int cond_mode;
-  unsigned off_a, off_b, off_y, off_consts, off_bar, smem_bytes;
+  unsigned off_a, off_b, off_y, off_consts, off_mask, off_tables, off_bar, smem_bytes;
 };
 
 struct TcMapSet {

@@ -27,6 +27,9 @@ SHAPES = [
     (O.Shape(2, 14, 14, 256, 64, groups=8), "G = 8, c_p = 32, c_out != c_in"),
     (O.Shape(2, 13, 11, 64, 192, groups=2), "odd extents, G = 2, three column tiles of 64"),
     (O.Shape(2, 9, 9, 64, 64, kh=1, kw=1, pad=0, groups=4), "1x1 kernel"),
+    (O.Shape(12, 56, 56, 64, 64, groups=4), "336 row tiles: up to three jobs per CTA, resident weights"),
+    (O.Shape(50, 28, 28, 128, 128, groups=4), "350 row tiles: streamed weights, three jobs per CTA"),
+    (O.Shape(40, 14, 14, 256, 256, groups=4), "80 row tiles x 2 column tiles, two jobs per CTA"),
 ]
 
 
@@ -99,3 +102,24 @@ def test_two_calls_accumulate_and_are_deterministic():
     np.testing.assert_array_equal(m1, m2)
     assert st1.active == st2.active and st1.calls == st2.calls == 1
     g.close()
+
+
+@pytest.mark.parametrize("layer", ["c64@56", "c128@28", "c256@14", "c512@7"])
+def test_full_size_layers_on_sampled_images(layer):
+    """Batch-64 ImageNet ResNet-18 layer shapes in the configuration the benchmark times;
+    images are independent, so the oracle checks a sample of them one by one."""
+    from paper_1805_12549_b200 import synth
+    ls = {l.name: l for l in synth.imagenet_resnet18_layers(64, 4)}[layer]
+    s = O.Shape(ls.n, ls.hw, ls.hw, ls.c_in, ls.c_out, groups=4)
+    c = K.make_float_case("full", s, "bf16", density=0.3, calib_images=2)
+    g = K.GpuCase(c, algo=TENSOR)
+    y, mask, st = g.run()
+    g.close()
+    assert abs(st.density - 0.3) < 0.04
+    words = s.words
+    per_img = s.ho * s.wo
+    for n in (0, 17, 40, 63):
+        s1 = O.Shape(**{**s.__dict__, "n": 1})
+        c1 = K.Case(c.name, s1, c.dtype, c.x[n:n + 1], c.wb, c.wc, c.bn, c.delta)
+        ref = K.run_oracle(c1)
+        K.compare(c1, ref, y[n:n + 1], mask[n * per_img:(n + 1) * per_img].reshape(-1, words), None)
