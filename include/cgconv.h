@@ -175,6 +175,34 @@ int cg_conv_uses_tensor_cores(cg_conv_t h);
 
 void cg_conv_destroy(cg_conv_t h);
 
+/* (No counterpart in the paper: a packaging variant of the same layer.)
+ * The gated layer for callers that cannot allocate device memory: code that runs inside a
+ * framework or memory pool that owns the whole device, loops that must not make calls which
+ * can synchronise the device, plug-ins that are handed tensors but no allocator.  The regular
+ * API needs a handle, and cg_conv_create allocates; this call needs no handle and allocates
+ * nothing, on the device or through any library.  Its scratch -- the activity counters and the
+ * per-channel gate/batch-norm constants that a small prologue kernel folds on every call -- is
+ * a fixed array inside the library image, which costs every GPU that loads the library about
+ * 40 KB until the process exits.
+ *   desc      the layer, as for cg_conv_create (algo and cond_mode are ignored: the CUDA-core
+ *             direct kernels run it, so results equal cg_conv_forward with CG_ALGO_DIRECT);
+ *             F32 and BF16 only, else CG_ERR_UNSUPPORTED
+ *   x .. mask_out   device pointers exactly as for cg_conv_forward
+ *   stats_out NULL, or a host struct to fill (outputs, active, dense/gated/executed MACs); a
+ *             non-NULL value makes the call synchronise the stream
+ * Limit: desc->c_out <= CG_STATIC_MAX_C_OUT, else CG_ERR_WORKSPACE (the constants would not
+ * fit the fixed array).  Other errors as cg_conv_forward.
+ * The first call on each device looks up the array's device address (with that device
+ * current); make that first call outside any stream capture.
+ * Every call on a device uses the same array and overwrites what the previous call left
+ * there (the counters are cleared by the prologue), so two calls that can overlap on the GPU
+ * -- different streams, or the same stream from two threads -- race; serialise them. */
+#define CG_STATIC_MAX_C_OUT 2048
+cg_status cg_conv_forward_static(const cg_conv_desc* desc, const void* x, const void* w_base,
+                                 const void* w_cond, const cg_bn_params* bn, const float* delta,
+                                 const void* residual, void* y, uint32_t* mask_out,
+                                 cg_stats* stats_out, void* cuda_stream);
+
 const char* cg_status_string(cg_status s);
 
 #ifdef __cplusplus

@@ -22,7 +22,7 @@ CG_COND_AUTO, CG_COND_DENSE, CG_COND_SKIP_TILES, CG_COND_COMPACT = 0, 1, 2, 3
 EXPORTS = ("cg_conv_create", "cg_conv_workspace_bytes", "cg_conv_forward",
            "cg_conv_host_staging_bytes", "cg_conv_forward_host", "cg_conv_partial_sums",
            "cg_conv_stats", "cg_conv_launches_per_forward", "cg_conv_uses_tensor_cores",
-           "cg_conv_destroy", "cg_status_string")
+           "cg_conv_destroy", "cg_status_string", "cg_conv_forward_static")
 
 
 class CgConvDesc(C.Structure):
@@ -81,6 +81,11 @@ def lib():
         L.cg_conv_uses_tensor_cores.argtypes = [C.c_void_p]
         L.cg_conv_destroy.restype = None
         L.cg_conv_destroy.argtypes = [C.c_void_p]
+        L.cg_conv_forward_static.restype = C.c_int
+        L.cg_conv_forward_static.argtypes = [C.POINTER(CgConvDesc), C.c_void_p, C.c_void_p,
+                                             C.c_void_p, C.POINTER(CgBnParams), C.c_void_p,
+                                             C.c_void_p, C.c_void_p, C.c_void_p,
+                                             C.POINTER(CgStats), C.c_void_p]
         L.cg_status_string.restype = C.c_char_p
         L.cg_status_string.argtypes = [C.c_int]
         _lib = L
@@ -186,6 +191,21 @@ def cg_conv_stats(h, stream=None, check=True) -> Stats:
     if check:
         _check(rc, f"cg_conv_stats (device site {out.device_site})")
     return out
+
+
+CG_STATIC_MAX_C_OUT = 2048
+
+
+def cg_conv_forward_static(desc: CgConvDesc, x, w_base, w_cond, bn: CgBnParams, delta, residual, y,
+                           mask_out, want_stats=False, stream=None):
+    """The layer without a handle and without any allocation (see include/cgconv.h): scratch
+    lives in a fixed array inside the library.  Calls on one device must not overlap."""
+    st = CgStats() if want_stats else None
+    _check(lib().cg_conv_forward_static(C.byref(desc), _ptr(x), _ptr(w_base), _ptr(w_cond),
+                                        C.byref(bn), _ptr(delta), _ptr(residual), _ptr(y),
+                                        _ptr(mask_out), C.byref(st) if st is not None else None,
+                                        _stream_ptr(stream)), "cg_conv_forward_static")
+    return None if st is None else Stats(*[getattr(st, k) for k, _ in CgStats._fields_])
 
 
 def cg_conv_launches_per_forward(h) -> int:
