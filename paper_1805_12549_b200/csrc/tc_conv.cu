@@ -22,7 +22,8 @@
 //   MMA issue order      base(0) | base(1) cond(0) | base(2) cond(1) | ...
 //   epilogue order       gate(0) | gate(1) combine(0) | gate(2) combine(1) | ...
 // so the tensor pipe works on the next tile's base path while the gate of the current tile is
-// being evaluated.  TMEM holds two job slots of (P, R) accumulators: 4*NT columns.
+// being evaluated.  TMEM (512 columns) holds a ring of P accumulators and a ring of R
+// accumulators: 4 + 4 at NT = 64, 3 + 1 at NT = 128, so the issuer can run ahead of the epilogue.
 // Weights stay resident in shared memory when they fit, otherwise they stream through a ring.
 //
 // Warp roles: 0 = patch (A) producer, 1 = MMA issuer (owns TMEM), 2 = weight (B) producer,
@@ -88,10 +89,11 @@ struct Shared {
   uint64_t a_full[8], a_empty[8];
   uint64_t b_full[8], b_empty[8];
   uint64_t w_ready;
-  uint64_t base_done[2], gate_done[2], cond_done[2], acc_free[2];
+  uint64_t base_done[4], gate_done[4], p_free[4];   // per P accumulator slot
+  uint64_t cond_done[4], r_free[4];                 // per R accumulator slot
   uint32_t tmem_base;
   uint32_t abort_flag;
-  uint32_t warp_blk[2][8];   // per job slot, per epilogue warp: column blocks with a firing gate
+  uint32_t warp_blk[4][8];   // per job slot, per epilogue warp: column blocks with a firing gate
 };
 
 struct Ctx {
@@ -308,7 +310,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   float* s_b1 = s_a1 + NT;
   float* s_a2 = s_b1 + NT;
   float* s_b2 = s_a2 + NT;
-  uint32_t* s_mask = (uint32_t*)(smem + P.off_mask);       // [2][128][NT/32]
+  uint32_t* s_mask = (uint32_t*)(smem + P.off_mask);       // [4][128][NT/32]
   int* s_wx = (int*)(smem + P.off_tables);                 // [base_tiles + cond_tiles] K coordinates
   Shared* sh = (Shared*)(smem + P.off_bar);
   const Ctx cx{sh, prm.counters};
@@ -326,6 +328,8 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   constexpr int kBlocks = NT / 64;
   constexpr uint32_t kAllBlocks = (1u << kBlocks) - 1u;
   constexpr int kWords = NT / 32;
+  constexpr int kNP = NT == 64 ? 4 : 3;      // P accumulators in TMEM
+  constexpr int kNR = NT == 64 ? 4 : 1;      // R accumulators in TMEM
   const uint32_t w_tile_bytes = NT * 128;
   const uint32_t patch_tx = (uint32_t)P.box_pixels * 128u;
 
@@ -340,18 +344,19 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     for (int i = 0; i < P.na; ++i) { ptx::mbar_init(&sh->a_full[i], 1); ptx::mbar_init(&sh->a_empty[i], 1); }
     for (int i = 0; i < P.nb; ++i) { ptx::mbar_init(&sh->b_full[i], 1); ptx::mbar_init(&sh->b_empty[i], 1); }
     ptx::mbar_init(&sh->w_ready, 1);
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < 4; ++i) {
       ptx::mbar_init(&sh->base_done[i], 1);
       ptx::mbar_init(&sh->gate_done[i], kEpiThreads);
+      ptx::mbar_init(&sh->p_free[i], kEpiThreads);
       ptx::mbar_init(&sh->cond_done[i], 1);
-      ptx::mbar_init(&sh->acc_free[i], kEpiThreads);
+      ptx::mbar_init(&sh->r_free[i], kEpiThreads);
     }
     sh->abort_flag = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&map_x); ptx::prefetch_tensormap(&map_wb);
     ptx::prefetch_tensormap(&map_wc); ptx::prefetch_tensormap(&map_y);
   }
-  if (warp == 1) ptx::tmem_alloc(&sh->tmem_base, 4 * NT);
+  if (warp == 1) ptx::tmem_alloc(&sh->tmem_base, 512);
   if (warp >= 3) {
     const int et = threadIdx.x - kEpiThread0;
     // zero the rows behind the TMA box of every patch buffer: they stand for the right padding
@@ -400,9 +405,9 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
           const int jj = j - 1;
           uint32_t blocks = kAllBlocks;
           if (!dense) {
-            ok = wait_bar(cx, &sh->gate_done[jj & 1], (jj >> 1) & 1, 2);
+            ok = wait_bar(cx, &sh->gate_done[jj % kNP], (jj / kNP) & 1, 2);
             if (!ok) break;
-            blocks = slot_blocks(sh, jj & 1);
+            blocks = slot_blocks(sh, jj % kNP);
           }
           if (blocks) load_chunks(jj, cond_first_chunk, P.chunks);
         }
@@ -438,9 +443,9 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
             const int jj = j - 1;
             uint32_t blocks = kAllBlocks;
             if (!dense) {
-              ok = wait_bar(cx, &sh->gate_done[jj & 1], (jj >> 1) & 1, 4);
+              ok = wait_bar(cx, &sh->gate_done[jj % kNP], (jj / kNP) & 1, 4);
               if (!ok) break;
-              blocks = slot_blocks(sh, jj & 1);
+              blocks = slot_blocks(sh, jj % kNP);
             }
             if (blocks) load_tiles(&map_wc, P.base_tiles, P.cond_tiles);
           }
@@ -457,26 +462,33 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       if (P.resident) ok = wait_bar(cx, &sh->w_ready, 0, 6);
       for (int j = 0; j <= jobs && ok; ++j) {
         if (j < jobs) {
-          ok = wait_bar(cx, &sh->acc_free[j & 1], ((j >> 1) & 1) ^ 1, 9);
+          const int ps = j % kNP;
+          ok = wait_bar(cx, &sh->p_free[ps], ((j / kNP) & 1) ^ 1, 9);
           if (!ok) break;
           ptx::tc_fence_after();
-          ok = mi.run_phase(tmem + (uint32_t)((j & 1) * 2 * NT), false, kAllBlocks);
+          ok = mi.run_phase(tmem + (uint32_t)(ps * NT), false, kAllBlocks);
           if (!ok) break;
-          ptx::umma_commit_if(mi.issue, &sh->base_done[j & 1]);
+          ptx::umma_commit_if(mi.issue, &sh->base_done[ps]);
         }
         if (j >= 1) {
           const int jj = j - 1;
+          const int rs = jj % kNR;
           if (has_cond) {
             uint32_t blocks = kAllBlocks;
             if (!dense) {
-              ok = wait_bar(cx, &sh->gate_done[jj & 1], (jj >> 1) & 1, 10);
+              ok = wait_bar(cx, &sh->gate_done[jj % kNP], (jj / kNP) & 1, 10);
               if (!ok) break;
-              blocks = slot_blocks(sh, jj & 1);
+              blocks = slot_blocks(sh, jj % kNP);
             }
-            if (blocks) ok = mi.run_phase(tmem + (uint32_t)((jj & 1) * 2 * NT + NT), true, blocks);
-            if (!ok) break;
+            if (blocks) {
+              ok = wait_bar(cx, &sh->r_free[rs], ((jj / kNR) & 1) ^ 1, 14);
+              if (!ok) break;
+              ptx::tc_fence_after();
+              ok = mi.run_phase(tmem + (uint32_t)((kNP + rs) * NT), true, blocks);
+              if (!ok) break;
+            }
           }
-          ptx::umma_commit_if(mi.issue, &sh->cond_done[jj & 1]);
+          ptx::umma_commit_if(mi.issue, &sh->cond_done[rs]);
         }
       }
     }
@@ -499,8 +511,8 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
 
     // gate of job j: P -> mask words (global + stash), block activity flags
     auto gate_pass = [&](int j) {
-      const int slot = j & 1;
-      ok = wait_bar(cx, &sh->base_done[slot], (j >> 1) & 1, 11);
+      const int slot = j % kNP;
+      ok = wait_bar(cx, &sh->base_done[slot], (j / kNP) & 1, 11);
       if (!ok) return;
       ptx::tc_fence_after();
       int n0, h0;
@@ -513,7 +525,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       for (int cc = 0; cc < kWords / 2; ++cc) {
         const int cb = cc * 2 + half;
         uint32_t r[32];
-        ptx::tmem_ld32(t_lane + (uint32_t)(slot * 2 * NT + cb * 32), r);
+        ptx::tmem_ld32(t_lane + (uint32_t)(slot * NT + cb * 32), r);
         uint32_t word = 0;
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
@@ -542,8 +554,8 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
 
     // combine of job j: y = f(BN1(P)) or f(BN2(P+R)) by mask bit, staged and stored
     auto combine_pass = [&](int j) {
-      const int slot = j & 1;
-      ok = wait_bar(cx, &sh->gate_done[slot], (j >> 1) & 1, 12);   // every warp's flags and words
+      const int slot = j % kNP, rslot = j % kNR;
+      ok = wait_bar(cx, &sh->gate_done[slot], (j / kNP) & 1, 12);   // every warp's flags and words
       if (!ok) return;
       const uint32_t blocks = !has_cond ? 0u : (dense ? kAllBlocks : slot_blocks(sh, slot));
       if (half == 0) {
@@ -553,7 +565,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         const uint32_t row_active = __ballot_sync(0xffffffffu, any != 0);
         if (lane == 0) st_rows_active += __popc(row_active);
       }
-      ok = wait_bar(cx, &sh->cond_done[slot], (j >> 1) & 1, 13);
+      ok = wait_bar(cx, &sh->cond_done[rslot], (j / kNR) & 1, 13);
       if (!ok) return;
       ptx::tc_fence_after();
       if (et == 0) {
@@ -566,10 +578,10 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         const int cb = cc * 2 + half;
         const uint32_t word = s_mask[(slot * 128 + row) * kWords + cb];
         uint32_t p[32], rr[32];
-        ptx::tmem_ld32(t_lane + (uint32_t)(slot * 2 * NT + cb * 32), p);
+        ptx::tmem_ld32(t_lane + (uint32_t)(slot * NT + cb * 32), p);
         const bool have_r = ((blocks >> (cb >> 1)) & 1u) && __ballot_sync(0xffffffffu, word != 0) != 0;
         if (have_r) {
-          ptx::tmem_ld32(t_lane + (uint32_t)(slot * 2 * NT + NT + cb * 32), rr);
+          ptx::tmem_ld32(t_lane + (uint32_t)((kNP + rslot) * NT + cb * 32), rr);
         } else {
 #pragma unroll
           for (int i = 0; i < 32; ++i) rr[i] = 0u;
@@ -601,7 +613,8 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         }
       }
       ptx::tc_fence_before();
-      ptx::mbar_arrive(&sh->acc_free[slot]);
+      ptx::mbar_arrive(&sh->p_free[slot]);
+      ptx::mbar_arrive(&sh->r_free[rslot]);
       ptx::fence_proxy_async();
       ptx::named_bar_sync(1, kEpiThreads);
       if (et == 0) {
@@ -644,7 +657,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   // ---------------------------------------------------------------- teardown
   ptx::tc_fence_before();
   __syncthreads();
-  if (warp == 1) ptx::tmem_dealloc(tmem, 4 * NT);
+  if (warp == 1) ptx::tmem_dealloc(tmem, 512);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -756,7 +769,7 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
     if (L.c_out % nt != 0) continue;
     const size_t fixed = align_up((size_t)(nt / 64) * P.stage_rows * 128, 1024) +
                          align_up((size_t)5 * nt * 4, 128) +
-                         align_up((size_t)2 * 128 * (nt / 32) * 4, 128) +
+                         align_up((size_t)4 * 128 * (nt / 32) * 4, 128) +
                          align_up((size_t)kMaxWTiles * 4, 128) + align_up(sizeof(Shared), 128);
     const size_t w_tile = (size_t)nt * 128;
     const size_t w_all = (size_t)(P.base_tiles + P.cond_tiles) * w_tile;
@@ -780,7 +793,7 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
     P.off_a = (unsigned)off; off += (size_t)na * P.patch_bytes;
     P.off_y = (unsigned)off; off += align_up((size_t)(nt / 64) * P.stage_rows * 128, 1024);
     P.off_consts = (unsigned)off; off += align_up((size_t)5 * nt * 4, 128);
-    P.off_mask = (unsigned)off; off += align_up((size_t)2 * 128 * (nt / 32) * 4, 128);
+    P.off_mask = (unsigned)off; off += align_up((size_t)4 * 128 * (nt / 32) * 4, 128);
     P.off_tables = (unsigned)off; off += align_up((size_t)kMaxWTiles * 4, 128);
     P.off_bar = (unsigned)off; off += align_up(sizeof(Shared), 128);
     P.nt = nt; P.na = na; P.nb = nb; P.resident = resident; P.tiles_n = L.c_out / nt;
