@@ -96,6 +96,24 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+# ------------------------------------------------------------------------------- ranks
+def max_over_ranks(ms_local, device="cuda"):
+    """Device time of the slowest rank (every rank shards the batch and runs alone: no
+    collective on the data path, only this reduction of the timing)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms_local)
+    t = torch.tensor([float(ms_local)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(images_per_rank, world, ms_per_step):
+    """Aggregate images/s of `world` ranks that each process `images_per_rank` per step."""
+    return world * images_per_rank / (ms_per_step * 1e-3)
+
+
 # ------------------------------------------------------------------------------- our arm
 class LayerBench:
     """Device buffers, calibrated gate parameters and the handle of one layer shape."""
@@ -233,16 +251,12 @@ def run_ours(args):
     e1.record(stream)
     torch.cuda.synchronize()
     t1 = time.time()
-    ms_total = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(e0.elapsed_time(e1))
     for lb in layers:
         lb.stats = lb.conv.stats()
     ms_step = ms_total / args.steps
     batch = shapes[0].n
-    value = world * batch / (ms_step * 1e-3)
+    value = whole_job_rate(batch, world, ms_step)
 
     # per-layer kernel durations: the same launches, one layer at a time, back to back
     reps = max(1, args.steps // LayerBench.SETS)
@@ -305,14 +319,10 @@ def run_ours(args):
             lb.forward_host()
     e1.record(stream)
     torch.cuda.synchronize()
-    ms_e2e = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms_e2e], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1))
     for lb in layers:
         lb.conv.stats()
-    e2e = {"value": round(world * batch / (ms_e2e / e2e_steps * 1e-3), 1), "unit": UNIT,
+    e2e = {"value": round(whole_job_rate(batch, world, ms_e2e / e2e_steps), 1), "unit": UNIT,
            "h2d_bytes_per_step": sum(lb.bytes_x for lb in layers),
            "d2h_bytes_per_step": sum(lb.bytes_y + lb.bytes_mask for lb in layers)}
 

@@ -44,6 +44,7 @@ constexpr int kEpiThreads = 256;
 constexpr int kBM = 128;            // MMA M: patch rows per job
 constexpr int kSpinLimit = 1 << 21; // try_wait polls (each up to ~2 us) before a wait gives up
 constexpr int kMaxWTiles = 192;     // weight tiles per job, both phases
+constexpr bool kUnroll3x3 = true;   // fully unrolled 3x3 issue code (measured faster than rolled tap loops)
 
 struct TcParams {
   LayerDims L;
@@ -202,7 +203,7 @@ struct MmaIssuer {
   template <bool RES, bool ALL, int KS0, int KS1>
   __device__ __forceinline__ void chunk_taps() {
     acquire_a();
-    if (kh == 3 && kw == 3) {
+    if (kUnroll3x3 && kh == 3 && kw == 3) {
 #pragma unroll
       for (int r = 0; r < 3; ++r) {
 #pragma unroll
@@ -235,7 +236,7 @@ struct MmaIssuer {
   __device__ __forceinline__ void base_small() {
     constexpr int TPT = 4 / KP;
     acquire_a();
-    if (kh == 3 && kw == 3) {
+    if (kUnroll3x3 && kh == 3 && kw == 3) {
 #pragma unroll
       for (int t = 0; t < 9; ++t) {
         if (t % TPT == 0) acquire_b<RES>();
