@@ -142,12 +142,12 @@ struct MmaIssuer {
   uint32_t desc_hi;                      // upper descriptor word (see ptx::smem_desc)
   uint32_t a_base_lo, b_base_lo;         // lower descriptor words of the ring bases
   uint32_t patch_lo, wtile_lo, row_lo;   // buffer sizes / one patch pixel row, in 16-byte units
-  int resident, na, nb, kp16, chunks, base_chunks, base_tiles, kh, kw;
+  int resident, na, nb, kp16, chunks, base_chunks, base_tiles, kh, kw, planes;
   int as, bs;                            // ring slots and the parities of their "full" barriers
   uint32_t apar, bpar;
   // per phase
-  uint32_t d_tmem, a_lo, b_lo, acc, blk_off_d, blk_off_b;
-  int a_held, b_held;
+  uint32_t d_tmem, a_lo[4], b_lo, acc, blk_off_d, blk_off_b;   // a_lo: one per plane
+  int a_held[4], b_held;
   bool ok;
 
   __device__ __forceinline__ void init(Shared* sh_, const Ctx& cx_, const uint8_t* s_a,
@@ -164,9 +164,10 @@ struct MmaIssuer {
     wtile_lo = (uint32_t)(NT * 128) >> 4;
     row_lo = (uint32_t)P.wp * 8u;
     resident = P.resident; na = P.na; nb = P.nb; kp16 = L.c_p / 16; chunks = P.chunks;
-    base_chunks = P.base_chunks; base_tiles = P.base_tiles; kh = L.kh; kw = L.kw;
+    base_chunks = P.base_chunks; base_tiles = P.base_tiles; kh = L.kh; kw = L.kw; planes = P.planes;
     as = 0; bs = 0; apar = 0; bpar = 0;
-    a_held = 0; b_held = 0; ok = true;
+    b_held = 0; ok = true;
+    for (int i = 0; i < 4; ++i) { a_held[i] = 0; a_lo[i] = 0; }
   }
   template <bool ALL>
   __device__ __forceinline__ void mma(uint32_t al, uint32_t bl) {
@@ -178,13 +179,34 @@ struct MmaIssuer {
                         ptx::idesc_bf16(kBM, 64), acc);
     acc = 1u;
   }
+  // the patch buffer(s) of the next chunk in the ring: one, or the four planes of a stride-2 layer
+  template <bool S2>
   __device__ __forceinline__ void acquire_a() {
-    ok = ok && wait_bar(cx, &sh->a_full[as], apar, 7);
-    a_held = as;
-    a_lo = a_base_lo + (uint32_t)as * patch_lo;
-    if (++as == na) { as = 0; apar ^= 1; }
+#pragma unroll
+    for (int pl = 0; pl < (S2 ? 4 : 1); ++pl) {
+      ok = ok && wait_bar(cx, &sh->a_full[as], apar, 7);
+      a_held[pl] = as;
+      a_lo[pl] = a_base_lo + (uint32_t)as * patch_lo;
+      if (++as == na) { as = 0; apar ^= 1; }
+    }
   }
-  __device__ __forceinline__ void release_a() { ptx::umma_commit_if(issue, &sh->a_empty[a_held]); }
+  template <bool S2>
+  __device__ __forceinline__ void release_a() {
+#pragma unroll
+    for (int pl = 0; pl < (S2 ? 4 : 1); ++pl) ptx::umma_commit_if(issue, &sh->a_empty[a_held[pl]]);
+  }
+  // descriptor word of the A operand of tap (r, sx).  Stride 1: the patch read from pixel
+  // r*(W+pad)+sx on.  Stride 2 (3x3, pad 1): output (h,w) reads input (2h+r-1, 2w+sx-1), i.e.
+  // plane (r odd ? 0 : 1, sx odd ? 0 : 1) at (h + (r ? 0 : -1), w + (sx ? 0 : -1)); every plane
+  // patch starts one row and one column early, so the offset is (r ? 1 : 0) rows + (sx ? 1 : 0).
+  template <bool S2>
+  __device__ __forceinline__ uint32_t tap_lo(int r, int sx) const {
+    if (S2) {
+      const uint32_t base = (r == 1) ? ((sx == 1) ? a_lo[0] : a_lo[1]) : ((sx == 1) ? a_lo[2] : a_lo[3]);
+      return base + (r ? row_lo : 0u) + (sx ? 8u : 0u);
+    }
+    return a_lo[0] + (uint32_t)r * row_lo + (uint32_t)sx * 8u;
+  }
   template <bool RES>
   __device__ __forceinline__ void acquire_b() {
     if (!RES) {
@@ -200,9 +222,9 @@ struct MmaIssuer {
     else ptx::umma_commit_if(issue, &sh->b_empty[b_held]);
   }
   // K steps [KS0, KS1) of every tap of the next chunk in the ring, one weight tile per tap
-  template <bool RES, bool ALL, int KS0, int KS1>
+  template <bool RES, bool ALL, bool S2, int KS0, int KS1>
   __device__ __forceinline__ void chunk_taps() {
-    acquire_a();
+    acquire_a<S2>();
     if (kUnroll3x3 && kh == 3 && kw == 3) {
 #pragma unroll
       for (int r = 0; r < 3; ++r) {
@@ -210,50 +232,48 @@ struct MmaIssuer {
         for (int sx = 0; sx < 3; ++sx) {
           acquire_b<RES>();
           if (!ok) return;
-          const uint32_t a_t = a_lo + (uint32_t)r * row_lo + (uint32_t)sx * 8u;
+          const uint32_t a_t = tap_lo<S2>(r, sx);
 #pragma unroll
           for (int ks = KS0; ks < KS1; ++ks) mma<ALL>(a_t + ks * 2, b_lo + (ks - KS0) * 2);
           release_b<RES>();
         }
       }
     } else {
-      uint32_t a_r = a_lo;
-      for (int r = 0; r < kh; ++r, a_r += row_lo) {
+      for (int r = 0; r < kh; ++r) {
         for (int sx = 0; sx < kw; ++sx) {
           acquire_b<RES>();
           if (!ok) return;
-          const uint32_t a_t = a_r + (uint32_t)sx * 8u;
+          const uint32_t a_t = tap_lo<S2>(r, sx);
 #pragma unroll
           for (int ks = KS0; ks < KS1; ++ks) mma<ALL>(a_t + ks * 2, b_lo + (ks - KS0) * 2);
           release_b<RES>();
         }
       }
     }
-    release_a();
+    release_a<S2>();
   }
   // base path when c_p < 64: the first KP K steps of chunk 0; a weight tile covers 4/KP taps
-  template <bool RES, bool ALL, int KP>
+  template <bool RES, bool ALL, bool S2, int KP>
   __device__ __forceinline__ void base_small() {
     constexpr int TPT = 4 / KP;
-    acquire_a();
+    acquire_a<S2>();
     if (kUnroll3x3 && kh == 3 && kw == 3) {
 #pragma unroll
       for (int t = 0; t < 9; ++t) {
         if (t % TPT == 0) acquire_b<RES>();
         if (!ok) return;
-        const uint32_t a_t = a_lo + (uint32_t)(t / 3) * row_lo + (uint32_t)(t % 3) * 8u;
+        const uint32_t a_t = tap_lo<S2>(t / 3, t % 3);
 #pragma unroll
         for (int ks = 0; ks < KP; ++ks) mma<ALL>(a_t + ks * 2, b_lo + ((t % TPT) * KP + ks) * 2);
         if (t % TPT == TPT - 1 || t == 8) release_b<RES>();
       }
     } else {
       int in_tile = 0;
-      uint32_t a_r = a_lo;
-      for (int r = 0; r < kh; ++r, a_r += row_lo) {
+      for (int r = 0; r < kh; ++r) {
         for (int sx = 0; sx < kw; ++sx) {
           if (in_tile == 0) acquire_b<RES>();
           if (!ok) return;
-          const uint32_t a_t = a_r + (uint32_t)sx * 8u;
+          const uint32_t a_t = tap_lo<S2>(r, sx);
 #pragma unroll
           for (int ks = 0; ks < KP; ++ks) mma<ALL>(a_t + ks * 2, b_lo + (uint32_t)(in_tile * KP + ks) * 2u);
           if (++in_tile == TPT) { release_b<RES>(); in_tile = 0; }
@@ -261,20 +281,24 @@ struct MmaIssuer {
       }
       if (in_tile != 0) release_b<RES>();
     }
-    release_a();
+    release_a<S2>();
   }
-  template <bool RES, bool ALL>
+  template <bool RES, bool ALL, bool S2>
   __device__ __forceinline__ void phase(bool cond) {
     if (kp16 >= 4) {
       const int q0 = cond ? base_chunks : 0, q1 = cond ? chunks : base_chunks;
-      for (int q = q0; q < q1 && ok; ++q) chunk_taps<RES, ALL, 0, 4>();
+      for (int q = q0; q < q1 && ok; ++q) chunk_taps<RES, ALL, S2, 0, 4>();
     } else if (!cond) {
-      if (kp16 == 1) base_small<RES, ALL, 1>(); else base_small<RES, ALL, 2>();
+      if (kp16 == 1) base_small<RES, ALL, S2, 1>(); else base_small<RES, ALL, S2, 2>();
     } else {
       // conditional channels of chunk 0 (K steps kp16..3), then the remaining chunks
-      if (kp16 == 1) chunk_taps<RES, ALL, 1, 4>(); else chunk_taps<RES, ALL, 2, 4>();
-      for (int q = 1; q < chunks && ok; ++q) chunk_taps<RES, ALL, 0, 4>();
+      if (kp16 == 1) chunk_taps<RES, ALL, S2, 1, 4>(); else chunk_taps<RES, ALL, S2, 2, 4>();
+      for (int q = 1; q < chunks && ok; ++q) chunk_taps<RES, ALL, S2, 0, 4>();
     }
+  }
+  template <bool RES, bool ALL>
+  __device__ __forceinline__ void phase_s(bool cond) {
+    if (planes == 4) phase<RES, ALL, true>(cond); else phase<RES, ALL, false>(cond);
   }
   // base or conditional MMAs of one job into the accumulator at d; `blocks` = column blocks to
   // compute (all of them for the base path)
@@ -286,8 +310,8 @@ struct MmaIssuer {
     b_lo = b_base_lo + (cond ? (uint32_t)base_tiles * wtile_lo : 0u);   // resident tiles
     blk_off_d = blocks == 2u ? 64u : 0u;
     blk_off_b = blocks == 2u ? (64u * 128u / 16u) : 0u;
-    if (blocks == kAll) { if (resident) phase<true, true>(cond); else phase<false, true>(cond); }
-    else { if (resident) phase<true, false>(cond); else phase<false, false>(cond); }
+    if (blocks == kAll) { if (resident) phase_s<true, true>(cond); else phase_s<false, true>(cond); }
+    else { if (resident) phase_s<true, false>(cond); else phase_s<false, false>(cond); }
     return ok;
   }
 };
@@ -295,6 +319,9 @@ struct MmaIssuer {
 template <int NT>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
+                     const __grid_constant__ CUtensorMap map_x1,
+                     const __grid_constant__ CUtensorMap map_x2,
+                     const __grid_constant__ CUtensorMap map_x3,
                      const __grid_constant__ CUtensorMap map_wb,
                      const __grid_constant__ CUtensorMap map_wc,
                      const __grid_constant__ CUtensorMap map_y,
@@ -355,6 +382,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     sh->abort_flag = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&map_x); ptx::prefetch_tensormap(&map_wb);
+    if (P.planes == 4) { ptx::prefetch_tensormap(&map_x1); ptx::prefetch_tensormap(&map_x2); ptx::prefetch_tensormap(&map_x3); }
     ptx::prefetch_tensormap(&map_wc); ptx::prefetch_tensormap(&map_y);
   }
   if (warp == 1) ptx::tmem_alloc(&sh->tmem_base, 512);
@@ -391,13 +419,17 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       auto load_chunks = [&](int j, int q0, int q1) {
         int n0, h0;
         job_origin(j, n0, h0);
+        const int lead = P.planes == 4 ? 1 : L.pad;   // zero rows/columns in front of the patch
         for (int q = q0; q < q1 && ok; ++q) {
-          ok = wait_bar(cx, &sh->a_empty[as], apar, 1);
-          if (!ok) return;
-          ptx::mbar_expect_tx(&sh->a_full[as], patch_tx);
-          ptx::tma_load_4d(s_a + (size_t)as * P.patch_bytes, &map_x, &sh->a_full[as], q * 64, -L.pad,
-                           h0 - L.pad, n0);
-          if (++as == P.na) { as = 0; apar ^= 1; }
+          for (int pl = 0; pl < P.planes && ok; ++pl) {
+            ok = wait_bar(cx, &sh->a_empty[as], apar, 1);
+            if (!ok) return;
+            const CUtensorMap* mx = pl == 0 ? &map_x : (pl == 1 ? &map_x1 : (pl == 2 ? &map_x2 : &map_x3));
+            ptx::mbar_expect_tx(&sh->a_full[as], patch_tx);
+            ptx::tma_load_4d(s_a + (size_t)as * P.patch_bytes, mx, &sh->a_full[as], q * 64, -lead,
+                             h0 - lead, n0);
+            if (++as == P.na) { as = 0; apar ^= 1; }
+          }
         }
       };
       for (int j = 0; j <= jobs && ok; ++j) {
@@ -518,8 +550,8 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       ptx::tc_fence_after();
       int n0, h0;
       job_origin(j, n0, h0);
-      const int rows_here = P.images_mode ? L.h : min(P.r, L.h - h0);
-      const bool valid = (w_out < L.w) && (h_loc < rows_here) && (n_loc < P.ni) && (n0 + n_loc < L.n);
+      const int rows_here = P.images_mode ? L.ho : min(P.r, L.ho - h0);
+      const bool valid = (w_out < L.wo) && (h_loc < rows_here) && (n_loc < P.ni) && (n0 + n_loc < L.n);
       const long long m = ((long long)(n0 + n_loc) * L.ho + (h0 + h_loc)) * L.wo + w_out;
       uint32_t my_blocks = 0;
 #pragma unroll
@@ -712,39 +744,45 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
   *plan = P;
   if (in_dtype != CG_BF16) return false;
   if (L.has_residual) return false;
-  if (L.stride != 1 || L.kh != L.kw || L.kh != 2 * L.pad + 1) return false;
+  if (L.kh != L.kw || L.kh != 2 * L.pad + 1) return false;
+  const bool s2 = L.stride == 2;
+  if (L.stride != 1 && !s2) return false;
+  // stride 2: 3x3 kernels over even extents; the patch is four sub-images of the input
+  if (s2 && (L.kh != 3 || (L.h & 1) || (L.w & 1))) return false;
   if (L.c_in % 64 != 0) return false;
   if (!(L.c_p == 16 || L.c_p == 32 || L.c_p % 64 == 0)) return false;
   if (L.c_out % 64 != 0) return false;
-  if (L.w + L.pad > kBM) return false;
+  const int xpad = s2 ? 1 : L.pad;                  // zero columns/rows shared between patch rows
+  if (L.wo + xpad > kBM) return false;
   P.elem_bytes = 2;
   P.ck = 64;
-  P.wp = L.w + L.pad;
-  P.ip = (L.h + L.pad) * P.wp;
+  P.planes = s2 ? 4 : 1;
+  P.wp = L.wo + xpad;
+  P.ip = (L.ho + xpad) * P.wp;
   // rows of one image that fit 128 patch rows; or whole images if at least two fit
-  const int last_valid_one_image = (L.h - 1) * P.wp + L.w - 1;
+  const int last_valid_one_image = (L.ho - 1) * P.wp + L.wo - 1;
   if (last_valid_one_image + P.ip <= kBM - 1) {
     P.images_mode = 1;
     P.ni = 1 + (kBM - 1 - last_valid_one_image) / P.ip;
-    P.r = L.h;
+    P.r = L.ho;
     P.tiles_per_image = 1;
     P.tiles_m = (L.n + P.ni - 1) / P.ni;
-    P.box_h = L.h + L.pad;
-    P.out_box_h = L.h + L.pad;
+    P.box_h = L.ho + xpad;
+    P.out_box_h = L.ho + xpad;
   } else {
     P.images_mode = 0;
     P.ni = 1;
     const int rmax = kBM / P.wp;
-    const int tiles = (L.h + rmax - 1) / rmax;
-    P.r = (L.h + tiles - 1) / tiles;
+    const int tiles = (L.ho + rmax - 1) / rmax;
+    P.r = (L.ho + tiles - 1) / tiles;
     P.tiles_per_image = tiles;
     P.tiles_m = L.n * tiles;
-    P.box_h = P.r + 2 * L.pad;
+    P.box_h = s2 ? P.r + 1 : P.r + 2 * L.pad;
     P.out_box_h = P.r;
   }
   if (P.box_h > 256 || P.wp > 256 || P.ni > 256) return false;
   P.box_pixels = P.wp * P.box_h * P.ni;
-  P.patch_rows = (int)align_up((size_t)kBM + (size_t)(L.kh - 1) * (P.wp + 1), 8);
+  P.patch_rows = (int)align_up((size_t)kBM + (size_t)(s2 ? 1 : L.kh - 1) * (P.wp + 1), 8);
   if (P.box_pixels > P.patch_rows) P.patch_rows = (int)align_up(P.box_pixels, 8);
   P.patch_bytes = (int)align_up((size_t)P.patch_rows * 128, 1024);
   P.chunks = L.c_in / 64;
@@ -775,19 +813,20 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
     const size_t w_tile = (size_t)nt * 128;
     const size_t w_all = (size_t)(P.base_tiles + P.cond_tiles) * w_tile;
     int na = 0, nb = 0, resident = 0;
-    if (fixed + w_all + 2 * (size_t)P.patch_bytes <= limit) {
+    const int na_min = 2 * P.planes, na_max = 4 * P.planes > 8 ? 8 : 4 * P.planes;
+    if (fixed + w_all + (size_t)na_min * P.patch_bytes <= limit) {
       resident = 1;
       na = (int)((limit - fixed - w_all) / P.patch_bytes);
-      if (na > 4) na = 4;
+      if (na > na_max) na = na_max;
     } else {
       bool found = false;
       for (nb = 6; nb >= 3 && !found; --nb) {
-        if (fixed + nb * w_tile + 2 * (size_t)P.patch_bytes > limit) continue;
+        if (fixed + nb * w_tile + (size_t)P.planes * P.patch_bytes > limit) continue;
         na = (int)((limit - fixed - nb * w_tile) / P.patch_bytes);
-        if (na > 4) na = 4;
-        if (na >= 3 || nb == 3) { found = true; break; }
+        if (na > na_max) na = na_max;
+        if (na >= na_min || nb == 3) { found = true; break; }
       }
-      if (!found || na < 2) continue;
+      if (!found || na < P.planes) continue;
     }
     size_t off = 0;
     P.off_b = (unsigned)off; off += resident ? w_all : nb * w_tile;
@@ -831,12 +870,24 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
     maps->next = (maps->next + 1) % TcMaps::kEntries;
     ms->key[0] = nullptr;
     const int taps = L.kh * L.kw;
-    {
+    if (L.stride == 1) {
       cuuint64_t dims[4] = {(cuuint64_t)L.c_in, (cuuint64_t)L.w, (cuuint64_t)L.h, (cuuint64_t)L.n};
       cuuint64_t str[3] = {(cuuint64_t)L.c_in * 2, (cuuint64_t)L.w * L.c_in * 2,
                            (cuuint64_t)L.h * L.w * L.c_in * 2};
       cuuint32_t box[4] = {64, (cuuint32_t)P.wp, (cuuint32_t)P.box_h, (cuuint32_t)P.ni};
-      if (!encode(&ms->x, const_cast<void*>(x), 4, dims, str, box)) return (int)cudaErrorInvalidValue;
+      if (!encode(&ms->x[0], const_cast<void*>(x), 4, dims, str, box)) return (int)cudaErrorInvalidValue;
+      ms->x[1] = ms->x[2] = ms->x[3] = ms->x[0];
+    } else {
+      // plane 2*ph + pw holds the input pixels (2a + ph, 2b + pw)
+      for (int pl = 0; pl < 4; ++pl) {
+        const int ph = pl >> 1, pw = pl & 1;
+        const char* base = static_cast<const char*>(x) + ((size_t)ph * L.w + pw) * L.c_in * 2;
+        cuuint64_t dims[4] = {(cuuint64_t)L.c_in, (cuuint64_t)L.w / 2, (cuuint64_t)L.h / 2, (cuuint64_t)L.n};
+        cuuint64_t str[3] = {(cuuint64_t)2 * L.c_in * 2, (cuuint64_t)2 * L.w * L.c_in * 2,
+                             (cuuint64_t)L.h * L.w * L.c_in * 2};
+        cuuint32_t box[4] = {64, (cuuint32_t)P.wp, (cuuint32_t)P.box_h, (cuuint32_t)P.ni};
+        if (!encode(&ms->x[pl], const_cast<char*>(base), 4, dims, str, box)) return (int)cudaErrorInvalidValue;
+      }
     }
     {
       cuuint64_t dims[2] = {(cuuint64_t)taps * L.c_p, (cuuint64_t)L.c_out};
@@ -876,7 +927,7 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
       if (e != cudaSuccess) return (int)e;
       attr128 = true;
     }
-    tc_gated_conv_kernel<128><<<grid, kThreads, P.smem_bytes, stream>>>(ms->x, ms->wb, ms->wc, ms->y, prm);
+    tc_gated_conv_kernel<128><<<grid, kThreads, P.smem_bytes, stream>>>(ms->x[0], ms->x[1], ms->x[2], ms->x[3], ms->wb, ms->wc, ms->y, prm);
   } else {
     static bool attr64 = false;
     if (!attr64) {
@@ -884,7 +935,7 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
       if (e != cudaSuccess) return (int)e;
       attr64 = true;
     }
-    tc_gated_conv_kernel<64><<<grid, kThreads, P.smem_bytes, stream>>>(ms->x, ms->wb, ms->wc, ms->y, prm);
+    tc_gated_conv_kernel<64><<<grid, kThreads, P.smem_bytes, stream>>>(ms->x[0], ms->x[1], ms->x[2], ms->x[3], ms->wb, ms->wc, ms->y, prm);
   }
   return (int)cudaGetLastError();
 }

@@ -21,6 +21,8 @@ struct TcPlan {
   int tiles_m, tiles_n, nt;
   int chunks;           // c_in / ck input-channel chunks
   int base_chunks;      // chunks that hold base-path channels
+  int planes;           // patch buffers per chunk: 1 (stride 1) or 4 (stride 2: the input's
+                        // even/odd row x even/odd column sub-images)
   int na;               // patch buffers in the ring
   int nb;               // weight-tile ring depth (0 when the weights are resident)
   int resident;         // 1: all weight tiles of a column tile stay in shared memory
@@ -37,7 +39,7 @@ struct TcPlan {
 
 struct TcMapSet {
   const void* key[4];   // x, w_base, w_cond, y the maps below were encoded for
-  CUtensorMap x, wb, wc, y;
+  CUtensorMap x[4], wb, wc, y;   // x[1..3] only for stride 2
 };
 
 // Small cache of encoded tensor maps, so that callers that rotate a few buffers do not pay

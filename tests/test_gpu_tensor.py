@@ -30,6 +30,10 @@ SHAPES = [
     (O.Shape(12, 56, 56, 64, 64, groups=4), "336 row tiles: up to three jobs per CTA, resident weights"),
     (O.Shape(50, 28, 28, 128, 128, groups=4), "350 row tiles: streamed weights, three jobs per CTA"),
     (O.Shape(40, 14, 14, 256, 256, groups=4), "80 row tiles x 2 column tiles, two jobs per CTA"),
+    (O.Shape(3, 56, 56, 64, 128, stride=2, groups=4), "stride 2, 56->28, c_p = 16"),
+    (O.Shape(3, 28, 28, 128, 256, stride=2, groups=4), "stride 2, 28->14, c_p = 32"),
+    (O.Shape(5, 14, 14, 256, 512, stride=2, groups=4), "stride 2, 14->7, c_p = 64, two images per tile"),
+    (O.Shape(2, 12, 20, 64, 64, stride=2, groups=2), "stride 2, odd tile split, G = 2"),
 ]
 
 
