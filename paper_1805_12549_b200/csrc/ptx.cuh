@@ -165,6 +165,19 @@ __device__ __forceinline__ void umma_bf16_if(uint32_t issue, uint32_t d_tmem, ui
       "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(issue)
       : "memory");
 }
+// Predicated int8 MMA (signed 8-bit operands, int32 accumulator, K = 32 per instruction).
+__device__ __forceinline__ void umma_s8_if(uint32_t issue, uint32_t d_tmem, uint64_t a_desc,
+                                           uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      " .reg .pred p, q;\n"
+      " setp.ne.b32 p, %4, 0;\n"
+      " setp.ne.b32 q, %5, 0;\n"
+      " @q tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n"
+      "}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(issue)
+      : "memory");
+}
 __device__ __forceinline__ void umma_commit_if(uint32_t issue, uint64_t* bar) {
   asm volatile(
       "{\n"

@@ -42,7 +42,8 @@ constexpr int kThreads = 352;       // 3 single-role warps + 8 epilogue warps
 constexpr int kEpiThread0 = 96;     // first epilogue thread
 constexpr int kEpiThreads = 256;
 constexpr int kBM = 128;            // MMA M: patch rows per job
-constexpr int kSpinLimit = 1 << 21; // try_wait polls (each up to ~2 us) before a wait gives up
+constexpr int kSpinLimit = 1 << 21; // try_wait polls before a wait gives up ...
+constexpr long long kWaitCycles = 2000000000ll;   // ... or about one second of SM clocks, whichever is first
 constexpr int kMaxWTiles = 192;     // weight tiles per job, both phases
 constexpr bool kUnroll3x3 = true;   // fully unrolled 3x3 issue code (measured faster than rolled tap loops)
 
@@ -65,25 +66,26 @@ struct WTile {
 // per tap when c_p >= 64; when c_p < 64 a tile covers 64/c_p taps of chunk 0.  Conditional
 // path: chunk-major, one tile per tap; when c_p < 64 chunk 0 comes first with the K slices
 // behind the base channels.
-__device__ __forceinline__ WTile base_tile(const LayerDims& L, int bt) {
+// (ck = channels per 128-byte patch row: 64 for bf16, 128 for int8.)
+__device__ __forceinline__ WTile base_tile(const LayerDims& L, int ck, int bt) {
   const int taps = L.kh * L.kw;
-  if (L.c_p >= 64) {
+  if (L.c_p >= ck) {
     const int q = bt / taps, t = bt - q * taps;
-    return {t * L.c_p + 64 * q, q};
+    return {t * L.c_p + ck * q, q};
   }
-  return {bt * 64, 0};
+  return {bt * ck, 0};
 }
 
-__device__ __forceinline__ WTile cond_tile(const LayerDims& L, int bt) {
+__device__ __forceinline__ WTile cond_tile(const LayerDims& L, int ck, int bt) {
   const int taps = L.kh * L.kw;
-  if (L.c_p >= 64) {
-    const int q = L.c_p / 64 + bt / taps, t = bt % taps;
-    return {t * L.c_r + 64 * q - L.c_p, q};
+  if (L.c_p >= ck) {
+    const int q = L.c_p / ck + bt / taps, t = bt % taps;
+    return {t * L.c_r + ck * q - L.c_p, q};
   }
   if (bt < taps) return {bt * L.c_r, 0};
   const int b2 = bt - taps;
   const int q = 1 + b2 / taps, t = b2 % taps;
-  return {t * L.c_r + 64 * q - L.c_p, q};
+  return {t * L.c_r + ck * q - L.c_p, q};
 }
 
 struct Shared {
@@ -103,13 +105,17 @@ struct Ctx {
 };
 
 // Bounded wait.  The first poll is inline; the loop lives in one out-of-line copy so that the
-// role loops stay small.  Each poll parks the thread in hardware for up to ~2 us, so the bound
-// is a few seconds; a CTA that already gave up elsewhere is noticed within a few polls.
+// role loops stay small.  Each poll parks the thread in hardware for a short time; the wait
+// gives up after about a second; a CTA that already gave up elsewhere is noticed within a few polls.
 __device__ __noinline__ bool wait_bar_slow(Shared* sh, unsigned long long* counters, uint64_t* bar,
                                            uint32_t parity, int site) {
+  const long long t0 = clock64();
   for (int i = 0; i < kSpinLimit; ++i) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
-    if ((i & 15) == 15 && *(volatile uint32_t*)&sh->abort_flag) return false;
+    if ((i & 15) == 15) {
+      if (*(volatile uint32_t*)&sh->abort_flag) return false;
+      if (clock64() - t0 > kWaitCycles) break;
+    }
   }
   if (atomicCAS(&counters[CNT_STATUS], 0ull, (unsigned long long)CG_ERR_DEVICE_TIMEOUT) == 0ull)
     atomicExch(&counters[CNT_SITE], (unsigned long long)site);
@@ -134,7 +140,7 @@ __device__ __forceinline__ uint32_t slot_blocks(const Shared* sh, int slot) {
 // dependent scalar instruction between two MMAs is tensor idle time.)  Weight tiles are
 // visited in the order base_tile()/cond_tile() enumerate them, which is the order the weight
 // producer loads them.
-template <int NT>
+template <int NT, bool I8>
 struct MmaIssuer {
   Shared* sh;
   Ctx cx;
@@ -142,7 +148,7 @@ struct MmaIssuer {
   uint32_t desc_hi;                      // upper descriptor word (see ptx::smem_desc)
   uint32_t a_base_lo, b_base_lo;         // lower descriptor words of the ring bases
   uint32_t patch_lo, wtile_lo, row_lo;   // buffer sizes / one patch pixel row, in 16-byte units
-  int resident, na, nb, kp16, chunks, base_chunks, base_tiles, kh, kw, planes;
+  int resident, na, nb, kp16 /* base K steps per tap */, chunks, base_chunks, base_tiles, kh, kw, planes;
   int as, bs;                            // ring slots and the parities of their "full" barriers
   uint32_t apar, bpar;
   // per phase
@@ -163,7 +169,7 @@ struct MmaIssuer {
     patch_lo = (uint32_t)P.patch_bytes >> 4;
     wtile_lo = (uint32_t)(NT * 128) >> 4;
     row_lo = (uint32_t)P.wp * 8u;
-    resident = P.resident; na = P.na; nb = P.nb; kp16 = L.c_p / 16; chunks = P.chunks;
+    resident = P.resident; na = P.na; nb = P.nb; kp16 = L.c_p / (P.ck / 4); chunks = P.chunks;
     base_chunks = P.base_chunks; base_tiles = P.base_tiles; kh = L.kh; kw = L.kw; planes = P.planes;
     as = 0; bs = 0; apar = 0; bpar = 0;
     b_held = 0; ok = true;
@@ -172,11 +178,10 @@ struct MmaIssuer {
   template <bool ALL>
   __device__ __forceinline__ void mma(uint32_t al, uint32_t bl) {
     const uint64_t da = ((uint64_t)desc_hi << 32) | al;
-    if (ALL)
-      ptx::umma_bf16_if(issue, d_tmem, da, ((uint64_t)desc_hi << 32) | bl, ptx::idesc_bf16(kBM, NT), acc);
-    else   // exactly one of the two 64-channel column blocks
-      ptx::umma_bf16_if(issue, d_tmem + blk_off_d, da, ((uint64_t)desc_hi << 32) | (bl + blk_off_b),
-                        ptx::idesc_bf16(kBM, 64), acc);
+    const uint64_t db = ((uint64_t)desc_hi << 32) | (ALL ? bl : bl + blk_off_b);
+    const uint32_t d = ALL ? d_tmem : d_tmem + blk_off_d;   // !ALL: exactly one of two 64-column blocks
+    if (I8) ptx::umma_s8_if(issue, d, da, db, ptx::idesc_s8(kBM, ALL ? NT : 64), acc);
+    else ptx::umma_bf16_if(issue, d, da, db, ptx::idesc_bf16(kBM, ALL ? NT : 64), acc);
     acc = 1u;
   }
   // the patch buffer(s) of the next chunk in the ring: one, or the four planes of a stride-2 layer
@@ -316,7 +321,7 @@ struct MmaIssuer {
   }
 };
 
-template <int NT>
+template <int NT, bool I8>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
                      const __grid_constant__ CUtensorMap map_x1,
@@ -333,11 +338,18 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   uint8_t* s_a = smem + P.off_a;
   uint8_t* s_b = smem + P.off_b;
   uint8_t* s_y = smem + P.off_y;
+  // per-channel constants of this column tile.  Floating point: t, a1, b1, a2, b2.  Integer
+  // layers reuse the region: threshold, two multipliers (int32), two offsets (int64).
   float* s_t = (float*)(smem + P.off_consts);
   float* s_a1 = s_t + NT;
   float* s_b1 = s_a1 + NT;
   float* s_a2 = s_b1 + NT;
   float* s_b2 = s_a2 + NT;
+  int* s_qt = (int*)s_t;
+  int* s_qm1 = s_qt + NT;
+  int* s_qm2 = s_qm1 + NT;
+  long long* s_qo1 = (long long*)(s_qm2 + NT + (NT & 1));
+  long long* s_qo2 = s_qo1 + NT;
   uint32_t* s_mask = (uint32_t*)(smem + P.off_mask);       // [4][128][NT/32]
   int* s_wx = (int*)(smem + P.off_tables);                 // [base_tiles + cond_tiles] K coordinates
   Shared* sh = (Shared*)(smem + P.off_bar);
@@ -352,7 +364,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   const int taps = L.kh * L.kw;
   const bool dense = (P.cond_mode == CG_COND_DENSE);
   const bool has_cond = P.cond_tiles > 0;
-  const int cond_first_chunk = L.c_p >= 64 ? P.base_chunks : 0;
+  const int cond_first_chunk = L.c_p >= P.ck ? P.base_chunks : 0;
   constexpr int kBlocks = NT / 64;
   constexpr uint32_t kAllBlocks = (1u << kBlocks) - 1u;
   constexpr int kWords = NT / 32;
@@ -397,10 +409,17 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     }
     // K coordinate of every weight tile, for the weight producer
     for (int bt = et; bt < P.base_tiles + P.cond_tiles; bt += kEpiThreads)
-      s_wx[bt] = (bt < P.base_tiles ? base_tile(L, bt) : cond_tile(L, bt - P.base_tiles)).x;
+      s_wx[bt] = (bt < P.base_tiles ? base_tile(L, P.ck, bt) : cond_tile(L, P.ck, bt - P.base_tiles)).x;
     for (int c = et; c < NT; c += kEpiThreads) {
-      const ChannelConsts k = fold_channel(prm.bn, prm.delta, L.eps, tile_n * NT + c);
-      s_t[c] = k.t; s_a1[c] = k.a1; s_b1[c] = k.b1; s_a2[c] = k.a2; s_b2[c] = k.b2;
+      const int cg_ = tile_n * NT + c;
+      if (I8) {
+        s_qt[c] = prm.bn.q_gate_thr[cg_];
+        s_qm1[c] = prm.bn.q_mul_base[cg_]; s_qm2[c] = prm.bn.q_mul_full[cg_];
+        s_qo1[c] = prm.bn.q_off_base[cg_]; s_qo2[c] = prm.bn.q_off_full[cg_];
+      } else {
+        const ChannelConsts k = fold_channel(prm.bn, prm.delta, L.eps, cg_);
+        s_t[c] = k.t; s_a1[c] = k.a1; s_b1[c] = k.b1; s_a2[c] = k.a2; s_b2[c] = k.b2;
+      }
     }
     ptx::fence_proxy_async();
   }
@@ -426,7 +445,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
             if (!ok) return;
             const CUtensorMap* mx = pl == 0 ? &map_x : (pl == 1 ? &map_x1 : (pl == 2 ? &map_x2 : &map_x3));
             ptx::mbar_expect_tx(&sh->a_full[as], patch_tx);
-            ptx::tma_load_4d(s_a + (size_t)as * P.patch_bytes, mx, &sh->a_full[as], q * 64, -lead,
+            ptx::tma_load_4d(s_a + (size_t)as * P.patch_bytes, mx, &sh->a_full[as], q * P.ck, -lead,
                              h0 - lead, n0);
             if (++as == P.na) { as = 0; apar ^= 1; }
           }
@@ -489,7 +508,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   } else if (warp == 1) {
     // ============================================================ MMA issuer
     if (jobs > 0) {
-      MmaIssuer<NT> mi;
+      MmaIssuer<NT, I8> mi;
       mi.init(sh, cx, s_a, s_b, P, L, lane);
       bool ok = true;
       if (P.resident) ok = wait_bar(cx, &sh->w_ready, 0, 6);
@@ -513,13 +532,18 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
               if (!ok) break;
               blocks = slot_blocks(sh, jj % kNP);
             }
+            // the R slot's previous user must be done with it even when this job skips the
+            // conditional path: otherwise cond_done could run two phases ahead of its waiters
+            ok = wait_bar(cx, &sh->r_free[rs], ((jj / kNR) & 1) ^ 1, 14);
+            if (!ok) break;
             if (blocks) {
-              ok = wait_bar(cx, &sh->r_free[rs], ((jj / kNR) & 1) ^ 1, 14);
-              if (!ok) break;
               ptx::tc_fence_after();
               ok = mi.run_phase(tmem + (uint32_t)((kNP + rs) * NT), true, blocks);
               if (!ok) break;
             }
+          } else {
+            ok = wait_bar(cx, &sh->r_free[rs], ((jj / kNR) & 1) ^ 1, 15);
+            if (!ok) break;
           }
           ptx::umma_commit_if(mi.issue, &sh->cond_done[rs]);
         }
@@ -562,11 +586,19 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         uint32_t word = 0;
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
-          const float4 t4 = *(const float4*)(s_t + cb * 32 + q * 4);
-          word |= (__uint_as_float(r[q * 4 + 0]) >= t4.x ? 1u : 0u) << (q * 4 + 0);
-          word |= (__uint_as_float(r[q * 4 + 1]) >= t4.y ? 1u : 0u) << (q * 4 + 1);
-          word |= (__uint_as_float(r[q * 4 + 2]) >= t4.z ? 1u : 0u) << (q * 4 + 2);
-          word |= (__uint_as_float(r[q * 4 + 3]) >= t4.w ? 1u : 0u) << (q * 4 + 3);
+          if (I8) {
+            const int4 t4 = *(const int4*)(s_qt + cb * 32 + q * 4);
+            word |= ((int)r[q * 4 + 0] >= t4.x ? 1u : 0u) << (q * 4 + 0);
+            word |= ((int)r[q * 4 + 1] >= t4.y ? 1u : 0u) << (q * 4 + 1);
+            word |= ((int)r[q * 4 + 2] >= t4.z ? 1u : 0u) << (q * 4 + 2);
+            word |= ((int)r[q * 4 + 3] >= t4.w ? 1u : 0u) << (q * 4 + 3);
+          } else {
+            const float4 t4 = *(const float4*)(s_t + cb * 32 + q * 4);
+            word |= (__uint_as_float(r[q * 4 + 0]) >= t4.x ? 1u : 0u) << (q * 4 + 0);
+            word |= (__uint_as_float(r[q * 4 + 1]) >= t4.y ? 1u : 0u) << (q * 4 + 1);
+            word |= (__uint_as_float(r[q * 4 + 2]) >= t4.z ? 1u : 0u) << (q * 4 + 2);
+            word |= (__uint_as_float(r[q * 4 + 3]) >= t4.w ? 1u : 0u) << (q * 4 + 3);
+          }
         }
         if (!valid) word = 0;
         s_mask[(slot * 128 + row) * kWords + cb] = word;
@@ -619,31 +651,61 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
 #pragma unroll
           for (int i = 0; i < 32; ++i) rr[i] = 0u;
         }
-        uint8_t* st = s_y + (size_t)(cb >> 1) * P.stage_rows * 128 + (size_t)row * 128;
+        if (I8) {
+          // quantised layer: z = acc*mul + off (64-bit), q = (z + 2^(S-1)) >> S, clamp to int8;
+          // 32 channels = 32 bytes = two 16-byte pieces of a 128-channel staging row
+          uint8_t* st = s_y + (size_t)(cb >> 2) * P.stage_rows * 128 + (size_t)row * 128;
+          const long long half_ulp = 1ll << (L.shift - 1);
+          const int lo = L.relu ? 0 : -128;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          uint32_t packed[4];
+          for (int q = 0; q < 2; ++q) {
+            uint32_t packed[4];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int jx = q * 8 + e * 2;
-            const int c = cb * 32 + jx;
-            const float2 a1 = *(const float2*)(s_a1 + c), b1 = *(const float2*)(s_b1 + c);
-            const float2 a2 = *(const float2*)(s_a2 + c), b2 = *(const float2*)(s_b2 + c);
-            const bool f0 = (word >> jx) & 1u, f1 = (word >> (jx + 1)) & 1u;
-            const float p0 = __uint_as_float(p[jx]), p1 = __uint_as_float(p[jx + 1]);
-            // Eq. 1: the full sum P+R where the gate fired, the partial sum elsewhere; then the
-            // batch norm of that path (Section 4) as one multiply and one add
-            const float s0 = f0 ? __fadd_rn(p0, __uint_as_float(rr[jx])) : p0;
-            const float s1 = f1 ? __fadd_rn(p1, __uint_as_float(rr[jx + 1])) : p1;
-            float v0 = __fadd_rn(__fmul_rn(f0 ? a2.x : a1.x, s0), f0 ? b2.x : b1.x);
-            float v1 = __fadd_rn(__fmul_rn(f1 ? a2.y : a1.y, s1), f1 ? b2.y : b1.y);
-            if (L.relu) { v0 = v0 > 0.f ? v0 : 0.f; v1 = v1 > 0.f ? v1 : 0.f; }
-            const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
-            packed[e] = *(const uint32_t*)&h2;
+            for (int e = 0; e < 4; ++e) {
+              uint32_t w4 = 0;
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const int jx = q * 16 + e * 4 + k;
+                const int c = cb * 32 + jx;
+                const bool f = (word >> jx) & 1u;
+                const long long acc = f ? (long long)(int)p[jx] + (long long)(int)rr[jx] : (long long)(int)p[jx];
+                const long long z = acc * (long long)(f ? s_qm2[c] : s_qm1[c]) + (f ? s_qo2[c] : s_qo1[c]);
+                long long qv = (z + half_ulp) >> L.shift;
+                qv = qv < lo ? lo : (qv > 127 ? 127 : qv);
+                w4 |= ((uint32_t)qv & 0xffu) << (8 * k);
+              }
+              packed[e] = w4;
+            }
+            const int c16 = (cb & 3) * 2 + q;
+            *(uint4*)(st + ((c16 ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
           }
-          const int c16 = (cb & 1) * 4 + q;
-          *(uint4*)(st + ((c16 ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-        }
+        } else {
+          uint8_t* st = s_y + (size_t)(cb >> 1) * P.stage_rows * 128 + (size_t)row * 128;
+  #pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            uint32_t packed[4];
+  #pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const int jx = q * 8 + e * 2;
+              const int c = cb * 32 + jx;
+              const float2 a1 = *(const float2*)(s_a1 + c), b1 = *(const float2*)(s_b1 + c);
+              const float2 a2 = *(const float2*)(s_a2 + c), b2 = *(const float2*)(s_b2 + c);
+              const bool f0 = (word >> jx) & 1u, f1 = (word >> (jx + 1)) & 1u;
+              const float p0 = __uint_as_float(p[jx]), p1 = __uint_as_float(p[jx + 1]);
+              // Eq. 1: the full sum P+R where the gate fired, the partial sum elsewhere; then the
+              // batch norm of that path (Section 4) as one multiply and one add
+              const float s0 = f0 ? __fadd_rn(p0, __uint_as_float(rr[jx])) : p0;
+              const float s1 = f1 ? __fadd_rn(p1, __uint_as_float(rr[jx + 1])) : p1;
+              float v0 = __fadd_rn(__fmul_rn(f0 ? a2.x : a1.x, s0), f0 ? b2.x : b1.x);
+              float v1 = __fadd_rn(__fmul_rn(f1 ? a2.y : a1.y, s1), f1 ? b2.y : b1.y);
+              if (L.relu) { v0 = v0 > 0.f ? v0 : 0.f; v1 = v1 > 0.f ? v1 : 0.f; }
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
+              packed[e] = *(const uint32_t*)&h2;
+            }
+            const int c16 = (cb & 1) * 4 + q;
+            *(uint4*)(st + ((c16 ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+          }
+              }
       }
       ptx::tc_fence_before();
       ptx::mbar_arrive(&sh->p_free[slot]);
@@ -653,9 +715,10 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       if (et == 0) {
         int n0, h0;
         job_origin(j, n0, h0);
+        constexpr int kStoreCh = I8 ? 128 : 64;   // channels per 128-byte staging row
 #pragma unroll
-        for (int b = 0; b < kBlocks; ++b)
-          ptx::tma_store_4d(&map_y, s_y + (size_t)b * P.stage_rows * 128, tile_n * NT + b * 64, 0, h0, n0);
+        for (int b = 0; b < NT / kStoreCh; ++b)
+          ptx::tma_store_4d(&map_y, s_y + (size_t)b * P.stage_rows * 128, tile_n * NT + b * kStoreCh, 0, h0, n0);
         ptx::tma_store_commit();
       }
     };
@@ -713,12 +776,12 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-bool encode(CUtensorMap* map, void* base, int rank, const cuuint64_t* dims,
+bool encode(CUtensorMap* map, int elem_bytes, void* base, int rank, const cuuint64_t* dims,
             const cuuint64_t* strides_bytes, const cuuint32_t* box) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
   cuuint32_t es[5] = {1, 1, 1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, base, dims, strides_bytes, box,
+  return fn(map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, base, dims, strides_bytes, box,
             es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -742,20 +805,23 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
   TcPlan P;
   std::memset(&P, 0, sizeof(P));
   *plan = P;
-  if (in_dtype != CG_BF16) return false;
+  if (in_dtype != CG_BF16 && in_dtype != CG_I8) return false;
+  const int eb = in_dtype == CG_BF16 ? 2 : 1;
+  const int ck = 128 / eb;          // channels per 128-byte patch row
+  const int kst = ck / 4;           // channels per MMA K step (32 bytes)
   if (L.has_residual) return false;
   if (L.kh != L.kw || L.kh != 2 * L.pad + 1) return false;
   const bool s2 = L.stride == 2;
   if (L.stride != 1 && !s2) return false;
   // stride 2: 3x3 kernels over even extents; the patch is four sub-images of the input
   if (s2 && (L.kh != 3 || (L.h & 1) || (L.w & 1))) return false;
-  if (L.c_in % 64 != 0) return false;
-  if (!(L.c_p == 16 || L.c_p == 32 || L.c_p % 64 == 0)) return false;
-  if (L.c_out % 64 != 0) return false;
+  if (L.c_in % ck != 0) return false;
+  if (!(L.c_p == kst || L.c_p == 2 * kst || L.c_p % ck == 0)) return false;
+  if (L.c_out % 64 != 0 || (eb == 1 && L.c_out % 128 != 0)) return false;
   const int xpad = s2 ? 1 : L.pad;                  // zero columns/rows shared between patch rows
   if (L.wo + xpad > kBM) return false;
-  P.elem_bytes = 2;
-  P.ck = 64;
+  P.elem_bytes = eb;
+  P.ck = ck;
   P.planes = s2 ? 4 : 1;
   P.wp = L.wo + xpad;
   P.ip = (L.ho + xpad) * P.wp;
@@ -785,14 +851,14 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
   P.patch_rows = (int)align_up((size_t)kBM + (size_t)(s2 ? 1 : L.kh - 1) * (P.wp + 1), 8);
   if (P.box_pixels > P.patch_rows) P.patch_rows = (int)align_up(P.box_pixels, 8);
   P.patch_bytes = (int)align_up((size_t)P.patch_rows * 128, 1024);
-  P.chunks = L.c_in / 64;
-  P.base_chunks = L.c_p >= 64 ? L.c_p / 64 : 1;
+  P.chunks = L.c_in / ck;
+  P.base_chunks = L.c_p >= ck ? L.c_p / ck : 1;
   const int taps = L.kh * L.kw;
-  if (L.c_p >= 64) {
-    P.base_tiles = (L.c_p / 64) * taps;
-    P.cond_tiles = (P.chunks - L.c_p / 64) * taps;
+  if (L.c_p >= ck) {
+    P.base_tiles = (L.c_p / ck) * taps;
+    P.cond_tiles = (P.chunks - L.c_p / ck) * taps;
   } else {
-    const int tpt = 64 / L.c_p;
+    const int tpt = ck / L.c_p;
     P.base_tiles = (taps + tpt - 1) / tpt;
     P.cond_tiles = L.c_r > 0 ? P.chunks * taps : 0;
   }
@@ -804,10 +870,10 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
   // [mask stash][tile coordinates][barriers]; widest column tile first, resident weights if
   // they fit next to at least two patch buffers
   const size_t limit = 227 * 1024 - 1024;
-  for (int nt = 128; nt >= 64; nt >>= 1) {
+  for (int nt = 128; nt >= (eb == 1 ? 128 : 64); nt >>= 1) {
     if (L.c_out % nt != 0) continue;
-    const size_t fixed = align_up((size_t)(nt / 64) * P.stage_rows * 128, 1024) +
-                         align_up((size_t)5 * nt * 4, 128) +
+    const size_t fixed = align_up((size_t)(nt * eb / 128) * P.stage_rows * 128, 1024) +
+                         align_up((size_t)8 * nt * 4, 128) +
                          align_up((size_t)4 * 128 * (nt / 32) * 4, 128) +
                          align_up((size_t)kMaxWTiles * 4, 128) + align_up(sizeof(Shared), 128);
     const size_t w_tile = (size_t)nt * 128;
@@ -831,8 +897,8 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
     size_t off = 0;
     P.off_b = (unsigned)off; off += resident ? w_all : nb * w_tile;
     P.off_a = (unsigned)off; off += (size_t)na * P.patch_bytes;
-    P.off_y = (unsigned)off; off += align_up((size_t)(nt / 64) * P.stage_rows * 128, 1024);
-    P.off_consts = (unsigned)off; off += align_up((size_t)5 * nt * 4, 128);
+    P.off_y = (unsigned)off; off += align_up((size_t)(nt * eb / 128) * P.stage_rows * 128, 1024);
+    P.off_consts = (unsigned)off; off += align_up((size_t)8 * nt * 4, 128);
     P.off_mask = (unsigned)off; off += align_up((size_t)4 * 128 * (nt / 32) * 4, 128);
     P.off_tables = (unsigned)off; off += align_up((size_t)kMaxWTiles * 4, 128);
     P.off_bar = (unsigned)off; off += align_up(sizeof(Shared), 128);
@@ -870,45 +936,47 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
     maps->next = (maps->next + 1) % TcMaps::kEntries;
     ms->key[0] = nullptr;
     const int taps = L.kh * L.kw;
+    const cuuint64_t eb = (cuuint64_t)P.elem_bytes;
+    const cuuint32_t ck = (cuuint32_t)P.ck;
     if (L.stride == 1) {
       cuuint64_t dims[4] = {(cuuint64_t)L.c_in, (cuuint64_t)L.w, (cuuint64_t)L.h, (cuuint64_t)L.n};
-      cuuint64_t str[3] = {(cuuint64_t)L.c_in * 2, (cuuint64_t)L.w * L.c_in * 2,
-                           (cuuint64_t)L.h * L.w * L.c_in * 2};
-      cuuint32_t box[4] = {64, (cuuint32_t)P.wp, (cuuint32_t)P.box_h, (cuuint32_t)P.ni};
-      if (!encode(&ms->x[0], const_cast<void*>(x), 4, dims, str, box)) return (int)cudaErrorInvalidValue;
+      cuuint64_t str[3] = {(cuuint64_t)L.c_in * eb, (cuuint64_t)L.w * L.c_in * eb,
+                           (cuuint64_t)L.h * L.w * L.c_in * eb};
+      cuuint32_t box[4] = {ck, (cuuint32_t)P.wp, (cuuint32_t)P.box_h, (cuuint32_t)P.ni};
+      if (!encode(&ms->x[0], P.elem_bytes, const_cast<void*>(x), 4, dims, str, box)) return (int)cudaErrorInvalidValue;
       ms->x[1] = ms->x[2] = ms->x[3] = ms->x[0];
     } else {
       // plane 2*ph + pw holds the input pixels (2a + ph, 2b + pw)
       for (int pl = 0; pl < 4; ++pl) {
         const int ph = pl >> 1, pw = pl & 1;
-        const char* base = static_cast<const char*>(x) + ((size_t)ph * L.w + pw) * L.c_in * 2;
+        const char* base = static_cast<const char*>(x) + ((size_t)ph * L.w + pw) * L.c_in * eb;
         cuuint64_t dims[4] = {(cuuint64_t)L.c_in, (cuuint64_t)L.w / 2, (cuuint64_t)L.h / 2, (cuuint64_t)L.n};
-        cuuint64_t str[3] = {(cuuint64_t)2 * L.c_in * 2, (cuuint64_t)2 * L.w * L.c_in * 2,
-                             (cuuint64_t)L.h * L.w * L.c_in * 2};
-        cuuint32_t box[4] = {64, (cuuint32_t)P.wp, (cuuint32_t)P.box_h, (cuuint32_t)P.ni};
-        if (!encode(&ms->x[pl], const_cast<char*>(base), 4, dims, str, box)) return (int)cudaErrorInvalidValue;
+        cuuint64_t str[3] = {(cuuint64_t)2 * L.c_in * eb, (cuuint64_t)2 * L.w * L.c_in * eb,
+                             (cuuint64_t)L.h * L.w * L.c_in * eb};
+        cuuint32_t box[4] = {ck, (cuuint32_t)P.wp, (cuuint32_t)P.box_h, (cuuint32_t)P.ni};
+        if (!encode(&ms->x[pl], P.elem_bytes, const_cast<char*>(base), 4, dims, str, box)) return (int)cudaErrorInvalidValue;
       }
     }
     {
       cuuint64_t dims[2] = {(cuuint64_t)taps * L.c_p, (cuuint64_t)L.c_out};
-      cuuint64_t str[1] = {(cuuint64_t)taps * L.c_p * 2};
-      cuuint32_t box[2] = {64, (cuuint32_t)P.nt};
-      if (!encode(&ms->wb, const_cast<void*>(w_base), 2, dims, str, box)) return (int)cudaErrorInvalidValue;
+      cuuint64_t str[1] = {(cuuint64_t)taps * L.c_p * eb};
+      cuuint32_t box[2] = {ck, (cuuint32_t)P.nt};
+      if (!encode(&ms->wb, P.elem_bytes, const_cast<void*>(w_base), 2, dims, str, box)) return (int)cudaErrorInvalidValue;
     }
     if (L.c_r > 0) {
       cuuint64_t dims[2] = {(cuuint64_t)taps * L.c_r, (cuuint64_t)L.c_out};
-      cuuint64_t str[1] = {(cuuint64_t)taps * L.c_r * 2};
-      cuuint32_t box[2] = {64, (cuuint32_t)P.nt};
-      if (!encode(&ms->wc, const_cast<void*>(w_cond), 2, dims, str, box)) return (int)cudaErrorInvalidValue;
+      cuuint64_t str[1] = {(cuuint64_t)taps * L.c_r * eb};
+      cuuint32_t box[2] = {ck, (cuuint32_t)P.nt};
+      if (!encode(&ms->wc, P.elem_bytes, const_cast<void*>(w_cond), 2, dims, str, box)) return (int)cudaErrorInvalidValue;
     } else {
       ms->wc = ms->wb;
     }
     {
       cuuint64_t dims[4] = {(cuuint64_t)L.c_out, (cuuint64_t)L.wo, (cuuint64_t)L.ho, (cuuint64_t)L.n};
-      cuuint64_t str[3] = {(cuuint64_t)L.c_out * 2, (cuuint64_t)L.wo * L.c_out * 2,
-                           (cuuint64_t)L.ho * L.wo * L.c_out * 2};
-      cuuint32_t box[4] = {64, (cuuint32_t)P.wp, (cuuint32_t)P.out_box_h, (cuuint32_t)P.ni};
-      if (!encode(&ms->y, y, 4, dims, str, box)) return (int)cudaErrorInvalidValue;
+      cuuint64_t str[3] = {(cuuint64_t)L.c_out * eb, (cuuint64_t)L.wo * L.c_out * eb,
+                           (cuuint64_t)L.ho * L.wo * L.c_out * eb};
+      cuuint32_t box[4] = {ck, (cuuint32_t)P.wp, (cuuint32_t)P.out_box_h, (cuuint32_t)P.ni};
+      if (!encode(&ms->y, P.elem_bytes, y, 4, dims, str, box)) return (int)cudaErrorInvalidValue;
     }
     ms->key[0] = x; ms->key[1] = w_base; ms->key[2] = wc_key; ms->key[3] = y;
   }
@@ -919,24 +987,21 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
   int grid = sms - sms % P.tiles_n;
   if (grid < P.tiles_n) grid = P.tiles_n;
   if (grid > P.tiles_m * P.tiles_n) grid = P.tiles_m * P.tiles_n;
-  cudaError_t e;
-  if (P.nt == 128) {
-    static bool attr128 = false;
-    if (!attr128) {
-      e = cudaFuncSetAttribute(tc_gated_conv_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-      if (e != cudaSuccess) return (int)e;
-      attr128 = true;
-    }
-    tc_gated_conv_kernel<128><<<grid, kThreads, P.smem_bytes, stream>>>(ms->x[0], ms->x[1], ms->x[2], ms->x[3], ms->wb, ms->wc, ms->y, prm);
-  } else {
-    static bool attr64 = false;
-    if (!attr64) {
-      e = cudaFuncSetAttribute(tc_gated_conv_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-      if (e != cudaSuccess) return (int)e;
-      attr64 = true;
-    }
-    tc_gated_conv_kernel<64><<<grid, kThreads, P.smem_bytes, stream>>>(ms->x[0], ms->x[1], ms->x[2], ms->x[3], ms->wb, ms->wc, ms->y, prm);
+  // kernel instances: <64, bf16>, <128, bf16>, <128, int8>
+  typedef void (*Kernel)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap,
+                         CUtensorMap, TcParams);
+  const int which = P.elem_bytes == 1 ? 2 : (P.nt == 128 ? 1 : 0);
+  const Kernel kernels[3] = {tc_gated_conv_kernel<64, false>, tc_gated_conv_kernel<128, false>,
+                             tc_gated_conv_kernel<128, true>};
+  static bool attr_set[3] = {false, false, false};
+  if (!attr_set[which]) {
+    const cudaError_t e = cudaFuncSetAttribute(kernels[which], cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               227 * 1024);
+    if (e != cudaSuccess) return (int)e;
+    attr_set[which] = true;
   }
+  kernels[which]<<<grid, kThreads, P.smem_bytes, stream>>>(ms->x[0], ms->x[1], ms->x[2], ms->x[3], ms->wb,
+                                                           ms->wc, ms->y, prm);
   return (int)cudaGetLastError();
 }
 

@@ -96,6 +96,17 @@ def test_idle_tiles_are_skipped():
     assert st.executed_macs == 128 * 64 * k2 * (s.c_p * 56 + s.c_r * (56 - st.tiles_skipped))
 
 
+@pytest.mark.parametrize("dv", [K.INF, -K.INF])
+def test_many_jobs_per_cta_all_shut_and_all_open(dv):
+    """Several jobs per CTA with every conditional phase skipped (or none): the barrier phases
+    of the skipped work must stay in step with the epilogue."""
+    s = O.Shape(30, 28, 28, 128, 128, groups=4)          # 210 row tiles on 148 CTAs
+    c = K.make_float_case("tcmany", s, "bf16", delta=dv)
+    ref, st, exempt = _run(c)
+    assert exempt == 0
+    assert st.tiles_skipped == (st.tiles_total if dv > 0 else 0)
+
+
 def test_two_calls_accumulate_and_are_deterministic():
     s = O.Shape(2, 28, 28, 128, 128, groups=4)
     c = K.make_float_case("tcdet", s, "bf16", density=0.3)
@@ -127,3 +138,29 @@ def test_full_size_layers_on_sampled_images(layer):
         c1 = K.Case(c.name, s1, c.dtype, c.x[n:n + 1], c.wb, c.wc, c.bn, c.delta)
         ref = K.run_oracle(c1)
         K.compare(c1, ref, y[n:n + 1], mask[n * per_img:(n + 1) * per_img].reshape(-1, words), None)
+
+
+I8_SHAPES = [
+    (O.Shape(2, 28, 28, 128, 128, groups=4), "int8 128@28, c_p = 32 bytes"),
+    (O.Shape(3, 14, 14, 256, 256, groups=4), "int8 256@14, c_p = 64 bytes, two column tiles"),
+    (O.Shape(5, 7, 7, 512, 512, groups=4), "int8 512@7, c_p = 128 bytes, two images per tile"),
+    (O.Shape(2, 28, 28, 128, 256, stride=2, groups=4), "int8 stride 2"),
+    (O.Shape(30, 28, 28, 128, 128, groups=2), "int8 G = 2, 210 row tiles"),
+]
+
+
+@pytest.mark.parametrize("s,why", I8_SHAPES, ids=[w for _, w in I8_SHAPES])
+@pytest.mark.parametrize("density", [0.3, 1.0, 0.0])
+def test_int8_tensor_path_is_bit_exact(s, why, density):
+    """Quantised layers on tcgen05 kind::i8: integer sums are order-independent, so masks and
+    int8 outputs must equal the oracle's bit for bit."""
+    c = K.make_int8_case("tci8", s, density=density)
+    ref = K.run_oracle(c)
+    g = K.GpuCase(c, algo=TENSOR)
+    assert g.conv.uses_tensor_cores
+    y, mask, st = g.run()
+    K.compare(c, ref, y, mask, st, exact=True)
+    assert st.active == ref.active
+    if density == 0.3:
+        assert 0.2 < st.density < 0.4 and len(np.unique(y)) > 16
+    g.close()
