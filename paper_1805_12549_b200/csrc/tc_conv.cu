@@ -885,12 +885,16 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
       na = (int)((limit - fixed - w_all) / P.patch_bytes);
       if (na > na_max) na = na_max;
     } else {
+      // streamed weights are latency-bound (bytes in flight per SM), so the weight ring gets
+      // the shared memory that three patch buffers (stride 1) or one set of planes leave
       bool found = false;
-      for (nb = 6; nb >= 3 && !found; --nb) {
-        if (fixed + nb * w_tile + (size_t)P.planes * P.patch_bytes > limit) continue;
+      const int na_want = P.planes == 1 ? 3 : P.planes;
+      for (nb = 8; nb >= 3 && !found; --nb) {
+        if (fixed + nb * w_tile + (size_t)na_want * P.patch_bytes > limit) continue;
         na = (int)((limit - fixed - nb * w_tile) / P.patch_bytes);
         if (na > na_max) na = na_max;
-        if (na >= na_min || nb == 3) { found = true; break; }
+        found = true;
+        break;
       }
       if (!found || na < P.planes) continue;
     }
