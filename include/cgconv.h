@@ -74,6 +74,11 @@ typedef struct {
   int32_t requant_shift;        /* I8 only: S in [1,31]                                        */
   int32_t algo;                 /* cg_algo                                                     */
   int32_t cond_mode;            /* cg_cond_mode (tensor-core path only)                        */
+  int32_t grouping;             /* 0: every output channel takes input channels [0,c_in/G) as
+                                   x_p (Fig. 5(a)).  1: channel grouping (Section 3.3, Fig. 5(b)):
+                                   output group i = channels [i*c_out/G,(i+1)*c_out/G) takes input
+                                   group i as x_p and the other groups, in ascending order, as
+                                   x_r; needs c_out % G == 0.  Direct kernels only for now.    */
 } cg_conv_desc;
 
 /* Per-output-channel parameters: DEVICE pointers to c_out entries, caller-owned.

@@ -30,7 +30,7 @@ class CgConvDesc(C.Structure):
                                          "pad", "groups", "in_dtype", "out_dtype")] + \
                [("bn_eps", C.c_float)] + \
                [(k, C.c_int32) for k in ("relu", "has_residual", "requant_shift", "algo",
-                                         "cond_mode")]
+                                         "cond_mode", "grouping")]
 
 
 class CgBnParams(C.Structure):
@@ -221,9 +221,10 @@ class GatedConv:
 
     def __init__(self, n, h, w, c_in, c_out, *, k=3, stride=1, pad=1, groups=4, dtype=CG_BF16,
                  bn_eps=1e-5, relu=True, has_residual=False, requant_shift=0,
-                 algo=CG_ALGO_AUTO, cond_mode=CG_COND_AUTO, device="cuda"):
+                 algo=CG_ALGO_AUTO, cond_mode=CG_COND_AUTO, grouping=False, device="cuda"):
         self.desc = CgConvDesc(n, h, w, c_in, c_out, k, k, stride, pad, groups, dtype, dtype,
-                               bn_eps, int(relu), int(has_residual), requant_shift, algo, cond_mode)
+                               bn_eps, int(relu), int(has_residual), requant_shift, algo, cond_mode,
+                               int(grouping))
         self.handle = cg_conv_create(self.desc)
         self.dtype = dtype
         self.ho = (h + 2 * pad - k) // stride + 1

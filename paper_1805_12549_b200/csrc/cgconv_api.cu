@@ -39,6 +39,9 @@ cg_status check_desc(const cg_conv_desc* d) {
   if (!(d->bn_eps >= 0.f)) return CG_ERR_INVALID_ARG;
   if (d->algo < CG_ALGO_AUTO || d->algo > CG_ALGO_TENSOR) return CG_ERR_INVALID_ARG;
   if (d->cond_mode < CG_COND_AUTO || d->cond_mode > CG_COND_COMPACT) return CG_ERR_INVALID_ARG;
+  if (d->grouping != 0 && d->grouping != 1) return CG_ERR_INVALID_ARG;
+  if (d->grouping && d->c_out % d->groups != 0) return CG_ERR_INVALID_ARG;
+  if (d->grouping && d->in_dtype == CG_I8) return CG_ERR_INVALID_ARG;   // not defined for I8 layers
   return CG_OK;
 }
 
@@ -53,6 +56,7 @@ cg::LayerDims make_dims(const cg_conv_desc& d) {
   L.words = (d.c_out + 31) / 32;
   L.eps = d.bn_eps; L.relu = d.relu ? 1 : 0; L.has_residual = d.has_residual ? 1 : 0;
   L.shift = d.requant_shift;
+  L.grouping = d.grouping;
   return L;
 }
 

@@ -19,6 +19,7 @@ struct LayerDims {
   int words;              // ceil(c_out / 32) mask words per pixel row
   float eps;
   int relu, has_residual, shift;
+  int grouping;           // 1: output group i uses input group i as x_p (Section 3.3)
 };
 
 // Device counter block owned by a handle: 16 x u64.

@@ -61,6 +61,51 @@ __device__ __forceinline__ int conv_point_i8(const LayerDims& L, const int8_t* _
   return acc;
 }
 
+// Channel grouping (Section 3.3): the conditional path of output group g reads every input
+// channel outside [g*c_p, (g+1)*c_p), in ascending order; weights are [c_out][kh][kw][c_r].
+template <typename T>
+__device__ __forceinline__ float conv_point_others(const LayerDims& L, const T* __restrict__ x,
+                                                   const T* __restrict__ w, int n, int ho, int wo,
+                                                   int co, int g) {
+  float acc = 0.f;
+  const int lo = g * L.c_p, hi2 = lo + L.c_p;
+  for (int r = 0; r < L.kh; ++r) {
+    const int hi = ho * L.stride + r - L.pad;
+    if (hi < 0 || hi >= L.h) continue;
+    for (int s = 0; s < L.kw; ++s) {
+      const int wi = wo * L.stride + s - L.pad;
+      if (wi < 0 || wi >= L.w) continue;
+      const T* xp = x + (((long long)n * L.h + hi) * L.w + wi) * L.c_in;
+      const T* wp = w + (((long long)co * L.kh + r) * L.kw + s) * L.c_r;
+      for (int ci = 0; ci < lo; ++ci)
+        acc = __fadd_rn(acc, __fmul_rn(Elem<T>::ld(xp + ci), Elem<T>::ld(wp + ci)));
+      for (int ci = hi2; ci < L.c_in; ++ci)
+        acc = __fadd_rn(acc, __fmul_rn(Elem<T>::ld(xp + ci), Elem<T>::ld(wp + ci - L.c_p)));
+    }
+  }
+  return acc;
+}
+
+__device__ __forceinline__ int conv_point_others_i8(const LayerDims& L, const int8_t* __restrict__ x,
+                                                    const int8_t* __restrict__ w, int n, int ho,
+                                                    int wo, int co, int g) {
+  int acc = 0;
+  const int lo = g * L.c_p, hi2 = lo + L.c_p;
+  for (int r = 0; r < L.kh; ++r) {
+    const int hi = ho * L.stride + r - L.pad;
+    if (hi < 0 || hi >= L.h) continue;
+    for (int s = 0; s < L.kw; ++s) {
+      const int wi = wo * L.stride + s - L.pad;
+      if (wi < 0 || wi >= L.w) continue;
+      const int8_t* xp = x + (((long long)n * L.h + hi) * L.w + wi) * L.c_in;
+      const int8_t* wp = w + (((long long)co * L.kh + r) * L.kw + s) * L.c_r;
+      for (int ci = 0; ci < lo; ++ci) acc += (int)xp[ci] * (int)wp[ci];
+      for (int ci = hi2; ci < L.c_in; ++ci) acc += (int)xp[ci] * (int)wp[ci - L.c_p];
+    }
+  }
+  return acc;
+}
+
 constexpr int kThreads = 256;
 
 template <typename TIn, typename TOut>
@@ -102,14 +147,16 @@ direct_gated_conv_kernel(LayerDims L, const TIn* __restrict__ x, const TIn* __re
     const int n = (int)(m / ((long long)L.wo * L.ho));
     bool fire = false;
     if (valid) {
-      const float p = conv_point<TIn>(L, x, w_base, n, ho, wo, co, 0, L.c_p);
+      const int grp = L.grouping ? co / (L.c_out / L.groups) : 0;   // input group of the base path
+      const float p = conv_point<TIn>(L, x, w_base, n, ho, wo, co, grp * L.c_p, L.c_p);
       if (base_only) {
         p_out[m * L.c_out + co] = p;
       } else {
         fire = (p >= s_t[co]);   // NaN compares false
         float v;
         if (fire) {
-          const float r = conv_point<TIn>(L, x, w_cond, n, ho, wo, co, L.c_p, L.c_r);
+          const float r = L.grouping ? conv_point_others<TIn>(L, x, w_cond, n, ho, wo, co, grp)
+                                     : conv_point<TIn>(L, x, w_cond, n, ho, wo, co, L.c_p, L.c_r);
           v = __fadd_rn(__fmul_rn(s_a2[co], __fadd_rn(p, r)), s_b2[co]);
         } else {
           v = __fadd_rn(__fmul_rn(s_a1[co], p), s_b1[co]);
@@ -161,13 +208,15 @@ direct_gated_conv_i8_kernel(LayerDims L, const int8_t* __restrict__ x,
     const int n = (int)(m / ((long long)L.wo * L.ho));
     bool fire = false;
     if (valid) {
-      const int p = conv_point_i8(L, x, w_base, n, ho, wo, co, 0, L.c_p);
+      const int grp = L.grouping ? co / (L.c_out / L.groups) : 0;
+      const int p = conv_point_i8(L, x, w_base, n, ho, wo, co, grp * L.c_p, L.c_p);
       if (base_only) {
         p_out[m * L.c_out + co] = p;
       } else {
         fire = (p >= bn.q_gate_thr[co]);
         long long acc = p;
-        if (fire) acc += conv_point_i8(L, x, w_cond, n, ho, wo, co, L.c_p, L.c_r);
+        if (fire) acc += L.grouping ? conv_point_others_i8(L, x, w_cond, n, ho, wo, co, grp)
+                                    : conv_point_i8(L, x, w_cond, n, ho, wo, co, L.c_p, L.c_r);
         const bool full = fire;
         const long long mul = full ? bn.q_mul_full[co] : bn.q_mul_base[co];
         const long long off = full ? bn.q_off_full[co] : bn.q_off_base[co];

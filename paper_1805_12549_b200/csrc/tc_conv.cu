@@ -809,7 +809,7 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
   const int eb = in_dtype == CG_BF16 ? 2 : 1;
   const int ck = 128 / eb;          // channels per 128-byte patch row
   const int kst = ck / 4;           // channels per MMA K step (32 bytes)
-  if (L.has_residual) return false;
+  if (L.has_residual || L.grouping) return false;
   if (L.kh != L.kw || L.kh != 2 * L.pad + 1) return false;
   const bool s2 = L.stride == 2;
   if (L.stride != 1 && !s2) return false;

@@ -29,6 +29,7 @@ class Case:
     delta: np.ndarray | None = None
     residual: np.ndarray | None = None
     shift: int = 0
+    grouped: bool = False
 
 
 def _quantile_delta(p_hat: np.ndarray, density: float) -> float:
@@ -41,7 +42,8 @@ def _quantile_delta(p_hat: np.ndarray, density: float) -> float:
 
 
 def make_float_case(name, s: O.Shape, dtype="bf16", density=0.3, delta=None, rho=0.0,
-                    calib_images=4, separate=True, residual=False, smooth=True) -> Case:
+                    calib_images=4, separate=True, residual=False, smooth=True,
+                    grouped=False) -> Case:
     """Seeded layer.  Gate statistics are the per-channel mean/variance of the oracle's partial
     sums over the first `calib_images` images; Delta is one scalar per layer, the quantile of the
     normalised partial sums that gives `density` (unless `delta` is given)."""
@@ -62,7 +64,8 @@ def make_float_case(name, s: O.Shape, dtype="bf16", density=0.3, delta=None, rho
     if delta is None:
         nc = max(1, min(calib_images, s.n))
         sc = O.Shape(**{**s.__dict__, "n": nc})
-        probe = O.gated_conv(sc, x[:nc], wb, wc, bn, np.full(s.c_out, INF, np.float32))
+        probe = O.gated_conv(sc, x[:nc], wb, wc, bn, np.full(s.c_out, INF, np.float32),
+                             grouped=grouped)
         p = probe.p.reshape(-1, s.c_out).astype(np.float64)
         bn["gate_mean"] = p.mean(axis=0).astype(np.float32)
         bn["gate_var"] = np.maximum(p.var(axis=0), 1e-6).astype(np.float32)
@@ -70,7 +73,7 @@ def make_float_case(name, s: O.Shape, dtype="bf16", density=0.3, delta=None, rho
         delta = np.full(s.c_out, _quantile_delta(p_hat, density), np.float32)
     else:
         delta = np.broadcast_to(np.asarray(delta, np.float32), (s.c_out,)).copy()
-    return Case(name, s, dtype, x, wb, wc, bn, delta, res)
+    return Case(name, s, dtype, x, wb, wc, bn, delta, res, 0, grouped)
 
 
 def make_int8_case(name, s: O.Shape, density=0.3, shift=24, calib_images=4) -> Case:
@@ -103,7 +106,7 @@ def run_oracle(c: Case, **kw) -> O.Result:
     if c.dtype == "i8":
         return O.gated_conv_i8(c.s, c.shift, c.x, c.wb, c.wc, c.bn)
     return O.gated_conv(c.s, c.x, c.wb, c.wc, c.bn, c.delta, c.residual,
-                        out_bf16=(c.dtype == "bf16"), **kw)
+                        out_bf16=(c.dtype == "bf16"), grouped=c.grouped, **kw)
 
 
 # ----------------------------------------------------------------------------- GPU side
@@ -131,7 +134,7 @@ class GpuCase:
         self.conv = B.GatedConv(s.n, s.h, s.w, s.c_in, s.c_out, k=s.kh, stride=s.stride, pad=s.pad,
                                 groups=s.groups, dtype=dt, bn_eps=s.bn_eps, relu=bool(s.relu),
                                 has_residual=c.residual is not None, requant_shift=c.shift,
-                                algo=algo, cond_mode=cond_mode)
+                                algo=algo, cond_mode=cond_mode, grouping=c.grouped)
         self.x = _to_dev(c.x, c.dtype)
         self.wb = _to_dev(c.wb, c.dtype)
         self.wc = _to_dev(c.wc, c.dtype)

@@ -54,6 +54,23 @@ def test_delta_limits(dv):
     g.close()
 
 
+@pytest.mark.parametrize("s", [O.Shape(2, 7, 7, 12, 8, groups=4),
+                               O.Shape(1, 9, 8, 64, 64, groups=4),
+                               O.Shape(2, 8, 8, 32, 48, stride=2, groups=2)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_channel_grouping(s, dtype):
+    """Section 3.3: output group i takes input group i as x_p and the other groups as x_r."""
+    c = K.make_float_case("grp", s, dtype, density=0.4, grouped=True)
+    ref = K.run_oracle(c)
+    g = K.GpuCase(c)                       # AUTO must fall back to the direct kernels
+    assert not g.conv.uses_tensor_cores
+    y, mask, st = g.run()
+    K.compare(c, ref, y, mask, st, exact=True)
+    plain = K.run_oracle(K.make_float_case("grp", s, dtype, delta=c.delta))
+    assert (plain.mask != ref.mask).any()  # grouping really changes the layer
+    g.close()
+
+
 def test_int8_bit_exact():
     s = O.Shape(2, 9, 9, 32, 48, groups=4)
     c = K.make_int8_case("i8", s, density=0.3)

@@ -36,7 +36,7 @@ def test_status_strings():
 def _desc(**kw):
     base = dict(n=2, h=8, w=8, c_in=16, c_out=16, kh=3, kw=3, stride=1, pad=1, groups=4,
                 in_dtype=B.CG_F32, out_dtype=B.CG_F32, bn_eps=1e-5, relu=1, has_residual=0,
-                requant_shift=0, algo=0, cond_mode=0)
+                requant_shift=0, algo=0, cond_mode=0, grouping=0)
     base.update(kw)
     return B.CgConvDesc(**base)
 
@@ -46,7 +46,10 @@ def _desc(**kw):
                                 dict(out_dtype=B.CG_BF16), dict(h=1, w=1, pad=0),
                                 dict(in_dtype=B.CG_I8, out_dtype=B.CG_I8, requant_shift=0),
                                 dict(in_dtype=B.CG_I8, out_dtype=B.CG_I8, requant_shift=32),
-                                dict(bn_eps=-1.0), dict(algo=9), dict(cond_mode=-1)])
+                                dict(bn_eps=-1.0), dict(algo=9), dict(cond_mode=-1),
+                                dict(grouping=2), dict(grouping=1, c_out=18),
+                                dict(grouping=1, in_dtype=B.CG_I8, out_dtype=B.CG_I8,
+                                     requant_shift=8)])
 def test_create_rejects_bad_descriptions(kw):
     h = C.c_void_p()
     d = _desc(**kw)
