@@ -131,7 +131,10 @@ size_t cg_conv_workspace_bytes(cg_conv_t h) {
   return h->use_tc ? cg::tc_workspace_bytes(h->L, h->plan) : 0;
 }
 
-int cg_conv_launches_per_forward(cg_conv_t h) { return h ? 1 : 0; }
+int cg_conv_launches_per_forward(cg_conv_t h) {
+  if (!h) return 0;
+  return (h->use_tc && h->plan.cond_mode == CG_COND_COMPACT) ? 2 : 1;
+}
 
 int cg_conv_uses_tensor_cores(cg_conv_t h) { return h ? h->use_tc : 0; }
 

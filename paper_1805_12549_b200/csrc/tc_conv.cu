@@ -54,6 +54,12 @@ struct TcParams {
   const float* delta;
   uint32_t* mask;
   unsigned long long* counters;
+  // CG_COND_COMPACT: per column tile, the pixel rows in which a gate fired, with their partial
+  // sums and mask words, for the second (gathered) kernel
+  uint32_t* ws_counts;     // [tiles_n] rows listed so far
+  uint32_t* ws_list;       // [tiles_n][M] pixel-row indices
+  uint32_t* ws_rows;       // [tiles_n][M] records of NT partial sums (fp32) + NT/32 mask words,
+                           // NT + 4 words apart
 };
 
 // One weight tile: 64 K-elements of NT output channels.
@@ -96,7 +102,8 @@ struct Shared {
   uint64_t cond_done[4], r_free[4];                 // per R accumulator slot
   uint32_t tmem_base;
   uint32_t abort_flag;
-  uint32_t warp_blk[4][8];   // per job slot, per epilogue warp: column blocks with a firing gate
+  uint32_t warp_blk[4][8];
+  int row_idx[128];          // compact mode: list slot of each pixel row of the job being combined   // per job slot, per epilogue warp: column blocks with a firing gate
 };
 
 struct Ctx {
@@ -363,7 +370,8 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   const int jobs = group < P.tiles_m ? (P.tiles_m - group + groups - 1) / groups : 0;
   const int taps = L.kh * L.kw;
   const bool dense = (P.cond_mode == CG_COND_DENSE);
-  const bool has_cond = P.cond_tiles > 0;
+  const bool compact = (P.cond_mode == CG_COND_COMPACT);   // R is computed by a second kernel
+  const bool has_cond = P.cond_tiles > 0 && !compact;
   const int cond_first_chunk = L.c_p >= P.ck ? P.base_chunks : 0;
   constexpr int kBlocks = NT / 64;
   constexpr uint32_t kAllBlocks = (1u << kBlocks) - 1u;
@@ -637,13 +645,42 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         ptx::tma_store_wait_read();   // the previous store has finished reading the staging tile
         st_blocks_run += __popc(blocks);
       }
+      if (compact && half == 0) {
+        // rows with a firing gate get a slot in this column tile's list (order is arbitrary)
+        uint32_t any = 0;
+#pragma unroll
+        for (int cb = 0; cb < kWords; ++cb) any |= s_mask[(slot * 128 + row) * kWords + cb];
+        const uint32_t act = __ballot_sync(0xffffffffu, any != 0);
+        uint32_t base = 0;
+        if (lane == 0 && act) base = atomicAdd(&prm.ws_counts[tile_n], (uint32_t)__popc(act));
+        base = __shfl_sync(0xffffffffu, base, 0);
+        sh->row_idx[row] = any ? (int)(base + __popc(act & ((1u << lane) - 1u))) : -1;
+      }
       ptx::named_bar_sync(1, kEpiThreads);
+      int list_idx = -1;
+      long long m_row = 0;
+      if (compact) {
+        list_idx = sh->row_idx[row];
+        if (list_idx >= 0) {
+          int n0, h0;
+          job_origin(j, n0, h0);
+          m_row = ((long long)(n0 + n_loc) * L.ho + (h0 + h_loc)) * L.wo + w_out;
+          if (half == 0) prm.ws_list[(long long)tile_n * L.m + list_idx] = (uint32_t)m_row;
+        }
+      }
 #pragma unroll
       for (int cc = 0; cc < kWords / 2; ++cc) {
         const int cb = cc * 2 + half;
         const uint32_t word = s_mask[(slot * 128 + row) * kWords + cb];
         uint32_t p[32], rr[32];
         ptx::tmem_ld32(t_lane + (uint32_t)(slot * NT + cb * 32), p);
+        if (compact && list_idx >= 0) {
+          uint32_t* rec = prm.ws_rows + ((long long)tile_n * L.m + list_idx) * (NT + 4);
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            *(uint4*)(rec + cb * 32 + q * 4) = make_uint4(p[q * 4], p[q * 4 + 1], p[q * 4 + 2], p[q * 4 + 3]);
+          rec[NT + cb] = word;
+        }
         const bool have_r = ((blocks >> (cb >> 1)) & 1u) && __ballot_sync(0xffffffffu, word != 0) != 0;
         if (have_r) {
           ptx::tmem_ld32(t_lane + (uint32_t)((kNP + rslot) * NT + cb * 32), rr);
@@ -757,6 +794,257 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
 }
 
 // ------------------------------------------------------------------------------------------
+// Second kernel of CG_COND_COMPACT: the conditional path on compacted rows.
+//
+// The first kernel left, per column tile, the list of pixel rows in which a gate fired, their
+// partial sums P and their mask words.  Here every 128 listed rows form one dense sub-GEMM:
+// the A operand is GATHERED -- thread j copies, for each filter tap and 64-channel chunk, the
+// 128 bytes of its row's input pixel (or zeros in the padding) into a swizzled tile with
+// cp.async -- the weights come by TMA, the MMAs accumulate R in TMEM, and the epilogue
+// overwrites y where d = 1 with f(BN2(P + R)) (Eq. 1, second case).  Work is proportional to
+// the number of rows with a firing gate, not to the number of pixels.
+constexpr int kCpThreads = 320;   // warp 0: weight TMA, warp 1: MMA, warps 2-5: gather, 6-9: epilogue
+constexpr int kCpStages = 4;
+
+struct CpShared {
+  uint64_t full[kCpStages], empty[kCpStages];   // full: 128 gather arrivals + 1 TMA arrival
+  uint64_t acc_done, acc_free;
+  uint32_t tmem_base;
+  uint32_t abort_flag;
+};
+
+struct CpParams {
+  LayerDims L;
+  TcPlan P;
+  cg_bn_params bn;
+  const float* delta;
+  const __nv_bfloat16* x;
+  __nv_bfloat16* y;
+  const uint32_t* ws_counts;
+  const uint32_t* ws_list;
+  const uint32_t* ws_rows;
+  unsigned long long* counters;
+};
+
+__device__ __forceinline__ bool cp_wait(CpShared* sh, unsigned long long* counters, uint64_t* bar,
+                                        uint32_t parity, int site) {
+  if (ptx::mbar_try_wait(bar, parity, 0u)) return true;
+  const long long t0 = clock64();
+  for (int i = 0; i < kSpinLimit; ++i) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if ((i & 15) == 15) {
+      if (*(volatile uint32_t*)&sh->abort_flag) return false;
+      if (clock64() - t0 > kWaitCycles) break;
+    }
+  }
+  if (atomicCAS(&counters[CNT_STATUS], 0ull, (unsigned long long)CG_ERR_DEVICE_TIMEOUT) == 0ull)
+    atomicExch(&counters[CNT_SITE], (unsigned long long)site);
+  atomicExch(&sh->abort_flag, 1u);
+  return false;
+}
+
+template <int NT>
+__global__ void __launch_bounds__(kCpThreads, 1)
+tc_compact_cond_kernel(const __grid_constant__ CUtensorMap map_wc, const __grid_constant__ CpParams prm) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const LayerDims& L = prm.L;
+  const TcPlan& P = prm.P;
+  constexpr int kWords = NT / 32;
+  constexpr int kRec = NT + 4;
+  constexpr uint32_t kStageBytes = 128 * 128 + NT * 128;
+  uint8_t* s_stage = smem;                                        // [kCpStages][A 16 KB | B NT*128]
+  float* s_a2 = (float*)(smem + kCpStages * kStageBytes);
+  float* s_b2 = s_a2 + P.tiles_n * NT;
+  CpShared* sh = (CpShared*)(s_b2 + P.tiles_n * NT);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int taps = L.kh * L.kw;
+  const int kp16 = L.c_p >= P.ck ? 4 : L.c_p / (P.ck / 4);        // first conditional K step of chunk 0
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kCpStages; ++i) { ptx::mbar_init(&sh->full[i], 129); ptx::mbar_init(&sh->empty[i], 1); }
+    ptx::mbar_init(&sh->acc_done, 1);
+    ptx::mbar_init(&sh->acc_free, 128);
+    sh->abort_flag = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tensormap(&map_wc);
+  }
+  if (warp == 1) ptx::tmem_alloc(&sh->tmem_base, NT);
+  for (int c = threadIdx.x; c < P.tiles_n * NT; c += kCpThreads) {
+    const ChannelConsts k = fold_channel(prm.bn, prm.delta, L.eps, c);
+    s_a2[c] = k.a2; s_b2[c] = k.b2;
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem = sh->tmem_base;
+
+  // work items: (column tile, group of 128 listed rows), strided over the grid
+  auto item_of = [&](int it, int& tn, int& g) -> bool {
+    for (tn = 0; tn < P.tiles_n; ++tn) {
+      const int groups = (int)((prm.ws_counts[tn] + 127u) / 128u);
+      if (it < groups) { g = it; return true; }
+      it -= groups;
+    }
+    return false;
+  };
+
+  if (warp == 0) {
+    // ============================================================ weight (B) producer
+    if (lane == 0) {
+      int st = 0; uint32_t par = 1; bool ok = true;
+      int tn, g;
+      for (int it = blockIdx.x; ok && item_of(it, tn, g); it += gridDim.x) {
+        for (int bt = 0; bt < P.cond_tiles && ok; ++bt) {
+          ok = cp_wait(sh, prm.counters, &sh->empty[st], par, 21);
+          if (!ok) break;
+          ptx::mbar_expect_tx(&sh->full[st], NT * 128);
+          ptx::tma_load_2d(s_stage + (size_t)st * kStageBytes + 128 * 128, &map_wc, &sh->full[st],
+                           cond_tile(L, P.ck, bt).x, tn * NT);
+          if (++st == kCpStages) { st = 0; par ^= 1; }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ============================================================ MMA issuer (convergent warp)
+    const uint32_t issue = lane == 0 ? 1u : 0u;
+    const uint32_t desc_hi = (uint32_t)(ptx::smem_desc(0, 1024, 2) >> 32);
+    int st = 0; uint32_t par = 0; bool ok = true;
+    int tn, g, n_item = 0;
+    for (int it = blockIdx.x; ok && item_of(it, tn, g); it += gridDim.x, ++n_item) {
+      ok = cp_wait(sh, prm.counters, &sh->acc_free, (n_item & 1) ^ 1, 22);
+      if (!ok) break;
+      ptx::tc_fence_after();
+      uint32_t acc = 0;
+      for (int bt = 0; bt < P.cond_tiles && ok; ++bt) {
+        ok = cp_wait(sh, prm.counters, &sh->full[st], par, 23);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        const uint32_t a_lo = ((ptx::smem_u32(s_stage + (size_t)st * kStageBytes)) >> 4) | 0x10000u;
+        const uint32_t b_lo = a_lo + (128 * 128 >> 4);
+        const int ks0 = (L.c_p < P.ck && bt < taps) ? kp16 : 0;     // chunk 0 also holds base channels
+        for (int ks = ks0; ks < 4; ++ks) {
+          ptx::umma_bf16_if(issue, tmem, ((uint64_t)desc_hi << 32) | (a_lo + ks * 2),
+                            ((uint64_t)desc_hi << 32) | (b_lo + (ks - ks0) * 2), ptx::idesc_bf16(kBM, NT), acc);
+          acc = 1u;
+        }
+        ptx::umma_commit_if(issue, &sh->empty[st]);
+        if (++st == kCpStages) { st = 0; par ^= 1; }
+      }
+      if (ok) ptx::umma_commit_if(issue, &sh->acc_done);
+    }
+    __syncwarp();
+  } else if (warp < 6) {
+    // ============================================================ gather (A) producers: thread = row
+    const int j = threadIdx.x - 64;
+    int st = 0; uint32_t par = 1; bool ok = true;
+    int tn, g;
+    for (int it = blockIdx.x; ok && item_of(it, tn, g); it += gridDim.x) {
+      const uint32_t cnt = prm.ws_counts[tn];
+      const uint32_t ridx = (uint32_t)g * 128u + (uint32_t)j;
+      const bool rvalid = ridx < cnt;
+      int n = 0, ho = 0, wo = 0;
+      if (rvalid) {
+        const uint32_t m = prm.ws_list[(long long)tn * L.m + ridx];
+        wo = (int)(m % (uint32_t)L.wo);
+        ho = (int)((m / (uint32_t)L.wo) % (uint32_t)L.ho);
+        n = (int)(m / ((uint32_t)L.wo * (uint32_t)L.ho));
+      }
+      int pending = 0;       // stages whose copies are issued but not yet published
+      int pub = st;          // next stage to publish
+      for (int bt = 0; bt < P.cond_tiles && ok; ++bt) {
+        const WTile w = cond_tile(L, P.ck, bt);
+        int t;
+        if (L.c_p >= P.ck) t = bt % taps; else t = bt < taps ? bt : (bt - taps) % taps;
+        const int hi = ho * L.stride + t / L.kw - L.pad, wi = wo * L.stride + t % L.kw - L.pad;
+        const bool pv = rvalid && hi >= 0 && hi < L.h && wi >= 0 && wi < L.w;
+        const __nv_bfloat16* src = prm.x + ((((long long)n * L.h + (pv ? hi : 0)) * L.w + (pv ? wi : 0)) * L.c_in + w.chunk * 64);
+        ok = cp_wait(sh, prm.counters, &sh->empty[st], par, 24);
+        if (!ok) break;
+        uint8_t* dst = s_stage + (size_t)st * kStageBytes + (size_t)j * 128;
+#pragma unroll
+        for (int c16 = 0; c16 < 8; ++c16)
+          ptx::cp_async_16(dst + ((c16 ^ (j & 7)) << 4), src + c16 * 8, pv);
+        ptx::cp_async_commit();
+        if (++st == kCpStages) { st = 0; par ^= 1; }
+        if (++pending == 3) {     // keep two stages of copies in flight, publish the oldest
+          ptx::cp_async_wait<2>();
+          ptx::fence_proxy_async();
+          ptx::mbar_arrive(&sh->full[pub]);
+          if (++pub == kCpStages) pub = 0;
+          --pending;
+        }
+      }
+      ptx::cp_async_wait<0>();
+      ptx::fence_proxy_async();
+      while (pending > 0) {
+        ptx::mbar_arrive(&sh->full[pub]);
+        if (++pub == kCpStages) pub = 0;
+        --pending;
+      }
+    }
+  } else {
+    // ============================================================ epilogue: thread = listed row
+    const int quad = warp & 3;
+    const int j = quad * 32 + lane;
+    const uint32_t t_lane = tmem + ((uint32_t)(quad * 32) << 16);
+    bool ok = true;
+    int tn, g, n_item = 0;
+    unsigned long long items_done = 0;
+    for (int it = blockIdx.x; ok && item_of(it, tn, g); it += gridDim.x, ++n_item) {
+      ok = cp_wait(sh, prm.counters, &sh->acc_done, n_item & 1, 25);
+      if (!ok) break;
+      ptx::tc_fence_after();
+      const uint32_t cnt = prm.ws_counts[tn];
+      const uint32_t ridx = (uint32_t)g * 128u + (uint32_t)j;
+      const bool rvalid = ridx < cnt;
+      const uint32_t* rec = prm.ws_rows + ((long long)tn * L.m + (rvalid ? ridx : 0)) * kRec;
+      const long long m = rvalid ? (long long)prm.ws_list[(long long)tn * L.m + ridx] : 0;
+      __nv_bfloat16* yrow = prm.y + m * L.c_out + tn * NT;
+#pragma unroll
+      for (int cb = 0; cb < kWords; ++cb) {
+        uint32_t r[32];
+        ptx::tmem_ld32(t_lane + (uint32_t)(cb * 32), r);
+        if (!rvalid) continue;
+        const uint32_t word = rec[NT + cb];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const uint32_t bits = (word >> (q * 8)) & 0xffu;
+          if (bits == 0) continue;
+          uint4* slot = (uint4*)(yrow + cb * 32 + q * 8);
+          uint4 cur = *slot;
+          uint32_t* cw = (uint32_t*)&cur;
+          const uint4 p0 = *(const uint4*)(rec + cb * 32 + q * 8), p1 = *(const uint4*)(rec + cb * 32 + q * 8 + 4);
+          const uint32_t pp[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int jx = q * 8 + e * 2;
+            const int c = tn * NT + cb * 32 + jx;
+            float v0 = __fadd_rn(__fmul_rn(s_a2[c], __fadd_rn(__uint_as_float(pp[e * 2]), __uint_as_float(r[jx]))), s_b2[c]);
+            float v1 = __fadd_rn(__fmul_rn(s_a2[c + 1], __fadd_rn(__uint_as_float(pp[e * 2 + 1]), __uint_as_float(r[jx + 1]))), s_b2[c + 1]);
+            if (L.relu) { v0 = v0 > 0.f ? v0 : 0.f; v1 = v1 > 0.f ? v1 : 0.f; }
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
+            const uint32_t nv = *(const uint32_t*)&h2;
+            const uint32_t sel = (((bits >> (e * 2)) & 1u) ? 0x0000ffffu : 0u) | (((bits >> (e * 2 + 1)) & 1u) ? 0xffff0000u : 0u);
+            cw[e] = (cw[e] & ~sel) | (nv & sel);
+          }
+          *slot = cur;
+        }
+      }
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(&sh->acc_free);
+      ++items_done;
+    }
+    if (threadIdx.x == 192 && ok && items_done)
+      atomicAdd(&prm.counters[CNT_EXEC_MACS], items_done * (unsigned long long)kBM * NT * taps * L.c_r);
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) ptx::tmem_dealloc(tmem, NT);
+}
+
+// ------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -864,7 +1152,8 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
   }
   P.stage_rows = (int)align_up((size_t)max(kBM, P.wp * P.out_box_h * P.ni), 8);
   P.cond_mode = cond_mode == CG_COND_AUTO ? CG_COND_SKIP_TILES : cond_mode;
-  if (P.cond_mode == CG_COND_COMPACT) P.cond_mode = CG_COND_SKIP_TILES;
+  // row compaction: bf16 layers with a conditional path; otherwise block skipping
+  if (P.cond_mode == CG_COND_COMPACT && (eb != 2 || L.c_r == 0)) P.cond_mode = CG_COND_SKIP_TILES;
   if (P.base_tiles + P.cond_tiles > kMaxWTiles) return false;
   // shared-memory layout: [weights: resident tiles or ring][patch ring][y staging][consts]
   // [mask stash][tile coordinates][barriers]; widest column tile first, resident weights if
@@ -921,13 +1210,19 @@ bool tc_device_ok(int device) {
   return prop.major == 10 && encode_tiled_fn() != nullptr;
 }
 
-size_t tc_workspace_bytes(const LayerDims&, const TcPlan&) { return 0; }
+// CG_COND_COMPACT workspace: [row counts, 256 B][row lists: tiles_n x M x u32][row records:
+// tiles_n x M x (NT + 4) words]
+size_t tc_workspace_bytes(const LayerDims& L, const TcPlan& P) {
+  if (!P.valid || P.cond_mode != CG_COND_COMPACT) return 0;
+  const size_t rows = (size_t)P.tiles_n * (size_t)L.m;
+  return 256 + align_up(rows * 4, 256) + rows * (size_t)(P.nt + 4) * 4;
+}
 
 int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, const void* x,
               const void* w_base, const void* w_cond, const cg_bn_params& bn, const float* delta,
               const void* residual, void* y, uint32_t* mask, void* workspace,
               unsigned long long* counters, cudaStream_t stream) {
-  (void)in_dtype; (void)residual; (void)workspace;
+  (void)in_dtype; (void)residual;
   if (!P.valid) return (int)cudaErrorInvalidValue;
   const void* wc_key = w_cond ? w_cond : w_base;
   TcMapSet* ms = nullptr;
@@ -986,6 +1281,18 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
   }
   TcParams prm;
   prm.L = L; prm.P = P; prm.bn = bn; prm.delta = delta; prm.mask = mask; prm.counters = counters;
+  prm.ws_counts = nullptr; prm.ws_list = nullptr; prm.ws_rows = nullptr;
+  const bool compact = P.cond_mode == CG_COND_COMPACT;
+  if (compact) {
+    if (!workspace) return (int)cudaErrorInvalidValue;
+    const size_t rows = (size_t)P.tiles_n * (size_t)L.m;
+    char* ws = static_cast<char*>(workspace);
+    prm.ws_counts = reinterpret_cast<uint32_t*>(ws);
+    prm.ws_list = reinterpret_cast<uint32_t*>(ws + 256);
+    prm.ws_rows = reinterpret_cast<uint32_t*>(ws + 256 + align_up(rows * 4, 256));
+    const cudaError_t e = cudaMemsetAsync(prm.ws_counts, 0, 256, stream);
+    if (e != cudaSuccess) return (int)e;
+  }
   // persistent grid: one CTA per SM, a multiple of the number of column tiles
   const int sms = sm_count();
   int grid = sms - sms % P.tiles_n;
@@ -1006,6 +1313,27 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
   }
   kernels[which]<<<grid, kThreads, P.smem_bytes, stream>>>(ms->x[0], ms->x[1], ms->x[2], ms->x[3], ms->wb,
                                                            ms->wc, ms->y, prm);
+  if (compact) {
+    // second kernel: gathered conditional path over the listed rows
+    CpParams cp;
+    cp.L = L; cp.P = P; cp.bn = bn; cp.delta = delta;
+    cp.x = static_cast<const __nv_bfloat16*>(x); cp.y = static_cast<__nv_bfloat16*>(y);
+    cp.ws_counts = prm.ws_counts; cp.ws_list = prm.ws_list; cp.ws_rows = prm.ws_rows;
+    cp.counters = counters;
+    const size_t smem2 = (size_t)kCpStages * (128 * 128 + (size_t)P.nt * 128) + (size_t)2 * L.c_out * 4 +
+                         sizeof(CpShared) + 2048;
+    long long items = (long long)P.tiles_n * ((L.m + 127) / 128);
+    const int grid2 = (int)(items < sms ? items : sms);
+    typedef void (*Kernel2)(CUtensorMap, CpParams);
+    const Kernel2 k2 = P.nt == 128 ? (Kernel2)tc_compact_cond_kernel<128> : (Kernel2)tc_compact_cond_kernel<64>;
+    static bool attr2[2] = {false, false};
+    if (!attr2[P.nt == 128]) {
+      const cudaError_t e = cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+      if (e != cudaSuccess) return (int)e;
+      attr2[P.nt == 128] = true;
+    }
+    k2<<<grid2, kCpThreads, smem2, stream>>>(ms->wc, cp);
+  }
   return (int)cudaGetLastError();
 }
 

@@ -164,3 +164,44 @@ def test_int8_tensor_path_is_bit_exact(s, why, density):
     if density == 0.3:
         assert 0.2 < st.density < 0.4 and len(np.unique(y)) > 16
     g.close()
+
+
+COMPACT = 3
+COMPACT_CASES = [
+    (O.Shape(2, 56, 56, 64, 64, groups=4), 0.3, 0.0, "c_p = 16, every row active"),
+    (O.Shape(3, 28, 28, 128, 128, groups=4), 0.05, 0.9, "c_p = 32, clustered gates"),
+    (O.Shape(3, 14, 14, 256, 256, groups=4), 0.1, 0.8, "c_p = 64, two column tiles"),
+    (O.Shape(5, 7, 7, 512, 512, groups=4), 0.02, 0.95, "c_p = 128, few rows"),
+    (O.Shape(3, 28, 28, 128, 256, stride=2, groups=4), 0.1, 0.5, "stride 2"),
+    (O.Shape(20, 28, 28, 128, 128, groups=8), 0.3, 0.0, "G = 8, many row groups per CTA"),
+]
+
+
+@pytest.mark.parametrize("s,density,rho,why", COMPACT_CASES, ids=[c[3] for c in COMPACT_CASES])
+def test_row_compaction_mode(s, density, rho, why):
+    """CG_COND_COMPACT: the first kernel lists the pixel rows with a firing gate, the second
+    gathers those rows into dense sub-GEMMs for the conditional path (Eq. 1, second case)."""
+    c = K.make_float_case("tccomp", s, "bf16", density=density, rho=rho)
+    ref = K.run_oracle(c)
+    g = K.GpuCase(c, algo=TENSOR, cond_mode=COMPACT)
+    assert g.conv.workspace is not None
+    y, mask, st = g.run()
+    K.compare(c, ref, y, mask, st)
+    assert st.rows_total % s.m == 0          # pixel rows x column tiles
+    print(f"{why}: density {st.density:.3f}, rows active {st.rows_active}/{st.rows_total}, "
+          f"executed/gated MACs {st.executed_macs / st.gated_macs:.2f}")
+    # a second call reuses the workspace
+    y2, mask2, _ = g.run()
+    np.testing.assert_array_equal(y.view(np.uint32), y2.view(np.uint32))
+    g.close()
+
+
+def test_compaction_with_no_active_rows_and_all_rows():
+    s = O.Shape(2, 28, 28, 128, 128, groups=4)
+    for dv in (K.INF, -K.INF):
+        c = K.make_float_case("tccomp2", s, "bf16", delta=dv)
+        ref = K.run_oracle(c)
+        g = K.GpuCase(c, algo=TENSOR, cond_mode=COMPACT)
+        y, mask, st = g.run()
+        K.compare(c, ref, y, mask, st)
+        g.close()
