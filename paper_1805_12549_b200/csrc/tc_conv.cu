@@ -38,14 +38,14 @@ namespace cg {
 
 namespace {
 
-constexpr int kThreads = 352;       // 3 single-role warps + 8 epilogue warps
-constexpr int kEpiThread0 = 96;     // first epilogue thread
+constexpr int kThreads = 384;       // 4 single-thread warps + 8 epilogue warps
+constexpr int kEpiWarp0 = 4;        // warps 0-3: patch producer, MMA issuer, weight producer, second MMA issuer
+constexpr int kEpiThread0 = kEpiWarp0 * 32;
 constexpr int kEpiThreads = 256;
 constexpr int kBM = 128;            // MMA M: patch rows per job
 constexpr int kSpinLimit = 1 << 21; // try_wait polls before a wait gives up ...
 constexpr long long kWaitCycles = 2000000000ll;   // ... or about one second of SM clocks, whichever is first
 constexpr int kMaxWTiles = 192;     // weight tiles per job, both phases
-constexpr bool kUnroll3x3 = true;   // fully unrolled 3x3 issue code (measured faster than rolled tap loops)
 
 struct TcParams {
   LayerDims L;
@@ -102,8 +102,8 @@ struct Shared {
   uint64_t cond_done[4], r_free[4];                 // per R accumulator slot
   uint32_t tmem_base;
   uint32_t abort_flag;
-  uint32_t warp_blk[4][8];
-  int row_idx[128];          // compact mode: list slot of each pixel row of the job being combined   // per job slot, per epilogue warp: column blocks with a firing gate
+  uint32_t warp_blk[4][8];   // per job slot, per epilogue warp: column blocks with a firing gate
+  int row_idx[128];          // compact mode: list slot of each pixel row of the job being combined
 };
 
 struct Ctx {
@@ -140,190 +140,195 @@ __device__ __forceinline__ uint32_t slot_blocks(const Shared* sh, int slot) {
   return w[0] | w[1] | w[2] | w[3] | w[4] | w[5] | w[6] | w[7];
 }
 
-// MMA issue for one CTA.  The whole warp runs this code convergently and one lane's tcgen05
-// instructions are predicated on, so addresses stay warp-uniform and there is no branch between
-// two MMAs: for 3x3 kernels the taps and K steps are fully unrolled with immediate descriptor
-// offsets.  (The issuing lane cannot hide latency: every branch, instruction-cache miss or
-// dependent scalar instruction between two MMAs is tensor idle time.)  Weight tiles are
-// visited in the order base_tile()/cond_tile() enumerate them, which is the order the weight
+// MMA issue for one CTA, run by ONE thread.  A lone thread executes about one dependent
+// instruction every 4-5 cycles and a branch costs several times that, while the tensor pipe
+// needs only 49/64/128 cycles per MMA at N = 64/128/256: with more than about eight
+// instructions per MMA the issue loop, not the tensor pipe, sets the pace (measured: 280 cycles
+// per filter tap with a rolled tap loop and a handful of run-time conditions in it).  So for 3x3
+// kernels the taps of a filter row and their K steps are unrolled, every descriptor is a
+// register plus an immediate, and what distinguishes the layer variants (stride-2 planes, a
+// single column block) is folded into those registers instead of into branches.  Weight tiles
+// are visited in the order base_tile()/cond_tile() enumerate them, which is the order the weight
 // producer loads them.
 template <int NT, bool I8>
 struct MmaIssuer {
+  static constexpr uint32_t kWTile = (uint32_t)(NT * 128) >> 4;   // weight tile, 16-byte units
   Shared* sh;
   Ctx cx;
-  uint32_t issue;                        // 1 on the issuing lane
   uint32_t desc_hi;                      // upper descriptor word (see ptx::smem_desc)
   uint32_t a_base_lo, b_base_lo;         // lower descriptor words of the ring bases
-  uint32_t patch_lo, wtile_lo, row_lo;   // buffer sizes / one patch pixel row, in 16-byte units
-  int resident, na, nb, kp16 /* base K steps per tap */, chunks, base_chunks, base_tiles, kh, kw, planes;
+  uint32_t patch_lo;                     // patch buffer size in 16-byte units
+  // A-descriptor offset of tap (r, sx) from the first patch buffer of a chunk = f[r] + c[sx]
+  // (3x3) or r * row_lo + sx * 8 (other sizes, stride 1).  Stride 1: the patch read from pixel
+  // r*(W+pad)+sx on.  Stride 2 (3x3, pad 1): output (h,w) reads input (2h+r-1, 2w+sx-1), i.e.
+  // plane (r odd ? 0 : 1, sx odd ? 0 : 1) at (h + (r ? 0 : -1), w + (sx ? 0 : -1)); every plane
+  // patch starts one row and one column early, so the offset within the plane's buffer is
+  // (r ? 1 : 0) rows + (sx ? 1 : 0) pixels, and plane p is the p-th buffer of the chunk.
+  uint32_t f0, f1, f2, c0, c1, c2, row_lo;
+  int resident, a0, na /* ring slots [a0, na) */, nb, kp16 /* base K steps per tap */, chunks, base_chunks, base_tiles, kh, kw, planes;
   int as, bs;                            // ring slots and the parities of their "full" barriers
   uint32_t apar, bpar;
   // per phase
-  uint32_t d_tmem, a_lo[4], b_lo, acc, blk_off_d, blk_off_b;   // a_lo: one per plane
-  int a_held[4], b_held;
+  uint32_t d_tmem, idesc, a_grp, b_lo, acc, blk_off_b;
+  int a_first, b_held;
   bool ok;
 
+  // slot0, slots: the part of the patch ring this issuer consumes
   __device__ __forceinline__ void init(Shared* sh_, const Ctx& cx_, const uint8_t* s_a,
                                        const uint8_t* s_b, const TcPlan& P, const LayerDims& L,
-                                       int lane) {
+                                       int slot0, int slots) {
     sh = sh_; cx = cx_;
-    issue = lane == 0 ? 1u : 0u;
     // descriptor words: upper = 8-row groups 1024 bytes apart, 128-byte swizzle, version 1;
     // lower = (address >> 4) | (1 << 16)
     desc_hi = (uint32_t)(ptx::smem_desc(0, 1024, 2) >> 32);
     a_base_lo = (ptx::smem_u32(s_a) >> 4) | 0x10000u;
     b_base_lo = (ptx::smem_u32(s_b) >> 4) | 0x10000u;
     patch_lo = (uint32_t)P.patch_bytes >> 4;
-    wtile_lo = (uint32_t)(NT * 128) >> 4;
     row_lo = (uint32_t)P.wp * 8u;
-    resident = P.resident; na = P.na; nb = P.nb; kp16 = L.c_p / (P.ck / 4); chunks = P.chunks;
+    if (P.planes == 4) {
+      f0 = 2u * patch_lo; f1 = row_lo; f2 = 2u * patch_lo + row_lo;
+      c0 = patch_lo; c1 = 8u; c2 = patch_lo + 8u;
+    } else {
+      f0 = 0u; f1 = row_lo; f2 = 2u * row_lo;
+      c0 = 0u; c1 = 8u; c2 = 16u;
+    }
+    resident = P.resident; a0 = slot0; na = slot0 + slots; nb = P.nb; kp16 = L.c_p / (P.ck / 4); chunks = P.chunks;
     base_chunks = P.base_chunks; base_tiles = P.base_tiles; kh = L.kh; kw = L.kw; planes = P.planes;
-    as = 0; bs = 0; apar = 0; bpar = 0;
-    b_held = 0; ok = true;
-    for (int i = 0; i < 4; ++i) { a_held[i] = 0; a_lo[i] = 0; }
+    as = slot0; bs = 0; apar = 0; bpar = 0;
+    a_first = slot0; b_held = 0; ok = true;
   }
-  template <bool ALL>
   __device__ __forceinline__ void mma(uint32_t al, uint32_t bl) {
     const uint64_t da = ((uint64_t)desc_hi << 32) | al;
-    const uint64_t db = ((uint64_t)desc_hi << 32) | (ALL ? bl : bl + blk_off_b);
-    const uint32_t d = ALL ? d_tmem : d_tmem + blk_off_d;   // !ALL: exactly one of two 64-column blocks
-    if (I8) ptx::umma_s8_if(issue, d, da, db, ptx::idesc_s8(kBM, ALL ? NT : 64), acc);
-    else ptx::umma_bf16_if(issue, d, da, db, ptx::idesc_bf16(kBM, ALL ? NT : 64), acc);
+    const uint64_t db = ((uint64_t)desc_hi << 32) | bl;
+    if (I8) ptx::umma_s8(d_tmem, da, db, idesc, acc);
+    else ptx::umma_bf16(d_tmem, da, db, idesc, acc);
     acc = 1u;
   }
-  // the patch buffer(s) of the next chunk in the ring: one, or the four planes of a stride-2 layer
-  template <bool S2>
+  // the patch buffer(s) of the next chunk in the ring: one, or the four planes of a stride-2
+  // layer, which sit in consecutive slots (the ring length is then a multiple of four)
   __device__ __forceinline__ void acquire_a() {
-#pragma unroll
-    for (int pl = 0; pl < (S2 ? 4 : 1); ++pl) {
+    a_first = as;
+    a_grp = a_base_lo + (uint32_t)as * patch_lo;
+    for (int pl = 0; pl < planes; ++pl) {
       ok = ok && wait_bar(cx, &sh->a_full[as], apar, 7);
-      a_held[pl] = as;
-      a_lo[pl] = a_base_lo + (uint32_t)as * patch_lo;
-      if (++as == na) { as = 0; apar ^= 1; }
+      if (++as == na) { as = a0; apar ^= 1; }
     }
   }
-  template <bool S2>
   __device__ __forceinline__ void release_a() {
-#pragma unroll
-    for (int pl = 0; pl < (S2 ? 4 : 1); ++pl) ptx::umma_commit_if(issue, &sh->a_empty[a_held[pl]]);
+    for (int pl = 0; pl < planes; ++pl) ptx::umma_commit(&sh->a_empty[a_first + pl]);
   }
-  // descriptor word of the A operand of tap (r, sx).  Stride 1: the patch read from pixel
-  // r*(W+pad)+sx on.  Stride 2 (3x3, pad 1): output (h,w) reads input (2h+r-1, 2w+sx-1), i.e.
-  // plane (r odd ? 0 : 1, sx odd ? 0 : 1) at (h + (r ? 0 : -1), w + (sx ? 0 : -1)); every plane
-  // patch starts one row and one column early, so the offset is (r ? 1 : 0) rows + (sx ? 1 : 0).
-  template <bool S2>
-  __device__ __forceinline__ uint32_t tap_lo(int r, int sx) const {
-    if (S2) {
-      const uint32_t base = (r == 1) ? ((sx == 1) ? a_lo[0] : a_lo[1]) : ((sx == 1) ? a_lo[2] : a_lo[3]);
-      return base + (r ? row_lo : 0u) + (sx ? 8u : 0u);
-    }
-    return a_lo[0] + (uint32_t)r * row_lo + (uint32_t)sx * 8u;
-  }
+  // Next weight tile.  Resident weights: tiles follow one another from b_lo on (b_lo includes
+  // the column-block offset).  Ring: wait for the slot.
   template <bool RES>
-  __device__ __forceinline__ void acquire_b() {
-    if (!RES) {
-      ok = ok && wait_bar(cx, &sh->b_full[bs], bpar, 8);
-      b_held = bs;
-      b_lo = b_base_lo + (uint32_t)bs * wtile_lo;
-      if (++bs == nb) { bs = 0; bpar ^= 1; }
-    }
+  __device__ __forceinline__ uint32_t acquire_b() {
+    if (RES) { const uint32_t b = b_lo; b_lo += kWTile; return b; }
+    ok = ok && wait_bar(cx, &sh->b_full[bs], bpar, 8);
+    b_held = bs;
+    const uint32_t b = b_base_lo + (uint32_t)bs * kWTile + blk_off_b;
+    if (++bs == nb) { bs = 0; bpar ^= 1; }
+    return b;
   }
   template <bool RES>
   __device__ __forceinline__ void release_b() {
-    if (RES) b_lo += wtile_lo;
-    else ptx::umma_commit_if(issue, &sh->b_empty[b_held]);
+    if (!RES) ptx::umma_commit(&sh->b_empty[b_held]);
   }
   // K steps [KS0, KS1) of every tap of the next chunk in the ring, one weight tile per tap
-  template <bool RES, bool ALL, bool S2, int KS0, int KS1>
+  template <bool RES, int KS0, int KS1>
   __device__ __forceinline__ void chunk_taps() {
-    acquire_a<S2>();
-    if (kUnroll3x3 && kh == 3 && kw == 3) {
-#pragma unroll
+    acquire_a();
+    if (!ok) return;
+    if (kh == 3 && kw == 3) {
+      uint32_t a_row = a_grp + f0;
+#pragma unroll 1
       for (int r = 0; r < 3; ++r) {
 #pragma unroll
         for (int sx = 0; sx < 3; ++sx) {
-          acquire_b<RES>();
-          if (!ok) return;
-          const uint32_t a_t = tap_lo<S2>(r, sx);
+          const uint32_t b_t = acquire_b<RES>();
+          if (!RES && !ok) return;
+          const uint32_t a_t = a_row + (sx == 0 ? c0 : sx == 1 ? c1 : c2);
 #pragma unroll
-          for (int ks = KS0; ks < KS1; ++ks) mma<ALL>(a_t + ks * 2, b_lo + (ks - KS0) * 2);
+          for (int ks = KS0; ks < KS1; ++ks) mma(a_t + ks * 2, b_t + (ks - KS0) * 2);
           release_b<RES>();
         }
+        a_row += r == 0 ? f1 - f0 : f2 - f1;
       }
     } else {
+      uint32_t a_row = a_grp;
       for (int r = 0; r < kh; ++r) {
         for (int sx = 0; sx < kw; ++sx) {
-          acquire_b<RES>();
-          if (!ok) return;
-          const uint32_t a_t = tap_lo<S2>(r, sx);
+          const uint32_t b_t = acquire_b<RES>();
+          if (!RES && !ok) return;
+          const uint32_t a_t = a_row + (uint32_t)sx * 8u;
 #pragma unroll
-          for (int ks = KS0; ks < KS1; ++ks) mma<ALL>(a_t + ks * 2, b_lo + (ks - KS0) * 2);
+          for (int ks = KS0; ks < KS1; ++ks) mma(a_t + ks * 2, b_t + (ks - KS0) * 2);
           release_b<RES>();
         }
+        a_row += row_lo;
       }
     }
-    release_a<S2>();
+    release_a();
   }
   // base path when c_p < 64: the first KP K steps of chunk 0; a weight tile covers 4/KP taps
-  template <bool RES, bool ALL, bool S2, int KP>
+  template <bool RES, int KP>
   __device__ __forceinline__ void base_small() {
     constexpr int TPT = 4 / KP;
-    acquire_a<S2>();
-    if (kUnroll3x3 && kh == 3 && kw == 3) {
+    acquire_a();
+    if (!ok) return;
+    if (kh == 3 && kw == 3) {
+      uint32_t b_t = 0;
 #pragma unroll
       for (int t = 0; t < 9; ++t) {
-        if (t % TPT == 0) acquire_b<RES>();
-        if (!ok) return;
-        const uint32_t a_t = tap_lo<S2>(t / 3, t % 3);
+        if (t % TPT == 0) b_t = acquire_b<RES>();
+        if (!RES && !ok) return;
+        const uint32_t a_t = a_grp + (t / 3 == 0 ? f0 : t / 3 == 1 ? f1 : f2) + (t % 3 == 0 ? c0 : t % 3 == 1 ? c1 : c2);
 #pragma unroll
-        for (int ks = 0; ks < KP; ++ks) mma<ALL>(a_t + ks * 2, b_lo + ((t % TPT) * KP + ks) * 2);
+        for (int ks = 0; ks < KP; ++ks) mma(a_t + ks * 2, b_t + ((t % TPT) * KP + ks) * 2);
         if (t % TPT == TPT - 1 || t == 8) release_b<RES>();
       }
     } else {
+      uint32_t a_row = a_grp, b_t = 0;
       int in_tile = 0;
       for (int r = 0; r < kh; ++r) {
         for (int sx = 0; sx < kw; ++sx) {
-          if (in_tile == 0) acquire_b<RES>();
-          if (!ok) return;
-          const uint32_t a_t = tap_lo<S2>(r, sx);
+          if (in_tile == 0) b_t = acquire_b<RES>();
+          if (!RES && !ok) return;
+          const uint32_t a_t = a_row + (uint32_t)sx * 8u;
 #pragma unroll
-          for (int ks = 0; ks < KP; ++ks) mma<ALL>(a_t + ks * 2, b_lo + (uint32_t)(in_tile * KP + ks) * 2u);
+          for (int ks = 0; ks < KP; ++ks) mma(a_t + ks * 2, b_t + (uint32_t)(in_tile * KP + ks) * 2u);
           if (++in_tile == TPT) { release_b<RES>(); in_tile = 0; }
         }
+        a_row += row_lo;
       }
       if (in_tile != 0) release_b<RES>();
     }
-    release_a<S2>();
+    release_a();
   }
-  template <bool RES, bool ALL, bool S2>
+  template <bool RES>
   __device__ __forceinline__ void phase(bool cond) {
     if (kp16 >= 4) {
       const int q0 = cond ? base_chunks : 0, q1 = cond ? chunks : base_chunks;
-      for (int q = q0; q < q1 && ok; ++q) chunk_taps<RES, ALL, S2, 0, 4>();
+      for (int q = q0; q < q1 && ok; ++q) chunk_taps<RES, 0, 4>();
     } else if (!cond) {
-      if (kp16 == 1) base_small<RES, ALL, S2, 1>(); else base_small<RES, ALL, S2, 2>();
+      if (kp16 == 1) base_small<RES, 1>(); else base_small<RES, 2>();
     } else {
       // conditional channels of chunk 0 (K steps kp16..3), then the remaining chunks
-      if (kp16 == 1) chunk_taps<RES, ALL, S2, 1, 4>(); else chunk_taps<RES, ALL, S2, 2, 4>();
-      for (int q = 1; q < chunks && ok; ++q) chunk_taps<RES, ALL, S2, 0, 4>();
+      if (kp16 == 1) chunk_taps<RES, 1, 4>(); else chunk_taps<RES, 2, 4>();
+      for (int q = 1; q < chunks && ok; ++q) chunk_taps<RES, 0, 4>();
     }
-  }
-  template <bool RES, bool ALL>
-  __device__ __forceinline__ void phase_s(bool cond) {
-    if (planes == 4) phase<RES, ALL, true>(cond); else phase<RES, ALL, false>(cond);
   }
   // base or conditional MMAs of one job into the accumulator at d; `blocks` = column blocks to
   // compute (all of them for the base path)
   __device__ __forceinline__ bool run_phase(uint32_t d, bool cond, uint32_t blocks) {
     constexpr uint32_t kAll = (1u << (NT / 64)) - 1u;
-    d_tmem = d;
+    // a single block of two: accumulator columns and weight rows 64..127
+    d_tmem = d + (blocks == 2u ? 64u : 0u);
+    blk_off_b = blocks == 2u ? (64u * 128u / 16u) : 0u;
+    const int n = blocks == kAll ? NT : 64;
+    idesc = I8 ? ptx::idesc_s8(kBM, n) : ptx::idesc_bf16(kBM, n);
     acc = 0u;   // the first K step overwrites the accumulator
     ok = true;
-    b_lo = b_base_lo + (cond ? (uint32_t)base_tiles * wtile_lo : 0u);   // resident tiles
-    blk_off_d = blocks == 2u ? 64u : 0u;
-    blk_off_b = blocks == 2u ? (64u * 128u / 16u) : 0u;
-    if (blocks == kAll) { if (resident) phase_s<true, true>(cond); else phase_s<false, true>(cond); }
-    else { if (resident) phase_s<true, false>(cond); else phase_s<false, false>(cond); }
+    b_lo = b_base_lo + blk_off_b + (cond ? (uint32_t)base_tiles * kWTile : 0u);   // resident tiles
+    if (resident) phase<true>(cond); else phase<false>(cond);
     return ok;
   }
 };
@@ -406,7 +411,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     ptx::prefetch_tensormap(&map_wc); ptx::prefetch_tensormap(&map_y);
   }
   if (warp == 1) ptx::tmem_alloc(&sh->tmem_base, 512);
-  if (warp >= 3) {
+  if (warp >= kEpiWarp0) {
     const int et = threadIdx.x - kEpiThread0;
     // zero the rows behind the TMA box of every patch buffer: they stand for the right padding
     // of the last patch row and are never written again
@@ -439,28 +444,35 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   if (warp == 0) {
     // ============================================================ patch (A) producer
     // Loads chunks in the order the MMA issuer consumes them: base(0) | base(1) cond(0) | ...
+    // With two issuers the ring is split: slots [0, split_a) for the base path, the rest for the
+    // conditional path, each part with its own cursor.
     if (lane == 0 && jobs > 0) {
-      int as = 0;              // ring slot and the parity of its "empty" barrier
-      uint32_t apar = 1;
+      // ring slot and the parity of its "empty" barrier, per ring part
+      int as0 = 0, as1 = P.split_a;
+      uint32_t apar0 = 1, apar1 = 1;
+      const int hi0 = P.split_a ? P.split_a : P.na;
       bool ok = true;
-      auto load_chunks = [&](int j, int q0, int q1) {
+      auto load_chunks = [&](int j, int q0, int q1, int part) {
         int n0, h0;
         job_origin(j, n0, h0);
         const int lead = P.planes == 4 ? 1 : L.pad;   // zero rows/columns in front of the patch
         for (int q = q0; q < q1 && ok; ++q) {
           for (int pl = 0; pl < P.planes && ok; ++pl) {
-            ok = wait_bar(cx, &sh->a_empty[as], apar, 1);
+            const int slot = part ? as1 : as0;
+            ok = wait_bar(cx, &sh->a_empty[slot], part ? apar1 : apar0, 1);
             if (!ok) return;
             const CUtensorMap* mx = pl == 0 ? &map_x : (pl == 1 ? &map_x1 : (pl == 2 ? &map_x2 : &map_x3));
-            ptx::mbar_expect_tx(&sh->a_full[as], patch_tx);
-            ptx::tma_load_4d(s_a + (size_t)as * P.patch_bytes, mx, &sh->a_full[as], q * P.ck, -lead,
+            ptx::mbar_expect_tx(&sh->a_full[slot], patch_tx);
+            ptx::tma_load_4d(s_a + (size_t)slot * P.patch_bytes, mx, &sh->a_full[slot], q * P.ck, -lead,
                              h0 - lead, n0);
-            if (++as == P.na) { as = 0; apar ^= 1; }
+            if (part) { if (++as1 == P.na) { as1 = P.split_a; apar1 ^= 1; } }
+            else if (++as0 == hi0) { as0 = 0; apar0 ^= 1; }
           }
         }
       };
+      const int cond_part = P.split_a ? 1 : 0;
       for (int j = 0; j <= jobs && ok; ++j) {
-        if (j < jobs) load_chunks(j, 0, P.base_chunks);
+        if (j < jobs) load_chunks(j, 0, P.base_chunks, 0);
         if (j >= 1 && has_cond && ok) {
           const int jj = j - 1;
           uint32_t blocks = kAllBlocks;
@@ -469,11 +481,10 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
             if (!ok) break;
             blocks = slot_blocks(sh, jj % kNP);
           }
-          if (blocks) load_chunks(jj, cond_first_chunk, P.chunks);
+          if (blocks) load_chunks(jj, cond_first_chunk, P.chunks, cond_part);
         }
       }
     }
-    __syncwarp();
   } else if (warp == 2) {
     // ============================================================ weight (B) producer
     if (lane == 0 && jobs > 0) {
@@ -512,25 +523,30 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         }
       }
     }
-    __syncwarp();
-  } else if (warp == 1) {
-    // ============================================================ MMA issuer
-    if (jobs > 0) {
+  } else if (warp == 1 || warp == 3) {
+    // ============================================================ MMA issuer(s)
+    // One thread issues the base path of job j+1 and then the conditional path of job j; when
+    // the patch ring is split (resident weights), warp 3 takes the conditional path instead, so
+    // the per-job bookkeeping of the two paths runs in parallel.
+    const bool do_base = warp == 1;
+    const bool do_cond = P.split_a ? warp == 3 : warp == 1;
+    if (lane == 0 && jobs > 0 && (do_base || do_cond)) {
       MmaIssuer<NT, I8> mi;
-      mi.init(sh, cx, s_a, s_b, P, L, lane);
+      if (P.split_a) mi.init(sh, cx, s_a, s_b, P, L, do_base ? 0 : P.split_a, do_base ? P.split_a : P.na - P.split_a);
+      else mi.init(sh, cx, s_a, s_b, P, L, 0, P.na);
       bool ok = true;
       if (P.resident) ok = wait_bar(cx, &sh->w_ready, 0, 6);
       for (int j = 0; j <= jobs && ok; ++j) {
-        if (j < jobs) {
+        if (do_base && j < jobs) {
           const int ps = j % kNP;
           ok = wait_bar(cx, &sh->p_free[ps], ((j / kNP) & 1) ^ 1, 9);
           if (!ok) break;
           ptx::tc_fence_after();
           ok = mi.run_phase(tmem + (uint32_t)(ps * NT), false, kAllBlocks);
           if (!ok) break;
-          ptx::umma_commit_if(mi.issue, &sh->base_done[ps]);
+          ptx::umma_commit(&sh->base_done[ps]);
         }
-        if (j >= 1) {
+        if (do_cond && j >= 1) {
           const int jj = j - 1;
           const int rs = jj % kNR;
           if (has_cond) {
@@ -553,16 +569,15 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
             ok = wait_bar(cx, &sh->r_free[rs], ((jj / kNR) & 1) ^ 1, 15);
             if (!ok) break;
           }
-          ptx::umma_commit_if(mi.issue, &sh->cond_done[rs]);
+          ptx::umma_commit(&sh->cond_done[rs]);
         }
       }
     }
-    __syncwarp();
   } else {
     // ============================================================ epilogue (8 warps)
     // Warps w and w+4 share a TMEM lane quadrant and split its 32-column blocks between them.
     const int quad = warp & 3;
-    const int half = (warp - 3) >> 2;
+    const int half = (warp - kEpiWarp0) >> 2;
     const int row = quad * 32 + lane;                      // TMEM lane = patch row i
     const int et = threadIdx.x - kEpiThread0;
     const int n_loc = P.images_mode ? row / P.ip : 0;
@@ -616,7 +631,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) my_blocks |= __shfl_xor_sync(0xffffffffu, my_blocks, o);
-      if (lane == 0) sh->warp_blk[slot][warp - 3] = my_blocks;
+      if (lane == 0) sh->warp_blk[slot][warp - kEpiWarp0] = my_blocks;
       if (half == 0) {
         const uint32_t row_valid = __ballot_sync(0xffffffffu, valid);
         if (lane == 0) st_rows_valid += __popc(row_valid);
@@ -788,9 +803,13 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     }
   }
   // ---------------------------------------------------------------- teardown
+  // (the idle lanes of the single-thread warps wait here, at the hardware barrier)
   ptx::tc_fence_before();
   __syncthreads();
-  if (warp == 1) ptx::tmem_dealloc(tmem, 512);
+  if (warp == 1) {
+    __syncwarp();
+    ptx::tmem_dealloc(tmem, 512);
+  }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1185,8 +1204,11 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
         found = true;
         break;
       }
-      if (!found || na < P.planes) continue;
+      if (!found) continue;
     }
+    // the four planes of a stride-2 chunk occupy four consecutive ring slots
+    if (P.planes == 4) na = na / 4 * 4;
+    if (na < P.planes) continue;
     size_t off = 0;
     P.off_b = (unsigned)off; off += resident ? w_all : nb * w_tile;
     P.off_a = (unsigned)off; off += (size_t)na * P.patch_bytes;
@@ -1196,6 +1218,10 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
     P.off_tables = (unsigned)off; off += align_up((size_t)kMaxWTiles * 4, 128);
     P.off_bar = (unsigned)off; off += align_up(sizeof(Shared), 128);
     P.nt = nt; P.na = na; P.nb = nb; P.resident = resident; P.tiles_n = L.c_out / nt;
+    // resident weights: the base and the conditional path get their own MMA issuer and their own
+    // half of the patch ring
+    P.split_a = (resident && P.cond_tiles > 0 && P.cond_mode != CG_COND_COMPACT && na >= 2 * P.planes &&
+                 (na / 2) % P.planes == 0) ? na / 2 : 0;
     P.smem_bytes = (unsigned)(off + 1024);
     P.valid = 1;
     *plan = P;

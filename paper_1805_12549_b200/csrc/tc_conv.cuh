@@ -24,6 +24,8 @@ struct TcPlan {
   int planes;           // patch buffers per chunk: 1 (stride 1) or 4 (stride 2: the input's
                         // even/odd row x even/odd column sub-images)
   int na;               // patch buffers in the ring
+  int split_a;          // > 0: slots [0, split_a) serve the base path and the rest the conditional
+                        // path, each with its own MMA-issuing thread; 0: one ring, one issuer
   int nb;               // weight-tile ring depth (0 when the weights are resident)
   int resident;         // 1: all weight tiles of a column tile stay in shared memory
   int box_h;            // patch box rows: r + 2*pad (rows mode) or h + pad (images mode)
