@@ -52,6 +52,7 @@ struct TcParams {
   TcPlan P;
   cg_bn_params bn;
   const float* delta;
+  const __nv_bfloat16* residual;   // optional, same layout as y (bf16 layers)
   uint32_t* mask;
   unsigned long long* counters;
   // CG_COND_COMPACT: per column tile, the pixel rows in which a gate fired, with their partial
@@ -672,6 +673,16 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         sh->row_idx[row] = any ? (int)(base + __popc(act & ((1u << lane) - 1u))) : -1;
       }
       ptx::named_bar_sync(1, kEpiThreads);
+      // residual rows (the shortcut of a residual block, added before the activation)
+      const __nv_bfloat16* res_row = nullptr;
+      if (!I8 && prm.residual) {
+        int n0, h0;
+        job_origin(j, n0, h0);
+        const int rows_here = P.images_mode ? L.ho : min(P.r, L.ho - h0);
+        const bool valid = (w_out < L.wo) && (h_loc < rows_here) && (n_loc < P.ni) && (n0 + n_loc < L.n);
+        if (valid)
+          res_row = prm.residual + (((long long)(n0 + n_loc) * L.ho + (h0 + h_loc)) * L.wo + w_out) * L.c_out + tile_n * NT;
+      }
       int list_idx = -1;
       long long m_row = 0;
       if (compact) {
@@ -736,6 +747,9 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   #pragma unroll
           for (int q = 0; q < 4; ++q) {
             uint32_t packed[4];
+            uint4 res4 = make_uint4(0u, 0u, 0u, 0u);
+            if (res_row) res4 = *(const uint4*)(res_row + cb * 32 + q * 8);
+            const uint32_t resw[4] = {res4.x, res4.y, res4.z, res4.w};
   #pragma unroll
             for (int e = 0; e < 4; ++e) {
               const int jx = q * 8 + e * 2;
@@ -750,6 +764,10 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
               const float s1 = f1 ? __fadd_rn(p1, __uint_as_float(rr[jx + 1])) : p1;
               float v0 = __fadd_rn(__fmul_rn(f0 ? a2.x : a1.x, s0), f0 ? b2.x : b1.x);
               float v1 = __fadd_rn(__fmul_rn(f1 ? a2.y : a1.y, s1), f1 ? b2.y : b1.y);
+              if (res_row) {
+                v0 = __fadd_rn(v0, __uint_as_float(resw[e] << 16));
+                v1 = __fadd_rn(v1, __uint_as_float(resw[e] & 0xffff0000u));
+              }
               if (L.relu) { v0 = v0 > 0.f ? v0 : 0.f; v1 = v1 > 0.f ? v1 : 0.f; }
               const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
               packed[e] = *(const uint32_t*)&h2;
@@ -1116,7 +1134,8 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
   const int eb = in_dtype == CG_BF16 ? 2 : 1;
   const int ck = 128 / eb;          // channels per 128-byte patch row
   const int kst = ck / 4;           // channels per MMA K step (32 bytes)
-  if (L.has_residual || L.grouping) return false;
+  if (L.grouping) return false;
+  if (L.has_residual && in_dtype != CG_BF16) return false;
   if (L.kh != L.kw || L.kh != 2 * L.pad + 1) return false;
   const bool s2 = L.stride == 2;
   if (L.stride != 1 && !s2) return false;
@@ -1171,13 +1190,16 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
   }
   P.stage_rows = (int)align_up((size_t)max(kBM, P.wp * P.out_box_h * P.ni), 8);
   P.cond_mode = cond_mode == CG_COND_AUTO ? CG_COND_SKIP_TILES : cond_mode;
-  // row compaction: bf16 layers with a conditional path; otherwise block skipping
-  if (P.cond_mode == CG_COND_COMPACT && (eb != 2 || L.c_r == 0)) P.cond_mode = CG_COND_SKIP_TILES;
+  // row compaction: bf16 layers with a conditional path and no residual input; otherwise block
+  // skipping
+  if (P.cond_mode == CG_COND_COMPACT && (eb != 2 || L.c_r == 0 || L.has_residual)) P.cond_mode = CG_COND_SKIP_TILES;
   if (P.base_tiles + P.cond_tiles > kMaxWTiles) return false;
   // shared-memory layout: [weights: resident tiles or ring][patch ring][y staging][consts]
-  // [mask stash][tile coordinates][barriers]; widest column tile first, resident weights if
-  // they fit next to at least two patch buffers
+  // [mask stash][tile coordinates][barriers].  First choice: a column tile whose weights stay
+  // resident next to at least two patch buffers (no weight traffic per job, which otherwise
+  // bounds the layer at the per-SM L2 ingest rate); else the widest tile with streamed weights.
   const size_t limit = 227 * 1024 - 1024;
+  for (int pass = 0; pass < 2; ++pass)
   for (int nt = 128; nt >= (eb == 1 ? 128 : 64); nt >>= 1) {
     if (L.c_out % nt != 0) continue;
     const size_t fixed = align_up((size_t)(nt * eb / 128) * P.stage_rows * 128, 1024) +
@@ -1192,6 +1214,8 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
       resident = 1;
       na = (int)((limit - fixed - w_all) / P.patch_bytes);
       if (na > na_max) na = na_max;
+    } else if (pass == 0) {
+      continue;
     } else {
       // streamed weights are latency-bound (bytes in flight per SM), so the weight ring gets
       // the shared memory that three patch buffers (stride 1) or one set of planes leave
@@ -1248,7 +1272,7 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
               const void* w_base, const void* w_cond, const cg_bn_params& bn, const float* delta,
               const void* residual, void* y, uint32_t* mask, void* workspace,
               unsigned long long* counters, cudaStream_t stream) {
-  (void)in_dtype; (void)residual;
+  (void)in_dtype;
   if (!P.valid) return (int)cudaErrorInvalidValue;
   const void* wc_key = w_cond ? w_cond : w_base;
   TcMapSet* ms = nullptr;
@@ -1306,7 +1330,7 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
     ms->key[0] = x; ms->key[1] = w_base; ms->key[2] = wc_key; ms->key[3] = y;
   }
   TcParams prm;
-  prm.L = L; prm.P = P; prm.bn = bn; prm.delta = delta; prm.mask = mask; prm.counters = counters;
+  prm.L = L; prm.P = P; prm.bn = bn; prm.delta = delta; prm.residual = (const __nv_bfloat16*)residual; prm.mask = mask; prm.counters = counters;
   prm.ws_counts = nullptr; prm.ws_list = nullptr; prm.ws_rows = nullptr;
   const bool compact = P.cond_mode == CG_COND_COMPACT;
   if (compact) {

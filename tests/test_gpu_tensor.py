@@ -205,3 +205,24 @@ def test_compaction_with_no_active_rows_and_all_rows():
         y, mask, st = g.run()
         K.compare(c, ref, y, mask, st)
         g.close()
+
+
+RESIDUAL_SHAPES = [
+    (O.Shape(3, 28, 28, 128, 128, groups=4), "streamed weights, NT = 128"),
+    (O.Shape(2, 56, 56, 64, 64, groups=4), "resident weights, two issuers"),
+    (O.Shape(7, 4, 4, 512, 512, groups=4), "images per tile, ragged batch"),
+    (O.Shape(3, 28, 28, 128, 256, stride=2, groups=4), "stride 2"),
+]
+
+
+@pytest.mark.parametrize("s,why", RESIDUAL_SHAPES, ids=[w for _, w in RESIDUAL_SHAPES])
+def test_residual_input_on_the_tensor_path(s, why):
+    """The shortcut of a residual block is added after the batch norm and before the ReLU
+    (second convolution of a block, Fig. 2 / Section 4)."""
+    c = K.make_float_case("tcres", s, "bf16", density=0.3, residual=True)
+    ref, st, exempt = _run(c)
+    assert abs(st.density - ref.density) < 2e-3
+    # the residual changes the output: without it the result must differ
+    c0 = K.make_float_case("tcres", s, "bf16", density=0.3, residual=False)
+    ref0 = K.run_oracle(c0)
+    assert np.abs(ref.y.astype(np.float64) - ref0.y.astype(np.float64)).max() > 0.1
