@@ -13,6 +13,12 @@
 //   * Eq. 2: the Heaviside step theta(v) = 1 when v >= 0 (a tie fires).
 //   * Eq. 3 (merged gate): d = theta(P - Delta*sqrt(Var) - E), with one
 //     threshold per output channel, P the partial sum W_p*x_p.
+//   * Eq. 4 (channel-wise gate, optional): per image, an output channel keeps
+//     its conditional path iff the number of its activations that fire is at
+//     least tau_c * w' * h'; otherwise all its activations take the first case
+//     of Eq. 1.
+//   * Section 3.3 (channel grouping, optional): output group i takes input
+//     group i as x_p and the other groups as x_r.
 //   * Section 4, first paragraph and its footnote: the two paths are
 //     normalised by two batch norms BN1 (base result) and BN2 (full result)
 //     that share gamma and beta; at inference each is a scale and a shift.
@@ -20,6 +26,9 @@
 //     eta*c_l*k^2*w'*h'*c_{l+1} multiplications; the conditional path costs the
 //     remaining (1-eta)*c_l*k^2 multiplications for every activation that fires.
 //
+// The layer runs in the three steps of the definition: partial sums and
+// activation-wise decisions for every output, then the channel-wise decision,
+// then the conditional path and the batch norm of the path taken.
 // Everything is a direct convolution written as nested loops over
 // (n, h', w', c_out, r, s, c_in) in NHWC order.  No blocking, no im2col,
 // no reordering.  Floating-point sums run in fp32 in the order (r, s, c_in)
@@ -29,8 +38,10 @@
 // Parity pins (tests/test_oracle_pins.py): all-open gate vs a library dense
 // convolution, all-shut gate vs a base-only convolution, the tie rule, the
 // merged vs unmerged gate, monotonicity in Delta, the Gaussian firing rate,
-// the multiplication-count closed form, a hand-computed 3x3 case, and an
-// exact integer re-computation of the quantised variant.
+// the multiplication-count closed form, a hand-computed 3x3 case, an
+// exact integer re-computation of the quantised variant, and for Eq. 4 a
+// hand-computed two-image case, its limits (tau_c = 0, tau_c > 1), a
+// restatement on the unpacked decisions and per-image independence.
 // Trained-model behaviour (accuracy, the tables' FLOP reductions, the
 // partial/final-sum correlations) is "parity unpinned": it needs data sets and
 // trained weights that are not available.
@@ -57,6 +68,7 @@ struct cgo_desc {
   int32_t acc_double;   // 1: accumulate P and R in fp64 instead of fp32
   int32_t gate_form;    // 0: merged gate of Eq. 3; 1: normalise P first, then compare with Delta
   int32_t grouped;      // 0: Fig. 5(a), base = channels [0,c_in/G); 1: Fig. 5(b), channel grouping
+  float channel_tau;    // tau_c of the channel-wise gate (Eq. 4); <= 0: no channel-wise gate
 };
 
 struct cgo_counts {
@@ -65,6 +77,8 @@ struct cgo_counts {
   int64_t base_macs;    // multiplications on the base path (padding taps counted)
   int64_t cond_macs;    // multiplications on the conditional path
   int64_t dense_macs;   // multiplications of the ungated layer
+  int64_t channels;          // n * c_out output channels (one per image)
+  int64_t channels_skipped;  // of those, channels whose conditional path Eq. 4 switched off
 };
 
 int cgo_out_dim(int in, int k, int stride, int pad) { return (in + 2 * pad - k) / stride + 1; }
@@ -200,20 +214,22 @@ int gated_conv_impl(const cgo_desc* d, const float* x, const float* w_base, cons
   const float* gm = gate_mean ? gate_mean : mean_base;
   const float* gv = gate_var ? gate_var : var_base;
 
-  int64_t active = 0, base_macs = 0, cond_macs = 0;
-#pragma omp parallel for collapse(2) schedule(dynamic, 1) reduction(+ : active, base_macs, cond_macs)
+  // Step 1 -- base path and activation-wise gate of every output (Section 3.1, Eq. 2, Eq. 3).
+  const int64_t outputs = (int64_t)d->n * ho_n * wo_n * d->c_out;
+  std::vector<Acc> p_all((size_t)outputs);
+  std::vector<uint8_t> fire_all((size_t)outputs);
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
   for (int n = 0; n < d->n; ++n) {
     for (int ho = 0; ho < ho_n; ++ho) {
       for (int wo = 0; wo < wo_n; ++wo) {
         const int64_t m = ((int64_t)n * ho_n + ho) * wo_n + wo;
-        if (mask) for (int q = 0; q < words; ++q) mask[m * words + q] = 0u;
         for (int co = 0; co < d->c_out; ++co) {
           // Base path: always computed (Section 3.1).
           const Acc p_acc = d->grouped
               ? conv_point_grouped<Acc>(d, x, w_base, n, ho, wo, co, co / og, true)
               : conv_point<Acc>(d, x, w_base, n, ho, wo, co, 0, cp);
           const float p = (float)p_acc;
-          base_macs += (int64_t)d->kh * d->kw * cp;
+          p_all[(size_t)(m * d->c_out + co)] = p_acc;
           if (p_out) p_out[m * d->c_out + co] = p;
           // Gate (Eq. 2, Eq. 3): a tie fires; a NaN partial sum does not.
           bool fire;
@@ -225,6 +241,46 @@ int gated_conv_impl(const cgo_desc* d, const float* x, const float* w_base, cons
             const float p_hat = centred / sg;
             fire = (p_hat >= delta[co]);
           }
+          fire_all[(size_t)(m * d->c_out + co)] = fire ? 1 : 0;
+        }
+      }
+    }
+  }
+
+  // Step 2 -- channel-wise gate (Eq. 4): output channel i of one image keeps its conditional
+  // path iff  sum_{j,k} s(x, Delta)  >=  tau_c * w' * h'  (theta(0) = 1, as for Eq. 2); the sum
+  // runs over the positions of that image's feature map.  Both sides are compared in fp32.
+  const bool channel_gate = d->channel_tau > 0.f;
+  std::vector<uint8_t> chan_on((size_t)d->n * d->c_out, 1);
+  int64_t channels_skipped = 0;
+  if (channel_gate) {
+    const float need = d->channel_tau * (float)(ho_n * wo_n);
+    for (int n = 0; n < d->n; ++n) {
+      for (int co = 0; co < d->c_out; ++co) {
+        int64_t cnt = 0;
+        for (int px = 0; px < ho_n * wo_n; ++px)
+          cnt += fire_all[(size_t)(((int64_t)n * ho_n * wo_n + px) * d->c_out + co)];
+        const bool on = ((float)cnt >= need);
+        chan_on[(size_t)n * d->c_out + co] = on ? 1 : 0;
+        if (!on) ++channels_skipped;
+      }
+    }
+  }
+
+  // Step 3 -- conditional path where both gates allow it, batch norm of the path taken,
+  // activation (Eq. 1, Section 4).
+  int64_t active = 0, base_macs = 0, cond_macs = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1) reduction(+ : active, base_macs, cond_macs)
+  for (int n = 0; n < d->n; ++n) {
+    for (int ho = 0; ho < ho_n; ++ho) {
+      for (int wo = 0; wo < wo_n; ++wo) {
+        const int64_t m = ((int64_t)n * ho_n + ho) * wo_n + wo;
+        if (mask) for (int q = 0; q < words; ++q) mask[m * words + q] = 0u;
+        for (int co = 0; co < d->c_out; ++co) {
+          const Acc p_acc = p_all[(size_t)(m * d->c_out + co)];
+          const float p = (float)p_acc;
+          base_macs += (int64_t)d->kh * d->kw * cp;
+          const bool fire = fire_all[(size_t)(m * d->c_out + co)] && chan_on[(size_t)n * d->c_out + co];
           float v;
           if (fire) {
             // Conditional path: only where the gate fires (Eq. 1, second case).
@@ -255,6 +311,8 @@ int gated_conv_impl(const cgo_desc* d, const float* x, const float* w_base, cons
     counts->base_macs = base_macs;
     counts->cond_macs = cond_macs;
     counts->dense_macs = counts->outputs * d->kh * d->kw * d->c_in;
+    counts->channels = (int64_t)d->n * d->c_out;
+    counts->channels_skipped = channels_skipped;
   }
   return 0;
 }
@@ -370,6 +428,8 @@ int cgo_gated_conv_i8(const cgo_desc* d, int32_t shift, const int8_t* x, const i
     counts->base_macs = base_macs;
     counts->cond_macs = cond_macs;
     counts->dense_macs = counts->outputs * d->kh * d->kw * d->c_in;
+    counts->channels = (int64_t)d->n * d->c_out;
+    counts->channels_skipped = 0;
   }
   return 0;
 }

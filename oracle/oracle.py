@@ -36,11 +36,13 @@ class _Desc(C.Structure):
     _fields_ = [(k, C.c_int32) for k in ("n", "h", "w", "c_in", "c_out", "kh", "kw", "stride", "pad",
                                          "groups")] + \
                [("bn_eps", C.c_float)] + \
-               [(k, C.c_int32) for k in ("relu", "out_bf16", "acc_double", "gate_form", "grouped")]
+               [(k, C.c_int32) for k in ("relu", "out_bf16", "acc_double", "gate_form", "grouped")] + \
+               [("channel_tau", C.c_float)]
 
 
 class _Counts(C.Structure):
-    _fields_ = [(k, C.c_int64) for k in ("outputs", "active", "base_macs", "cond_macs", "dense_macs")]
+    _fields_ = [(k, C.c_int64) for k in ("outputs", "active", "base_macs", "cond_macs", "dense_macs",
+                                         "channels", "channels_skipped")]
 
 
 _lib = None
@@ -107,6 +109,8 @@ class Result:
     base_macs: int
     cond_macs: int
     dense_macs: int
+    channels: int = 0            # n * c_out
+    channels_skipped: int = 0    # channels switched off by the channel-wise gate (Eq. 4)
 
     @property
     def density(self):
@@ -143,7 +147,7 @@ def round_bf16(a: np.ndarray) -> np.ndarray:
 def fold_params(s: Shape, bn: dict, delta) -> dict:
     """Per-channel t, a1, b1, a2, b2 exactly as the oracle derives them."""
     d = _Desc(s.n, s.h, s.w, s.c_in, s.c_out, s.kh, s.kw, s.stride, s.pad, s.groups, s.bn_eps,
-              s.relu, 0, 0, 0, 0)
+              s.relu, 0, 0, 0, 0, 0.0)
     arrs = {k: _f32(bn.get(k)) for k in ("gamma", "beta", "mean_base", "var_base", "mean_full",
                                         "var_full", "gate_mean", "gate_var")}
     delta = _f32(delta)
@@ -157,11 +161,13 @@ def fold_params(s: Shape, bn: dict, delta) -> dict:
 
 
 def gated_conv(s: Shape, x, w_base, w_cond, bn: dict, delta, residual=None, *, out_bf16=False,
-               acc_double=False, gate_form=0, grouped=False) -> Result:
+               acc_double=False, gate_form=0, grouped=False, channel_tau=0.0) -> Result:
     """Floating-point gated layer.  bn holds gamma, beta, mean_base, var_base, mean_full,
-    var_full and optionally gate_mean, gate_var (absent/None: BN1's statistics)."""
+    var_full and optionally gate_mean, gate_var (absent/None: BN1's statistics).
+    channel_tau > 0 adds the channel-wise gate of Eq. 4."""
     d = _Desc(s.n, s.h, s.w, s.c_in, s.c_out, s.kh, s.kw, s.stride, s.pad, s.groups, s.bn_eps,
-              s.relu, int(out_bf16), int(acc_double), int(gate_form), int(grouped))
+              s.relu, int(out_bf16), int(acc_double), int(gate_form), int(grouped),
+              float(channel_tau))
     x = _f32(x)
     w_base = _f32(w_base)
     w_cond = _f32(w_cond)
@@ -187,14 +193,15 @@ def gated_conv(s: Shape, x, w_base, w_cond, bn: dict, delta, residual=None, *, o
         _ptr(mask, C.c_uint32), _ptr(p, C.c_float), C.byref(cnt))
     if rc != 0:
         raise ValueError("oracle rejected the layer description")
-    return Result(y, mask, p, cnt.outputs, cnt.active, cnt.base_macs, cnt.cond_macs, cnt.dense_macs)
+    return Result(y, mask, p, cnt.outputs, cnt.active, cnt.base_macs, cnt.cond_macs, cnt.dense_macs,
+                  cnt.channels, cnt.channels_skipped)
 
 
 def gated_conv_i8(s: Shape, shift: int, x, w_base, w_cond, q: dict) -> Result:
     """Quantised gated layer.  q holds q_gate_thr, q_mul_base, q_mul_full (int32) and
     q_off_base, q_off_full (int64), one entry per output channel."""
     d = _Desc(s.n, s.h, s.w, s.c_in, s.c_out, s.kh, s.kw, s.stride, s.pad, s.groups, s.bn_eps,
-              s.relu, 0, 0, 0, 0)
+              s.relu, 0, 0, 0, 0, 0.0)
     x = np.ascontiguousarray(x, dtype=np.int8)
     w_base = np.ascontiguousarray(w_base, dtype=np.int8)
     w_cond = np.ascontiguousarray(w_cond, dtype=np.int8)

@@ -358,3 +358,93 @@ def test_int8_threshold_limits():
     assert O.gated_conv_i8(s, 20, x, wb, wc, q).active == s.m * s.c_out
     q["q_gate_thr"] = np.full(s.c_out, np.iinfo(np.int32).max, np.int32)
     assert O.gated_conv_i8(s, 20, x, wb, wc, q).active == 0
+
+
+# ----------------------------------------------------------------------------- channel-wise gate
+def _golden(name):
+    out = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", name)) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            k, *v = line.split()
+            out[k] = np.array([float(t) for t in v])
+    return out
+
+
+def test_channel_gate_hand_case():
+    """Eq. 4 on the worked example of tests/golden/channel_gate_case.txt (per-image counts,
+    ties keep the channel, a dropped channel takes Eq. 1's first case everywhere)."""
+    g = _golden("channel_gate_case.txt")
+    s = O.Shape(2, 2, 2, 2, 2, kh=1, kw=1, pad=0, groups=2, bn_eps=0.0)
+    x = np.stack([g["x_p"], g["x_r"]], axis=-1).reshape(2, 2, 2, 2).astype(np.float32)
+    wb = np.array([1.0, 2.0], np.float32).reshape(2, 1, 1, 1)
+    wc = np.array([1.0, -1.0], np.float32).reshape(2, 1, 1, 1)
+    one, zero = np.ones(2, np.float32), np.zeros(2, np.float32)
+    bn = dict(gamma=one, beta=zero, mean_base=zero, var_base=one, mean_full=zero, var_full=one,
+              gate_mean=zero, gate_var=one)
+    for tag in ("a", "b"):
+        res = O.gated_conv(s, x, wb, wc, bn, g["delta"].astype(np.float32),
+                           channel_tau=float(g["tau_" + tag][0]))
+        d = O.unpack_mask(res.mask, 2).reshape(-1).astype(int)
+        assert d.tolist() == g["d_" + tag].astype(int).tolist()
+        np.testing.assert_array_equal(res.y.reshape(-1), g["y_" + tag].astype(np.float32))
+        assert res.channels == 4 and res.channels_skipped == int(g["skipped_" + tag][0])
+        assert res.cond_macs == int(g["cond_macs_" + tag][0]) and res.active == res.cond_macs
+
+
+@pytest.mark.parametrize("s", SHAPES[:3])
+def test_channel_gate_limits(s):
+    """Eq. 4: tau_c = 0 keeps every channel (any count >= 0), so the layer is unchanged;
+    tau_c > 1 drops every channel (no count reaches more than w*h), so the layer is the base
+    path alone, as with Delta = +inf."""
+    x, wb, wc, bn = make_layer(("cg-lim", s.c_in, s.h), s)
+    delta = np.zeros(s.c_out, np.float32)
+    plain = O.gated_conv(s, x, wb, wc, bn, delta)
+    off = O.gated_conv(s, x, wb, wc, bn, delta, channel_tau=0.0)
+    np.testing.assert_array_equal(plain.y, off.y)
+    np.testing.assert_array_equal(plain.mask, off.mask)
+    assert off.channels_skipped == 0
+    shut = O.gated_conv(s, x, wb, wc, bn, delta, channel_tau=1.5)
+    base = O.gated_conv(s, x, wb, wc, bn, np.full(s.c_out, INF, np.float32))
+    np.testing.assert_array_equal(shut.y, base.y)
+    assert not shut.mask.any() and shut.active == 0
+    assert shut.channels_skipped == shut.channels == s.n * s.c_out
+
+
+@pytest.mark.parametrize("s", SHAPES[:3])
+@pytest.mark.parametrize("tau", [0.35, 0.45, 0.55])
+def test_channel_gate_restated_with_numpy(s, tau):
+    """Eq. 4 restated on the activation-wise decisions: per image and channel, count the firing
+    gates over the feature map, keep the channel iff count >= tau_c*w*h, and AND that with the
+    activation-wise mask; the conditional path runs exactly on the surviving activations."""
+    x, wb, wc, bn = make_layer(("cg-np", s.c_in, s.h), s)
+    delta = synth.rng("cg-np-delta", s.c_in).uniform(-0.3, 0.3, s.c_out).astype(np.float32)
+    plain = O.gated_conv(s, x, wb, wc, bn, delta)
+    res = O.gated_conv(s, x, wb, wc, bn, delta, channel_tau=tau)
+    d = O.unpack_mask(plain.mask, s.c_out).reshape(s.n, s.ho * s.wo, s.c_out)
+    cnt = d.sum(axis=1)                                   # [n, c_out]
+    keep = cnt.astype(np.float32) >= np.float32(tau) * np.float32(s.ho * s.wo)
+    d_eff = d & keep[:, None, :]
+    got = O.unpack_mask(res.mask, s.c_out).reshape(d.shape)
+    np.testing.assert_array_equal(got, d_eff)
+    assert res.channels_skipped == int((~keep).sum())
+    assert res.active == int(d_eff.sum()) and res.cond_macs == res.active * s.kh * s.kw * s.c_r
+    # kept channels are untouched, dropped ones equal the base-path-only layer
+    base = O.gated_conv(s, x, wb, wc, bn, np.full(s.c_out, INF, np.float32))
+    ky = np.broadcast_to(keep[:, None, None, :], res.y.shape)
+    np.testing.assert_array_equal(res.y[ky], plain.y[ky])
+    np.testing.assert_array_equal(res.y[~ky], base.y[~ky])
+    assert 0 < res.channels_skipped < res.channels
+
+
+def test_channel_gate_is_per_image():
+    """Eq. 4 sums over one feature map: an image's decision does not depend on its batch."""
+    s2 = O.Shape(2, 6, 6, 8, 8, groups=2)
+    x, wb, wc, bn = make_layer(("cg-img", 8), s2)
+    delta = np.full(8, 0.2, np.float32)
+    both = O.gated_conv(s2, x, wb, wc, bn, delta, channel_tau=0.45)
+    s1 = O.Shape(1, 6, 6, 8, 8, groups=2)
+    for i in range(2):
+        one = O.gated_conv(s1, x[i:i + 1], wb, wc, bn, delta, channel_tau=0.45)
+        np.testing.assert_array_equal(one.y[0], both.y[i])
