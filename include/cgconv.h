@@ -79,6 +79,15 @@ typedef struct {
                                    output group i = channels [i*c_out/G,(i+1)*c_out/G) takes input
                                    group i as x_p and the other groups, in ascending order, as
                                    x_r; needs c_out % G == 0.  Direct kernels only for now.    */
+  float channel_tau;            /* tau_c of the channel-wise gate (Eq. 4).  0: off.  > 0: per
+                                   image, an output channel whose gate fires at fewer than
+                                   tau_c * h' * w' positions loses its conditional path (all its
+                                   activations take Eq. 1's first case, its mask bits are 0);
+                                   a count equal to tau_c*h'*w' keeps the channel (theta(0) = 1);
+                                   the comparison is (float)count >= tau_c * (float)(h'*w').
+                                   Floating-point layers, direct kernels, three launches (partial
+                                   sums and counts, decisions, conditional path); needs the
+                                   workspace cg_conv_workspace_bytes reports.                  */
 } cg_conv_desc;
 
 /* Per-output-channel parameters: DEVICE pointers to c_out entries, caller-owned.
@@ -117,6 +126,9 @@ typedef struct {
   int64_t rows_active;   /* ... of which contained at least one firing gate                    */
   int32_t device_status; /* CG_OK, CG_ERR_DEVICE_TIMEOUT or CG_ERR_DEVICE_BOUNDS               */
   int32_t device_site;   /* which wait/check reported it (kernel-internal id), 0 if none       */
+  int64_t channels;         /* calls * n * c_out: output channels, one per image (Eq. 4)       */
+  int64_t channels_skipped; /* ... of which the channel-wise gate switched off (their
+                               conditional weights need not be fetched); 0 when channel_tau = 0 */
 } cg_stats;
 
 /* Section 3.1: fixes the layer and picks kernels.  Host work only, plus one small device

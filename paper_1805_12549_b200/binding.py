@@ -30,7 +30,8 @@ class CgConvDesc(C.Structure):
                                          "pad", "groups", "in_dtype", "out_dtype")] + \
                [("bn_eps", C.c_float)] + \
                [(k, C.c_int32) for k in ("relu", "has_residual", "requant_shift", "algo",
-                                         "cond_mode", "grouping")]
+                                         "cond_mode", "grouping")] + \
+               [("channel_tau", C.c_float)]
 
 
 class CgBnParams(C.Structure):
@@ -43,7 +44,8 @@ class CgStats(C.Structure):
     _fields_ = [(k, C.c_int64) for k in ("calls", "outputs", "active", "dense_macs", "gated_macs",
                                          "executed_macs", "tiles_total", "tiles_skipped",
                                          "rows_total", "rows_active")] + \
-               [("device_status", C.c_int32), ("device_site", C.c_int32)]
+               [("device_status", C.c_int32), ("device_site", C.c_int32)] + \
+               [("channels", C.c_int64), ("channels_skipped", C.c_int64)]
 
 
 _lib = None
@@ -129,6 +131,8 @@ class Stats:
     rows_active: int
     device_status: int
     device_site: int
+    channels: int = 0
+    channels_skipped: int = 0
 
     @property
     def density(self):
@@ -221,10 +225,11 @@ class GatedConv:
 
     def __init__(self, n, h, w, c_in, c_out, *, k=3, stride=1, pad=1, groups=4, dtype=CG_BF16,
                  bn_eps=1e-5, relu=True, has_residual=False, requant_shift=0,
-                 algo=CG_ALGO_AUTO, cond_mode=CG_COND_AUTO, grouping=False, device="cuda"):
+                 algo=CG_ALGO_AUTO, cond_mode=CG_COND_AUTO, grouping=False, channel_tau=0.0,
+                 device="cuda"):
         self.desc = CgConvDesc(n, h, w, c_in, c_out, k, k, stride, pad, groups, dtype, dtype,
                                bn_eps, int(relu), int(has_residual), requant_shift, algo, cond_mode,
-                               int(grouping))
+                               int(grouping), float(channel_tau))
         self.handle = cg_conv_create(self.desc)
         self.dtype = dtype
         self.ho = (h + 2 * pad - k) // stride + 1

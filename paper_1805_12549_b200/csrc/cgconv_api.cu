@@ -42,6 +42,8 @@ cg_status check_desc(const cg_conv_desc* d) {
   if (d->grouping != 0 && d->grouping != 1) return CG_ERR_INVALID_ARG;
   if (d->grouping && d->c_out % d->groups != 0) return CG_ERR_INVALID_ARG;
   if (d->grouping && d->in_dtype == CG_I8) return CG_ERR_INVALID_ARG;   // not defined for I8 layers
+  if (!(d->channel_tau >= 0.f)) return CG_ERR_INVALID_ARG;               // negative or NaN
+  if (d->channel_tau > 0.f && d->in_dtype == CG_I8) return CG_ERR_INVALID_ARG;
   return CG_OK;
 }
 
@@ -57,6 +59,7 @@ cg::LayerDims make_dims(const cg_conv_desc& d) {
   L.eps = d.bn_eps; L.relu = d.relu ? 1 : 0; L.has_residual = d.has_residual ? 1 : 0;
   L.shift = d.requant_shift;
   L.grouping = d.grouping;
+  L.channel_tau = d.channel_tau;
   return L;
 }
 
@@ -102,7 +105,10 @@ cg_status cg_conv_create(cg_conv_t* out, const cg_conv_desc* desc) {
   h->L = make_dims(*desc);
   h->counters = nullptr;
   std::memset(&h->maps, 0, sizeof(h->maps));
-  const bool tc_ok = cg::tc_plan(h->L, desc->in_dtype, desc->cond_mode, &h->plan);
+  // the channel-wise gate needs every partial sum of an image before any conditional path: it
+  // runs on the direct kernels
+  const bool tc_ok = !(desc->channel_tau > 0.f) &&
+                     cg::tc_plan(h->L, desc->in_dtype, desc->cond_mode, &h->plan);
   if (desc->algo == CG_ALGO_TENSOR && !tc_ok) { delete h; return CG_ERR_UNSUPPORTED; }
   h->use_tc = (desc->algo != CG_ALGO_DIRECT) && tc_ok;
   if (cudaGetDevice(&h->device) != cudaSuccess) { delete h; return CG_ERR_CUDA; }
@@ -128,11 +134,13 @@ void cg_conv_destroy(cg_conv_t h) {
 
 size_t cg_conv_workspace_bytes(cg_conv_t h) {
   if (!h) return 0;
+  if (h->L.channel_tau > 0.f) return cg::channel_gate_workspace_bytes(h->L);
   return h->use_tc ? cg::tc_workspace_bytes(h->L, h->plan) : 0;
 }
 
 int cg_conv_launches_per_forward(cg_conv_t h) {
   if (!h) return 0;
+  if (h->L.channel_tau > 0.f) return 2;
   return (h->use_tc && h->plan.cond_mode == CG_COND_COMPACT) ? 2 : 1;
 }
 
@@ -157,6 +165,10 @@ cg_status cg_conv_forward(cg_conv_t h, const void* x, const void* w_base, const 
   if (h->use_tc) {
     err = cg::launch_tc(h->L, h->plan, h->desc.in_dtype, &h->maps, x, w_base, w_cond, *bn, delta,
                         residual, y, mask_out, workspace, h->counters, stream);
+  } else if (h->L.channel_tau > 0.f) {
+    if (!aligned(workspace, 256)) return CG_ERR_ALIGNMENT;
+    err = cg::launch_direct_channel_gate(h->L, h->desc.in_dtype, x, w_base, w_cond, *bn, delta,
+                                         residual, y, mask_out, workspace, h->counters, stream);
   } else {
     err = cg::launch_direct(h->L, h->desc.in_dtype, x, w_base, w_cond, *bn, delta, residual, y,
                             mask_out, nullptr, 0, h->counters, stream);
@@ -250,6 +262,8 @@ cg_status cg_conv_stats(cg_conv_t h, cg_stats* out, void* cuda_stream) {
   out->rows_active = (int64_t)c[cg::CNT_ROWS_ACTIVE];
   out->device_status = (int32_t)c[cg::CNT_STATUS];
   out->device_site = (int32_t)c[cg::CNT_SITE];
+  out->channels = out->calls * L.n * L.c_out;
+  out->channels_skipped = (int64_t)c[cg::CNT_CH_SKIPPED];
   return out->device_status ? (cg_status)out->device_status : CG_OK;
 }
 

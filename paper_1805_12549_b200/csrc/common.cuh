@@ -20,6 +20,7 @@ struct LayerDims {
   float eps;
   int relu, has_residual, shift;
   int grouping;           // 1: output group i uses input group i as x_p (Section 3.3)
+  float channel_tau;      // > 0: channel-wise gate (Eq. 4)
 };
 
 // Device counter block owned by a handle: 16 x u64.
@@ -33,6 +34,7 @@ enum CounterSlot {
   CNT_STATUS = 6,   // first non-zero cg_status reported by a kernel
   CNT_SITE = 7,     // id of the wait/check that reported it
   CNT_CALLS = 8,    // forward passes executed (counted on the device: graph replays count)
+  CNT_CH_SKIPPED = 9,   // (image, output channel) pairs switched off by the channel-wise gate
   CNT_SLOTS = 16
 };
 
@@ -63,5 +65,13 @@ int launch_direct(const LayerDims& L, int in_dtype, const void* x, const void* w
                   const void* w_cond, const cg_bn_params& bn, const float* delta,
                   const void* residual, void* y, uint32_t* mask, void* p_out, int base_only,
                   unsigned long long* counters, cudaStream_t stream);
+// Layer with the channel-wise gate (Eq. 4), floating point only: partial sums and per-(image,
+// channel) counts, then the conditional path under both gates.  workspace as sized by
+// channel_gate_workspace_bytes.
+size_t channel_gate_workspace_bytes(const LayerDims& L);
+int launch_direct_channel_gate(const LayerDims& L, int in_dtype, const void* x, const void* w_base,
+                               const void* w_cond, const cg_bn_params& bn, const float* delta,
+                               const void* residual, void* y, uint32_t* mask, void* workspace,
+                               unsigned long long* counters, cudaStream_t stream);
 
 }  // namespace cg

@@ -115,7 +115,12 @@ direct_gated_conv_kernel(LayerDims L, const TIn* __restrict__ x, const TIn* __re
                          const float* __restrict__ delta, const TOut* __restrict__ residual,
                          TOut* __restrict__ y, uint32_t* __restrict__ mask,
                          float* __restrict__ p_out, int base_only,
-                         unsigned long long* __restrict__ counters) {
+                         unsigned long long* __restrict__ counters,
+                         int chan_pass = 0, int* __restrict__ chan_cnt = nullptr, float chan_need = 0.f) {
+  // chan_pass (channel-wise gate, Eq. 4): 1 = first pass: partial sums to p_out and, per image
+  // and output channel, the number of firing gates to chan_cnt; 2 = second pass: partial sums
+  // read back from p_out, conditional path only where the activation's gate fires AND the
+  // channel's count reaches chan_need = tau_c * h' * w'.
   extern __shared__ float s_consts[];   // 5 * c_out: t, a1, b1, a2, b2
   __shared__ unsigned long long s_active;
   float* s_t = s_consts;
@@ -148,11 +153,20 @@ direct_gated_conv_kernel(LayerDims L, const TIn* __restrict__ x, const TIn* __re
     bool fire = false;
     if (valid) {
       const int grp = L.grouping ? co / (L.c_out / L.groups) : 0;   // input group of the base path
-      const float p = conv_point<TIn>(L, x, w_base, n, ho, wo, co, grp * L.c_p, L.c_p);
+      const float p = chan_pass == 2 ? p_out[m * L.c_out + co]
+                                     : conv_point<TIn>(L, x, w_base, n, ho, wo, co, grp * L.c_p, L.c_p);
       if (base_only) {
         p_out[m * L.c_out + co] = p;
+      } else if (chan_pass == 1) {
+        p_out[m * L.c_out + co] = p;
+        if (p >= s_t[co]) atomicAdd(&chan_cnt[(long long)n * L.c_out + co], 1);
       } else {
         fire = (p >= s_t[co]);   // NaN compares false
+        if (chan_pass == 2) {
+          const bool on = ((float)chan_cnt[(long long)n * L.c_out + co] >= chan_need);
+          fire = fire && on;
+          if (!on && ho == 0 && wo == 0) atomicAdd(&counters[CNT_CH_SKIPPED], 1ull);
+        }
         float v;
         if (fire) {
           const float r = L.grouping ? conv_point_others<TIn>(L, x, w_cond, n, ho, wo, co, grp)
@@ -166,7 +180,7 @@ direct_gated_conv_kernel(LayerDims L, const TIn* __restrict__ x, const TIn* __re
         st_out(y + m * L.c_out + co, v);
       }
     }
-    if (!base_only) {
+    if (!base_only && chan_pass != 1) {
       const unsigned word = __ballot_sync(0xffffffffu, fire);
       if (lane == 0) {
         if (mask) mask[it] = word;
@@ -174,7 +188,7 @@ direct_gated_conv_kernel(LayerDims L, const TIn* __restrict__ x, const TIn* __re
       }
     }
   }
-  if (!base_only) {
+  if (!base_only && chan_pass != 1) {
     if (lane == 0 && my_active) atomicAdd(&s_active, my_active);
     __syncthreads();
     if (threadIdx.x == 0 && blockIdx.x == 0) atomicAdd(&counters[CNT_CALLS], 1ull);
@@ -272,6 +286,48 @@ int launch_direct(const LayerDims& L, int in_dtype, const void* x, const void* w
         (int*)p_out, base_only, counters);
   }
   return (int)cudaGetLastError();
+}
+
+// workspace of the channel-wise gate: [partial sums: M x c_out fp32][counts: n x c_out int32]
+size_t channel_gate_workspace_bytes(const LayerDims& L) {
+  const size_t p_bytes = ((size_t)L.m * L.c_out * sizeof(float) + 255) / 256 * 256;
+  return p_bytes + ((size_t)L.n * L.c_out * sizeof(int) + 255) / 256 * 256;
+}
+
+int launch_direct_channel_gate(const LayerDims& L, int in_dtype, const void* x, const void* w_base,
+                               const void* w_cond, const cg_bn_params& bn, const float* delta,
+                               const void* residual, void* y, uint32_t* mask, void* workspace,
+                               unsigned long long* counters, cudaStream_t stream) {
+  const long long items = L.m * L.words;
+  if (items == 0) return 0;
+  if (in_dtype != CG_F32 && in_dtype != CG_BF16) return (int)cudaErrorInvalidValue;
+  const size_t p_bytes = ((size_t)L.m * L.c_out * sizeof(float) + 255) / 256 * 256;
+  float* p_ws = (float*)workspace;
+  int* cnt_ws = (int*)((char*)workspace + p_bytes);
+  cudaError_t e = cudaMemsetAsync(cnt_ws, 0, (size_t)L.n * L.c_out * sizeof(int), stream);
+  if (e != cudaSuccess) return (int)e;
+  const int warps_per_block = kThreads / 32;
+  long long blocks = (items + warps_per_block - 1) / warps_per_block;
+  const long long cap = 148ll * 8 * 8;
+  if (blocks > cap) blocks = cap;
+  const size_t smem = (size_t)5 * L.c_out * sizeof(float);
+  // Eq. 4's threshold on the count, in fp32 like the comparison itself
+  const float need = L.channel_tau * (float)(L.ho * L.wo);
+  for (int pass = 1; pass <= 2; ++pass) {
+    if (in_dtype == CG_F32) {
+      direct_gated_conv_kernel<float, float><<<(unsigned)blocks, kThreads, smem, stream>>>(
+          L, (const float*)x, (const float*)w_base, (const float*)w_cond, bn, delta,
+          (const float*)residual, (float*)y, mask, p_ws, 0, counters, pass, cnt_ws, need);
+    } else {
+      direct_gated_conv_kernel<__nv_bfloat16, __nv_bfloat16><<<(unsigned)blocks, kThreads, smem, stream>>>(
+          L, (const __nv_bfloat16*)x, (const __nv_bfloat16*)w_base, (const __nv_bfloat16*)w_cond, bn,
+          delta, (const __nv_bfloat16*)residual, (__nv_bfloat16*)y, mask, p_ws, 0, counters, pass,
+          cnt_ws, need);
+    }
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return (int)e;
+  }
+  return 0;
 }
 
 }  // namespace cg

@@ -138,7 +138,7 @@ extern "C" cg_status cg_conv_forward_static(const cg_conv_desc* d, const void* x
     return CG_ERR_INVALID_ARG;
   if (d->in_dtype != d->out_dtype || (d->in_dtype != CG_F32 && d->in_dtype != CG_BF16))
     return CG_ERR_UNSUPPORTED;
-  if (d->grouping) return CG_ERR_UNSUPPORTED;
+  if (d->grouping || d->channel_tau > 0.f) return CG_ERR_UNSUPPORTED;
   if (d->c_out > kMaxChannels) return CG_ERR_WORKSPACE;   // would not fit the static scratch
   if (!bn->gamma || !bn->beta || !bn->mean_base || !bn->var_base || !bn->mean_full || !bn->var_full ||
       (bn->gate_mean == nullptr) != (bn->gate_var == nullptr))
@@ -169,7 +169,7 @@ extern "C" cg_status cg_conv_forward_static(const cg_conv_desc* d, const void* x
   L.wo = (d->w + 2 * d->pad - d->kw) / d->stride + 1;
   L.m = (long long)d->n * L.ho * L.wo;
   L.words = (d->c_out + 31) / 32;
-  L.eps = d->bn_eps; L.relu = d->relu ? 1 : 0; L.has_residual = d->has_residual ? 1 : 0; L.shift = 0; L.grouping = 0;
+  L.eps = d->bn_eps; L.relu = d->relu ? 1 : 0; L.has_residual = d->has_residual ? 1 : 0; L.shift = 0; L.grouping = 0; L.channel_tau = 0.f;
 
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   const int pro_threads = 256;
@@ -202,6 +202,7 @@ extern "C" cg_status cg_conv_forward_static(const cg_conv_desc* d, const void* x
     stats_out->dense_macs = stats_out->outputs * k2 * L.c_in;
     stats_out->gated_macs = k2 * ((long long)L.c_p * stats_out->outputs + (long long)L.c_r * stats_out->active);
     stats_out->executed_macs = stats_out->gated_macs;
+    stats_out->channels = (int64_t)L.n * L.c_out;
   }
   return CG_OK;
 }

@@ -30,6 +30,7 @@ class Case:
     residual: np.ndarray | None = None
     shift: int = 0
     grouped: bool = False
+    channel_tau: float = 0.0    # tau_c of the channel-wise gate (Eq. 4); 0 = off
 
 
 def _quantile_delta(p_hat: np.ndarray, density: float) -> float:
@@ -106,7 +107,8 @@ def run_oracle(c: Case, **kw) -> O.Result:
     if c.dtype == "i8":
         return O.gated_conv_i8(c.s, c.shift, c.x, c.wb, c.wc, c.bn)
     return O.gated_conv(c.s, c.x, c.wb, c.wc, c.bn, c.delta, c.residual,
-                        out_bf16=(c.dtype == "bf16"), grouped=c.grouped, **kw)
+                        out_bf16=(c.dtype == "bf16"), grouped=c.grouped,
+                        channel_tau=c.channel_tau, **kw)
 
 
 # ----------------------------------------------------------------------------- GPU side
@@ -134,7 +136,8 @@ class GpuCase:
         self.conv = B.GatedConv(s.n, s.h, s.w, s.c_in, s.c_out, k=s.kh, stride=s.stride, pad=s.pad,
                                 groups=s.groups, dtype=dt, bn_eps=s.bn_eps, relu=bool(s.relu),
                                 has_residual=c.residual is not None, requant_shift=c.shift,
-                                algo=algo, cond_mode=cond_mode, grouping=c.grouped)
+                                algo=algo, cond_mode=cond_mode, grouping=c.grouped,
+                                channel_tau=c.channel_tau)
         self.x = _to_dev(c.x, c.dtype)
         self.wb = _to_dev(c.wb, c.dtype)
         self.wc = _to_dev(c.wc, c.dtype)

@@ -143,3 +143,62 @@ def test_forward_argument_errors():
     assert lib.cg_conv_forward(*args(bn=bad)) == 1
     g.conv.stats()
     g.close()
+
+
+# ----------------------------------------------------------------------------- channel-wise gate
+CHANNEL_GATE_SHAPES = [
+    O.Shape(2, 8, 8, 16, 16, groups=4),
+    O.Shape(3, 7, 9, 8, 40, groups=2),
+    O.Shape(5, 14, 14, 64, 96, groups=4),
+    O.Shape(2, 9, 9, 12, 33, stride=2, groups=4),
+]
+
+
+@pytest.mark.parametrize("s", CHANNEL_GATE_SHAPES)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("tau", [0.3, 0.45])
+def test_channel_wise_gate(s, dtype, tau):
+    """Eq. 4 through the C ABI: per image, channels whose gate fires at fewer than tau_c*h'*w'
+    positions take the base path everywhere.  Integer counts and one fp32 comparison, so the
+    decisions, masks and outputs are bit-exact against the oracle."""
+    c = K.make_float_case("chgate", s, dtype, density=0.4)
+    c.channel_tau = tau
+    ref = K.run_oracle(c)
+    g = K.GpuCase(c)            # algo AUTO: the channel-wise gate selects the direct kernels
+    assert not g.conv.uses_tensor_cores
+    y, mask, st = g.run()
+    K.compare(c, ref, y, mask, st, exact=True)
+    assert st.channels == ref.channels == s.n * s.c_out
+    assert st.channels_skipped == ref.channels_skipped
+    assert st.active == ref.active
+    assert 0 < st.channels_skipped < st.channels, "the case should drop some channels, not all"
+    # a second call reuses the workspace (counts are cleared per call)
+    y2, mask2, st2 = g.run()
+    np.testing.assert_array_equal(mask, mask2)
+    assert st2.channels_skipped == ref.channels_skipped
+    g.close()
+
+
+def test_channel_wise_gate_limits_and_rejections():
+    from paper_1805_12549_b200 import binding as B
+    s = O.Shape(2, 8, 8, 16, 32, groups=4)
+    c = K.make_float_case("chlim", s, "bf16", density=0.4)
+    plain = K.run_oracle(c)
+    c.channel_tau = 1.5                       # no count reaches 1.5*h'*w': every channel off
+    ref = K.run_oracle(c)
+    g = K.GpuCase(c)
+    y, mask, st = g.run()
+    K.compare(c, ref, y, mask, st, exact=True)
+    assert st.active == 0 and st.channels_skipped == st.channels
+    g.close()
+    assert plain.active > 0
+    # tensor-core kernels and int8 layers do not take the channel-wise gate
+    with pytest.raises(B.CgError) as e:
+        B.GatedConv(2, 28, 28, 128, 128, algo=B.CG_ALGO_TENSOR, channel_tau=0.2)
+    assert e.value.status == 2
+    with pytest.raises(B.CgError) as e:
+        B.GatedConv(2, 28, 28, 128, 128, dtype=B.CG_I8, requant_shift=8, channel_tau=0.2)
+    assert e.value.status == 1
+    with pytest.raises(B.CgError) as e:
+        B.GatedConv(2, 8, 8, 16, 16, channel_tau=-0.1)
+    assert e.value.status == 1
