@@ -173,6 +173,7 @@ struct MmaIssuer {
   uint32_t d_tmem, idesc, a_grp, b_lo, acc, blk_off_b;
   int a_first, b_held;
   bool ok;
+  bool share, release;   // shared patch ring: slot by job index; release: this issuer frees patches
 
   // slot0, slots: the part of the patch ring this issuer consumes
   __device__ __forceinline__ void init(Shared* sh_, const Ctx& cx_, const uint8_t* s_a,
@@ -197,6 +198,7 @@ struct MmaIssuer {
     base_chunks = P.base_chunks; base_tiles = P.base_tiles; kh = L.kh; kw = L.kw; planes = P.planes;
     as = slot0; bs = 0; apar = 0; bpar = 0;
     a_first = slot0; b_held = 0; ok = true;
+    share = false; release = true;
   }
   __device__ __forceinline__ void mma(uint32_t al, uint32_t bl) {
     const uint64_t da = ((uint64_t)desc_hi << 32) | al;
@@ -216,6 +218,7 @@ struct MmaIssuer {
     }
   }
   __device__ __forceinline__ void release_a() {
+    if (!release) return;
     for (int pl = 0; pl < planes; ++pl) ptx::umma_commit(&sh->a_empty[a_first + pl]);
   }
   // Next weight tile.  Resident weights: tiles follow one another from b_lo on (b_lo includes
@@ -319,8 +322,9 @@ struct MmaIssuer {
   }
   // base or conditional MMAs of one job into the accumulator at d; `blocks` = column blocks to
   // compute (all of them for the base path)
-  __device__ __forceinline__ bool run_phase(uint32_t d, bool cond, uint32_t blocks) {
+  __device__ __forceinline__ bool run_phase(uint32_t d, bool cond, uint32_t blocks, int j) {
     constexpr uint32_t kAll = (1u << (NT / 64)) - 1u;
+    if (share) { as = j % na; apar = (uint32_t)(j / na) & 1u; }   // (a0 = 0 in this mode)
     // a single block of two: accumulator columns and weight rows 64..127
     d_tmem = d + (blocks == 2u ? 64u : 0u);
     blk_off_b = blocks == 2u ? (64u * 128u / 16u) : 0u;
@@ -445,8 +449,10 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   if (warp == 0) {
     // ============================================================ patch (A) producer
     // Loads chunks in the order the MMA issuer consumes them: base(0) | base(1) cond(0) | ...
-    // With two issuers the ring is split: slots [0, split_a) for the base path, the rest for the
-    // conditional path, each part with its own cursor.
+    // With two issuers the ring is either split -- slots [0, split_a) for the base path, the
+    // rest for the conditional path, each part with its own cursor -- or, when the layer has a
+    // single input chunk, shared: job j's patch is loaded once into slot j % na and serves both
+    // paths (the conditional issuer releases it).
     if (lane == 0 && jobs > 0) {
       // ring slot and the parity of its "empty" barrier, per ring part
       int as0 = 0, as1 = P.split_a;
@@ -474,7 +480,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       const int cond_part = P.split_a ? 1 : 0;
       for (int j = 0; j <= jobs && ok; ++j) {
         if (j < jobs) load_chunks(j, 0, P.base_chunks, 0);
-        if (j >= 1 && has_cond && ok) {
+        if (j >= 1 && has_cond && ok && !P.share_a) {
           const int jj = j - 1;
           uint32_t blocks = kAllBlocks;
           if (!dense) {
@@ -530,11 +536,13 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     // the patch ring is split (resident weights), warp 3 takes the conditional path instead, so
     // the per-job bookkeeping of the two paths runs in parallel.
     const bool do_base = warp == 1;
-    const bool do_cond = P.split_a ? warp == 3 : warp == 1;
+    const bool do_cond = P.issuers == 2 ? warp == 3 : warp == 1;
     if (lane == 0 && jobs > 0 && (do_base || do_cond)) {
       MmaIssuer<NT, I8> mi;
       if (P.split_a) mi.init(sh, cx, s_a, s_b, P, L, do_base ? 0 : P.split_a, do_base ? P.split_a : P.na - P.split_a);
       else mi.init(sh, cx, s_a, s_b, P, L, 0, P.na);
+      mi.share = P.share_a != 0;
+      mi.release = !(P.share_a && do_base);   // a shared patch is released by the conditional issuer
       bool ok = true;
       if (P.resident) ok = wait_bar(cx, &sh->w_ready, 0, 6);
       for (int j = 0; j <= jobs && ok; ++j) {
@@ -543,7 +551,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
           ok = wait_bar(cx, &sh->p_free[ps], ((j / kNP) & 1) ^ 1, 9);
           if (!ok) break;
           ptx::tc_fence_after();
-          ok = mi.run_phase(tmem + (uint32_t)(ps * NT), false, kAllBlocks);
+          ok = mi.run_phase(tmem + (uint32_t)(ps * NT), false, kAllBlocks, j);
           if (!ok) break;
           ptx::umma_commit(&sh->base_done[ps]);
         }
@@ -563,8 +571,10 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
             if (!ok) break;
             if (blocks) {
               ptx::tc_fence_after();
-              ok = mi.run_phase(tmem + (uint32_t)((kNP + rs) * NT), true, blocks);
+              ok = mi.run_phase(tmem + (uint32_t)((kNP + rs) * NT), true, blocks, jj);
               if (!ok) break;
+            } else if (P.share_a) {
+              ptx::mbar_arrive(&sh->a_empty[jj % P.na]);   // the job's patch is not needed again
             }
           } else {
             ok = wait_bar(cx, &sh->r_free[rs], ((jj / kNR) & 1) ^ 1, 15);
@@ -1244,8 +1254,10 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
     P.nt = nt; P.na = na; P.nb = nb; P.resident = resident; P.tiles_n = L.c_out / nt;
     // resident weights: the base and the conditional path get their own MMA issuer and their own
     // half of the patch ring
-    P.split_a = (resident && P.cond_tiles > 0 && P.cond_mode != CG_COND_COMPACT && na >= 2 * P.planes &&
-                 (na / 2) % P.planes == 0) ? na / 2 : 0;
+    const bool two = resident && P.cond_tiles > 0 && P.cond_mode != CG_COND_COMPACT;
+    P.share_a = (two && P.chunks == 1 && P.planes == 1) ? 1 : 0;
+    P.split_a = (two && !P.share_a && na >= 2 * P.planes && (na / 2) % P.planes == 0) ? na / 2 : 0;
+    P.issuers = (P.share_a || P.split_a) ? 2 : 1;
     P.smem_bytes = (unsigned)(off + 1024);
     P.valid = 1;
     *plan = P;

@@ -24,8 +24,12 @@ struct TcPlan {
   int planes;           // patch buffers per chunk: 1 (stride 1) or 4 (stride 2: the input's
                         // even/odd row x even/odd column sub-images)
   int na;               // patch buffers in the ring
-  int split_a;          // > 0: slots [0, split_a) serve the base path and the rest the conditional
-                        // path, each with its own MMA-issuing thread; 0: one ring, one issuer
+  int issuers;          // MMA-issuing threads: 1, or 2 (base path / conditional path) when the
+                        // weights are resident
+  int split_a;          // 2 issuers, > 0: slots [0, split_a) serve the base path and the rest the
+                        // conditional path
+  int share_a;          // 2 issuers, 1: one input chunk serves both paths, so job j's patch stays
+                        // in slot j % na from its base MMAs until its conditional MMAs are done
   int nb;               // weight-tile ring depth (0 when the weights are resident)
   int resident;         // 1: all weight tiles of a column tile stay in shared memory
   int box_h;            // patch box rows: r + 2*pad (rows mode) or h + pad (images mode)
