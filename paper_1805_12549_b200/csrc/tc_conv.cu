@@ -27,7 +27,7 @@
 // Weights stay resident in shared memory when they fit, otherwise they stream through a ring.
 //
 // Warp roles: 0 = patch (A) producer, 1 = MMA issuer (owns TMEM), 2 = weight (B) producer,
-// 3-10 = epilogue.  Every mbarrier wait is bounded; on expiry the CTA records
+// 3 = second MMA issuer (conditional path, resident weights), 4-19 = epilogue.  Every mbarrier wait is bounded; on expiry the CTA records
 // CG_ERR_DEVICE_TIMEOUT with the id of the wait and leaves.
 #include <cstring>
 
@@ -38,10 +38,13 @@ namespace cg {
 
 namespace {
 
-constexpr int kThreads = 384;       // 4 single-thread warps + 8 epilogue warps
+constexpr int kThreads = 640;       // 4 single-thread warps + 16 epilogue warps
 constexpr int kEpiWarp0 = 4;        // warps 0-3: patch producer, MMA issuer, weight producer, second MMA issuer
 constexpr int kEpiThread0 = kEpiWarp0 * 32;
-constexpr int kEpiThreads = 256;
+constexpr int kEpiThreads = 512;
+constexpr int kEpiWarps = kEpiThreads / 32;
+constexpr int kGroupWarps = kEpiWarps / 2;   // gate group, combine group
+constexpr int kGroupThreads = kGroupWarps * 32;
 constexpr int kBM = 128;            // MMA M: patch rows per job
 constexpr int kSpinLimit = 1 << 21; // try_wait polls before a wait gives up ...
 constexpr long long kWaitCycles = 2000000000ll;   // ... or about one second of SM clocks, whichever is first
@@ -112,6 +115,22 @@ struct Ctx {
   unsigned long long* counters;
 };
 
+#ifdef CG_PROF
+// Profiling build only: cycles that each warp of CTA 0 spent inside every bounded wait
+// ([warp][site]), and the cycles of its role loops ([warp][31]).
+__device__ unsigned long long g_prof[24 * 32];
+__device__ unsigned long long g_tl[16 * 16];   // [job][event] clock stamps of CTA 0
+#define CG_PROF_EV(j, ev) \
+  do { if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && (j) < 16) g_tl[(j) * 16 + (ev)] = (unsigned long long)clock64(); } while (0)
+#define CG_PROF_T(var) const long long var = clock64()
+#define CG_PROF_ADD(slot, t0, t1) \
+  do { if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) atomicAdd(&g_prof[(threadIdx.x >> 5) * 32 + (slot)], (unsigned long long)((t1) - (t0))); } while (0)
+#else
+#define CG_PROF_EV(j, ev)
+#define CG_PROF_T(var)
+#define CG_PROF_ADD(slot, t0, t1)
+#endif
+
 // Bounded wait.  The first poll is inline; the loop lives in one out-of-line copy so that the
 // role loops stay small.  Each poll parks the thread in hardware for a short time; the wait
 // gives up after about a second; a CTA that already gave up elsewhere is noticed within a few polls.
@@ -119,7 +138,13 @@ __device__ __noinline__ bool wait_bar_slow(Shared* sh, unsigned long long* count
                                            uint32_t parity, int site) {
   const long long t0 = clock64();
   for (int i = 0; i < kSpinLimit; ++i) {
-    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if (ptx::mbar_try_wait(bar, parity)) {
+#ifdef CG_PROF
+      if (blockIdx.x == 0 && (threadIdx.x & 31) == 0)
+        atomicAdd(&g_prof[(threadIdx.x >> 5) * 32 + site], (unsigned long long)(clock64() - t0));
+#endif
+      return true;
+    }
     if ((i & 15) == 15) {
       if (*(volatile uint32_t*)&sh->abort_flag) return false;
       if (clock64() - t0 > kWaitCycles) break;
@@ -132,25 +157,42 @@ __device__ __noinline__ bool wait_bar_slow(Shared* sh, unsigned long long* count
 }
 
 __device__ __forceinline__ bool wait_bar(const Ctx& cx, uint64_t* bar, uint32_t parity, int site) {
+#ifdef CG_PROF
+  const long long t0 = clock64();
+  const bool fast = ptx::mbar_try_wait(bar, parity, 0u);
+  if (blockIdx.x == 0 && (threadIdx.x & 31) == 0)
+    atomicAdd(&g_prof[(threadIdx.x >> 5) * 32 + 26 + (fast ? 0 : 1)], (unsigned long long)(clock64() - t0));
+  if (fast) return true;
+#else
   if (ptx::mbar_try_wait(bar, parity, 0u)) return true;
+#endif
   return wait_bar_slow(cx.sh, cx.counters, bar, parity, site);
+}
+
+// The same wait taken by every lane of a convergent warp; the outcome is made warp-uniform.
+__device__ __forceinline__ bool wait_bar_warp(const Ctx& cx, uint64_t* bar, uint32_t parity, int site) {
+  return __all_sync(0xffffffffu, wait_bar(cx, bar, parity, site));
 }
 
 __device__ __forceinline__ uint32_t slot_blocks(const Shared* sh, int slot) {
   const volatile uint32_t* w = sh->warp_blk[slot];
-  return w[0] | w[1] | w[2] | w[3] | w[4] | w[5] | w[6] | w[7];
+  uint32_t b = 0;
+#pragma unroll
+  for (int i = 0; i < kGroupWarps; ++i) b |= w[i];
+  return b;
 }
 
-// MMA issue for one CTA, run by ONE thread.  A lone thread executes about one dependent
-// instruction every 4-5 cycles and a branch costs several times that, while the tensor pipe
-// needs only 49/64/128 cycles per MMA at N = 64/128/256: with more than about eight
-// instructions per MMA the issue loop, not the tensor pipe, sets the pace (measured: 280 cycles
-// per filter tap with a rolled tap loop and a handful of run-time conditions in it).  So for 3x3
-// kernels the taps of a filter row and their K steps are unrolled, every descriptor is a
-// register plus an immediate, and what distinguishes the layer variants (stride-2 planes, a
-// single column block) is folded into those registers instead of into branches.  Weight tiles
-// are visited in the order base_tile()/cond_tile() enumerate them, which is the order the weight
-// producer loads them.
+// MMA issue for one CTA, run by ONE thread.  Two measured facts shape this code.  (1) The
+// whole kernel must fit the instruction cache: with every tap, K step and layer variant unrolled
+// at two call sites it was about 260 KB of code, every role ran from instruction-cache misses,
+// and one MMA took 130-300 cycles to issue.  (2) A tcgen05.mma slot costs about 50 cycles of
+// the issuing thread whether or not its predicate is on, and a rolled loop with run-time
+// bounds costs 200-300 cycles per tap; with the three taps of a filter row and their K steps
+// unrolled (compile-time K range, descriptors = register + immediate) the same thread issues
+// at the rate of the tensor pipe (50-62 cycles per 128x64x16 MMA).  So: 3x3 layers run through
+// a few small unrolled variants selected once per phase, everything else through one rolled
+// loop, and the phase is inlined at a single call site.  Weight tiles are visited in the order
+// base_tile()/cond_tile() enumerate them, which is the order the weight producer loads them.
 template <int NT, bool I8>
 struct MmaIssuer {
   static constexpr uint32_t kWTile = (uint32_t)(NT * 128) >> 4;   // weight tile, 16-byte units
@@ -174,6 +216,7 @@ struct MmaIssuer {
   int a_first, b_held;
   bool ok;
   bool share, release;   // shared patch ring: slot by job index; release: this issuer frees patches
+  uint32_t lead;         // 1 in the lane that issues the tcgen05 instructions (the whole warp runs this code)
 
   // slot0, slots: the part of the patch ring this issuer consumes
   __device__ __forceinline__ void init(Shared* sh_, const Ctx& cx_, const uint8_t* s_a,
@@ -203,8 +246,8 @@ struct MmaIssuer {
   __device__ __forceinline__ void mma(uint32_t al, uint32_t bl) {
     const uint64_t da = ((uint64_t)desc_hi << 32) | al;
     const uint64_t db = ((uint64_t)desc_hi << 32) | bl;
-    if (I8) ptx::umma_s8(d_tmem, da, db, idesc, acc);
-    else ptx::umma_bf16(d_tmem, da, db, idesc, acc);
+    if (I8) ptx::umma_s8_if(lead, d_tmem, da, db, idesc, acc);
+    else ptx::umma_bf16_if(lead, d_tmem, da, db, idesc, acc);
     acc = 1u;
   }
   // the patch buffer(s) of the next chunk in the ring: one, or the four planes of a stride-2
@@ -213,20 +256,20 @@ struct MmaIssuer {
     a_first = as;
     a_grp = a_base_lo + (uint32_t)as * patch_lo;
     for (int pl = 0; pl < planes; ++pl) {
-      ok = ok && wait_bar(cx, &sh->a_full[as], apar, 7);
+      ok = ok && wait_bar_warp(cx, &sh->a_full[as], apar, 7);
       if (++as == na) { as = a0; apar ^= 1; }
     }
   }
   __device__ __forceinline__ void release_a() {
     if (!release) return;
-    for (int pl = 0; pl < planes; ++pl) ptx::umma_commit(&sh->a_empty[a_first + pl]);
+    for (int pl = 0; pl < planes; ++pl) ptx::umma_commit_if(lead, &sh->a_empty[a_first + pl]);
   }
   // Next weight tile.  Resident weights: tiles follow one another from b_lo on (b_lo includes
   // the column-block offset).  Ring: wait for the slot.
   template <bool RES>
   __device__ __forceinline__ uint32_t acquire_b() {
     if (RES) { const uint32_t b = b_lo; b_lo += kWTile; return b; }
-    ok = ok && wait_bar(cx, &sh->b_full[bs], bpar, 8);
+    ok = ok && wait_bar_warp(cx, &sh->b_full[bs], bpar, 8);
     b_held = bs;
     const uint32_t b = b_base_lo + (uint32_t)bs * kWTile + blk_off_b;
     if (++bs == nb) { bs = 0; bpar ^= 1; }
@@ -234,90 +277,102 @@ struct MmaIssuer {
   }
   template <bool RES>
   __device__ __forceinline__ void release_b() {
-    if (!RES) ptx::umma_commit(&sh->b_empty[b_held]);
+    if (!RES) ptx::umma_commit_if(lead, &sh->b_empty[b_held]);
   }
-  // K steps [KS0, KS1) of every tap of the next chunk in the ring, one weight tile per tap
+  // 3x3: K steps [KS0, KS1) of every tap of the next chunk in the ring, one weight tile per tap
   template <bool RES, int KS0, int KS1>
-  __device__ __forceinline__ void chunk_taps() {
+  __device__ __forceinline__ void chunk_taps3() {
     acquire_a();
     if (!ok) return;
-    if (kh == 3 && kw == 3) {
-      uint32_t a_row = a_grp + f0;
+    // (the row step is carried in a variable, not selected by r, so that the loop stays rolled)
+    uint32_t a_row = a_grp + f0, step = f1 - f0;
 #pragma unroll 1
-      for (int r = 0; r < 3; ++r) {
+    for (int r = 0; r < 3; ++r) {
 #pragma unroll
-        for (int sx = 0; sx < 3; ++sx) {
-          const uint32_t b_t = acquire_b<RES>();
-          if (!RES && !ok) return;
-          const uint32_t a_t = a_row + (sx == 0 ? c0 : sx == 1 ? c1 : c2);
+      for (int sx = 0; sx < 3; ++sx) {
+        const uint32_t b_t = acquire_b<RES>();
+        if (!RES && !ok) return;
+        const uint32_t a_t = a_row + (sx == 0 ? c0 : sx == 1 ? c1 : c2);
 #pragma unroll
-          for (int ks = KS0; ks < KS1; ++ks) mma(a_t + ks * 2, b_t + (ks - KS0) * 2);
-          release_b<RES>();
-        }
-        a_row += r == 0 ? f1 - f0 : f2 - f1;
+        for (int ks = KS0; ks < KS1; ++ks) mma(a_t + ks * 2, b_t + (ks - KS0) * 2);
+        release_b<RES>();
       }
-    } else {
-      uint32_t a_row = a_grp;
-      for (int r = 0; r < kh; ++r) {
-        for (int sx = 0; sx < kw; ++sx) {
-          const uint32_t b_t = acquire_b<RES>();
-          if (!RES && !ok) return;
-          const uint32_t a_t = a_row + (uint32_t)sx * 8u;
-#pragma unroll
-          for (int ks = KS0; ks < KS1; ++ks) mma(a_t + ks * 2, b_t + (ks - KS0) * 2);
-          release_b<RES>();
-        }
-        a_row += row_lo;
-      }
+      a_row += step;
+      step = f2 - f1;
     }
     release_a();
   }
-  // base path when c_p < 64: the first KP K steps of chunk 0; a weight tile covers 4/KP taps
+  // 3x3 base path when c_p < 64: the first KP K steps of chunk 0; a weight tile covers 4/KP taps
   template <bool RES, int KP>
-  __device__ __forceinline__ void base_small() {
+  __device__ __forceinline__ void base_small3() {
     constexpr int TPT = 4 / KP;
     acquire_a();
     if (!ok) return;
-    if (kh == 3 && kw == 3) {
-      uint32_t b_t = 0;
+    uint32_t b_t = 0;
 #pragma unroll
-      for (int t = 0; t < 9; ++t) {
-        if (t % TPT == 0) b_t = acquire_b<RES>();
-        if (!RES && !ok) return;
-        const uint32_t a_t = a_grp + (t / 3 == 0 ? f0 : t / 3 == 1 ? f1 : f2) + (t % 3 == 0 ? c0 : t % 3 == 1 ? c1 : c2);
+    for (int t = 0; t < 9; ++t) {
+      if (t % TPT == 0) b_t = acquire_b<RES>();
+      if (!RES && !ok) return;
+      const uint32_t a_t = a_grp + (t / 3 == 0 ? f0 : t / 3 == 1 ? f1 : f2) + (t % 3 == 0 ? c0 : t % 3 == 1 ? c1 : c2);
 #pragma unroll
-        for (int ks = 0; ks < KP; ++ks) mma(a_t + ks * 2, b_t + ((t % TPT) * KP + ks) * 2);
-        if (t % TPT == TPT - 1 || t == 8) release_b<RES>();
-      }
-    } else {
-      uint32_t a_row = a_grp, b_t = 0;
-      int in_tile = 0;
-      for (int r = 0; r < kh; ++r) {
-        for (int sx = 0; sx < kw; ++sx) {
-          if (in_tile == 0) b_t = acquire_b<RES>();
-          if (!RES && !ok) return;
-          const uint32_t a_t = a_row + (uint32_t)sx * 8u;
-#pragma unroll
-          for (int ks = 0; ks < KP; ++ks) mma(a_t + ks * 2, b_t + (uint32_t)(in_tile * KP + ks) * 2u);
-          if (++in_tile == TPT) { release_b<RES>(); in_tile = 0; }
-        }
-        a_row += row_lo;
-      }
-      if (in_tile != 0) release_b<RES>();
+      for (int ks = 0; ks < KP; ++ks) mma(a_t + ks * 2, b_t + ((t % TPT) * KP + ks) * 2);
+      if (t % TPT == TPT - 1 || t == 8) release_b<RES>();
     }
     release_a();
   }
+  // any kernel size (stride 1): K steps [ks0, ks1) of every tap of the next chunk, a weight
+  // tile covering `tpt` taps.  Rolled; slow to issue, small in code.
+  __device__ __forceinline__ void chunk_taps_any(int ks0, int ks1, int tpt) {
+    acquire_a();
+    if (!ok) return;
+    int in_tile = 0;
+    uint32_t b_t = 0;
+    for (int r = 0; r < kh; ++r) {
+      const uint32_t a_row = a_grp + (uint32_t)r * row_lo;
+      for (int sx = 0; sx < kw; ++sx) {
+        if (in_tile == 0) {
+          b_t = resident ? acquire_b<true>() : acquire_b<false>();
+          if (!ok) return;
+        }
+        const uint32_t a_t = a_row + (uint32_t)sx * 8u;
+        const uint32_t b_k = b_t + (uint32_t)((in_tile * (ks1 - ks0) - ks0) * 2);
+        for (int ks = ks0; ks < ks1; ++ks) mma(a_t + ks * 2, b_k + ks * 2);
+        if (++in_tile == tpt) { if (!resident) release_b<false>(); in_tile = 0; }
+      }
+    }
+    if (in_tile != 0 && !resident) release_b<false>();
+    release_a();
+  }
+  // Chunks and K ranges of a phase.
+  //   c_p >= one chunk: the base path takes chunks [0, base_chunks), the conditional path the
+  //   rest; every tap of a chunk has its own weight tile and four K steps.
+  //   c_p < one chunk (kp16 = 1 or 2 K steps): the base path takes K steps [0, kp16) of chunk
+  //   0, a weight tile covering 4/kp16 taps; the conditional path takes K steps [kp16, 4) of
+  //   chunk 0 and then the remaining chunks.
   template <bool RES>
-  __device__ __forceinline__ void phase(bool cond) {
+  __device__ __forceinline__ void phase3(bool cond) {
+    int nfull;   // whole chunks (four K steps per tap) after the first, partial one
+    if (kp16 >= 4) {
+      nfull = cond ? chunks - base_chunks : base_chunks;
+    } else if (!cond) {
+      if (kp16 == 1) base_small3<RES, 1>(); else base_small3<RES, 2>();
+      nfull = 0;
+    } else {
+      if (kp16 == 1) chunk_taps3<RES, 1, 4>(); else chunk_taps3<RES, 2, 4>();
+      nfull = chunks - 1;
+    }
+#pragma unroll 1
+    for (int q = 0; q < nfull && ok; ++q) chunk_taps3<RES, 0, 4>();
+  }
+  __device__ __forceinline__ void phase_any(bool cond) {
     if (kp16 >= 4) {
       const int q0 = cond ? base_chunks : 0, q1 = cond ? chunks : base_chunks;
-      for (int q = q0; q < q1 && ok; ++q) chunk_taps<RES, 0, 4>();
+      for (int q = q0; q < q1 && ok; ++q) chunk_taps_any(0, 4, 1);
     } else if (!cond) {
-      if (kp16 == 1) base_small<RES, 1>(); else base_small<RES, 2>();
+      chunk_taps_any(0, kp16, 4 / kp16);
     } else {
-      // conditional channels of chunk 0 (K steps kp16..3), then the remaining chunks
-      if (kp16 == 1) chunk_taps<RES, 1, 4>(); else chunk_taps<RES, 2, 4>();
-      for (int q = 1; q < chunks && ok; ++q) chunk_taps<RES, 0, 4>();
+      chunk_taps_any(kp16, 4, 1);
+      for (int q = 1; q < chunks && ok; ++q) chunk_taps_any(0, 4, 1);
     }
   }
   // base or conditional MMAs of one job into the accumulator at d; `blocks` = column blocks to
@@ -333,7 +388,11 @@ struct MmaIssuer {
     acc = 0u;   // the first K step overwrites the accumulator
     ok = true;
     b_lo = b_base_lo + blk_off_b + (cond ? (uint32_t)base_tiles * kWTile : 0u);   // resident tiles
-    if (resident) phase<true>(cond); else phase<false>(cond);
+    if (kh == 3 && kw == 3) {
+      if (resident) phase3<true>(cond); else phase3<false>(cond);
+    } else {
+      phase_any(cond);
+    }
     return ok;
   }
 };
@@ -349,7 +408,10 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
                      const __grid_constant__ CUtensorMap map_y,
                      const __grid_constant__ TcParams prm) {
   extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  CG_PROF_T(prof_k0);
+  // 1024-byte alignment as an offset from the array, so that every pointer below is still known
+  // to point into shared memory (shared-memory loads and stores, not generic ones)
+  uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
   const LayerDims& L = prm.L;
   const TcPlan& P = prm.P;
   uint8_t* s_a = smem + P.off_a;
@@ -358,10 +420,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   // per-channel constants of this column tile.  Floating point: t, a1, b1, a2, b2.  Integer
   // layers reuse the region: threshold, two multipliers (int32), two offsets (int64).
   float* s_t = (float*)(smem + P.off_consts);
-  float* s_a1 = s_t + NT;
-  float* s_b1 = s_a1 + NT;
-  float* s_a2 = s_b1 + NT;
-  float* s_b2 = s_a2 + NT;
+  float4* s_k = (float4*)(s_t + NT);                       // per channel {a1, b1, a2, b2}
   int* s_qt = (int*)s_t;
   int* s_qm1 = s_qt + NT;
   int* s_qm2 = s_qm1 + NT;
@@ -404,10 +463,10 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     ptx::mbar_init(&sh->w_ready, 1);
     for (int i = 0; i < 4; ++i) {
       ptx::mbar_init(&sh->base_done[i], 1);
-      ptx::mbar_init(&sh->gate_done[i], kEpiThreads);
-      ptx::mbar_init(&sh->p_free[i], kEpiThreads);
+      ptx::mbar_init(&sh->gate_done[i], kGroupWarps);   // one arrival per warp of the group
+      ptx::mbar_init(&sh->p_free[i], kGroupWarps);
       ptx::mbar_init(&sh->cond_done[i], 1);
-      ptx::mbar_init(&sh->r_free[i], kEpiThreads);
+      ptx::mbar_init(&sh->r_free[i], kGroupWarps);
     }
     sh->abort_flag = 0;
     ptx::fence_mbar_init();
@@ -436,7 +495,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         s_qo1[c] = prm.bn.q_off_base[cg_]; s_qo2[c] = prm.bn.q_off_full[cg_];
       } else {
         const ChannelConsts k = fold_channel(prm.bn, prm.delta, L.eps, cg_);
-        s_t[c] = k.t; s_a1[c] = k.a1; s_b1[c] = k.b1; s_a2[c] = k.a2; s_b2[c] = k.b2;
+        s_t[c] = k.t; s_k[c] = make_float4(k.a1, k.b1, k.a2, k.b2);
       }
     }
     ptx::fence_proxy_async();
@@ -445,6 +504,9 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem = sh->tmem_base;
+#ifdef CG_PROF
+  const long long prof_t0 = clock64();
+#endif
 
   if (warp == 0) {
     // ============================================================ patch (A) producer
@@ -453,7 +515,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     // rest for the conditional path, each part with its own cursor -- or, when the layer has a
     // single input chunk, shared: job j's patch is loaded once into slot j % na and serves both
     // paths (the conditional issuer releases it).
-    if (lane == 0 && jobs > 0) {
+    if (jobs > 0) {   // (the whole warp, convergent; lane 0 issues the copies)
       // ring slot and the parity of its "empty" barrier, per ring part
       int as0 = 0, as1 = P.split_a;
       uint32_t apar0 = 1, apar1 = 1;
@@ -466,12 +528,14 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         for (int q = q0; q < q1 && ok; ++q) {
           for (int pl = 0; pl < P.planes && ok; ++pl) {
             const int slot = part ? as1 : as0;
-            ok = wait_bar(cx, &sh->a_empty[slot], part ? apar1 : apar0, 1);
+            ok = wait_bar_warp(cx, &sh->a_empty[slot], part ? apar1 : apar0, 1);
             if (!ok) return;
             const CUtensorMap* mx = pl == 0 ? &map_x : (pl == 1 ? &map_x1 : (pl == 2 ? &map_x2 : &map_x3));
-            ptx::mbar_expect_tx(&sh->a_full[slot], patch_tx);
-            ptx::tma_load_4d(s_a + (size_t)slot * P.patch_bytes, mx, &sh->a_full[slot], q * P.ck, -lead,
-                             h0 - lead, n0);
+            if (lane == 0) {
+              ptx::mbar_expect_tx(&sh->a_full[slot], patch_tx);
+              ptx::tma_load_4d(s_a + (size_t)slot * P.patch_bytes, mx, &sh->a_full[slot], q * P.ck, -lead,
+                               h0 - lead, n0);
+            }
             if (part) { if (++as1 == P.na) { as1 = P.split_a; apar1 ^= 1; } }
             else if (++as0 == hi0) { as0 = 0; apar0 ^= 1; }
           }
@@ -479,14 +543,14 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       };
       const int cond_part = P.split_a ? 1 : 0;
       for (int j = 0; j <= jobs && ok; ++j) {
-        if (j < jobs) load_chunks(j, 0, P.base_chunks, 0);
+        if (j < jobs) { load_chunks(j, 0, P.base_chunks, 0); CG_PROF_EV(j, 0); }
         if (j >= 1 && has_cond && ok && !P.share_a) {
           const int jj = j - 1;
           uint32_t blocks = kAllBlocks;
           if (!dense) {
-            ok = wait_bar(cx, &sh->gate_done[jj % kNP], (jj / kNP) & 1, 2);
+            ok = wait_bar_warp(cx, &sh->gate_done[jj % kNP], (jj / kNP) & 1, 2);
             if (!ok) break;
-            blocks = slot_blocks(sh, jj % kNP);
+            blocks = __shfl_sync(0xffffffffu, slot_blocks(sh, jj % kNP), 0);
           }
           if (blocks) load_chunks(jj, cond_first_chunk, P.chunks, cond_part);
         }
@@ -494,24 +558,28 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     }
   } else if (warp == 2) {
     // ============================================================ weight (B) producer
-    if (lane == 0 && jobs > 0) {
+    if (jobs > 0) {   // (the whole warp, convergent; lane 0 issues the copies)
       if (P.resident) {
         const uint32_t total = (uint32_t)(P.base_tiles + P.cond_tiles) * w_tile_bytes;
-        ptx::mbar_expect_tx(&sh->w_ready, total);
-        for (int bt = 0; bt < P.base_tiles + P.cond_tiles; ++bt)
-          ptx::tma_load_2d(s_b + (size_t)bt * w_tile_bytes, bt < P.base_tiles ? &map_wb : &map_wc,
-                           &sh->w_ready, s_wx[bt], tile_n * NT);
+        if (lane == 0) {
+          ptx::mbar_expect_tx(&sh->w_ready, total);
+          for (int bt = 0; bt < P.base_tiles + P.cond_tiles; ++bt)
+            ptx::tma_load_2d(s_b + (size_t)bt * w_tile_bytes, bt < P.base_tiles ? &map_wb : &map_wc,
+                             &sh->w_ready, s_wx[bt], tile_n * NT);
+        }
       } else {
         int bs = 0;            // ring slot and the parity of its "empty" barrier
         uint32_t bpar = 1;
         bool ok = true;
         auto load_tiles = [&](const CUtensorMap* map, int t0, int n) {
           for (int bt = 0; bt < n && ok; ++bt) {
-            ok = wait_bar(cx, &sh->b_empty[bs], bpar, 3);
+            ok = wait_bar_warp(cx, &sh->b_empty[bs], bpar, 3);
             if (!ok) return;
-            ptx::mbar_expect_tx(&sh->b_full[bs], w_tile_bytes);
-            ptx::tma_load_2d(s_b + (size_t)bs * w_tile_bytes, map, &sh->b_full[bs], s_wx[t0 + bt],
-                             tile_n * NT);
+            if (lane == 0) {
+              ptx::mbar_expect_tx(&sh->b_full[bs], w_tile_bytes);
+              ptx::tma_load_2d(s_b + (size_t)bs * w_tile_bytes, map, &sh->b_full[bs], s_wx[t0 + bt],
+                               tile_n * NT);
+            }
             if (++bs == P.nb) { bs = 0; bpar ^= 1; }
           }
         };
@@ -521,9 +589,9 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
             const int jj = j - 1;
             uint32_t blocks = kAllBlocks;
             if (!dense) {
-              ok = wait_bar(cx, &sh->gate_done[jj % kNP], (jj / kNP) & 1, 4);
+              ok = wait_bar_warp(cx, &sh->gate_done[jj % kNP], (jj / kNP) & 1, 4);
               if (!ok) break;
-              blocks = slot_blocks(sh, jj % kNP);
+              blocks = __shfl_sync(0xffffffffu, slot_blocks(sh, jj % kNP), 0);
             }
             if (blocks) load_tiles(&map_wc, P.base_tiles, P.cond_tiles);
           }
@@ -537,67 +605,85 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     // the per-job bookkeeping of the two paths runs in parallel.
     const bool do_base = warp == 1;
     const bool do_cond = P.issuers == 2 ? warp == 3 : warp == 1;
-    if (lane == 0 && jobs > 0 && (do_base || do_cond)) {
+    if (jobs > 0 && (do_base || do_cond)) {   // (the whole warp, convergent; lane 0 issues)
       MmaIssuer<NT, I8> mi;
+      mi.lead = lane == 0 ? 1u : 0u;
       if (P.split_a) mi.init(sh, cx, s_a, s_b, P, L, do_base ? 0 : P.split_a, do_base ? P.split_a : P.na - P.split_a);
       else mi.init(sh, cx, s_a, s_b, P, L, 0, P.na);
       mi.share = P.share_a != 0;
       mi.release = !(P.share_a && do_base);   // a shared patch is released by the conditional issuer
       bool ok = true;
-      if (P.resident) ok = wait_bar(cx, &sh->w_ready, 0, 6);
-      for (int j = 0; j <= jobs && ok; ++j) {
-        if (do_base && j < jobs) {
+      if (P.resident) ok = wait_bar_warp(cx, &sh->w_ready, 0, 6);
+      // steps 2j (base path of job j) and 2j+1 (conditional path of job j-1), through ONE
+      // inlined copy of the issue loop
+      for (int s = 0; s < 2 * (jobs + 1) && ok; ++s) {
+        const int j = s >> 1;
+        const bool cond = (s & 1) != 0;
+        uint32_t d, blocks = kAllBlocks;
+        int jr;
+        uint64_t* done;
+        if (!cond) {
+          if (!do_base || j >= jobs) continue;
           const int ps = j % kNP;
-          ok = wait_bar(cx, &sh->p_free[ps], ((j / kNP) & 1) ^ 1, 9);
+          ok = wait_bar_warp(cx, &sh->p_free[ps], ((j / kNP) & 1) ^ 1, 9);
           if (!ok) break;
-          ptx::tc_fence_after();
-          ok = mi.run_phase(tmem + (uint32_t)(ps * NT), false, kAllBlocks, j);
-          if (!ok) break;
-          ptx::umma_commit(&sh->base_done[ps]);
-        }
-        if (do_cond && j >= 1) {
+          d = tmem + (uint32_t)(ps * NT); jr = j; done = &sh->base_done[ps];
+          CG_PROF_EV(j, 1);
+        } else {
+          if (!do_cond || j < 1) continue;
           const int jj = j - 1;
           const int rs = jj % kNR;
+          d = tmem + (uint32_t)((kNP + rs) * NT); jr = jj; done = &sh->cond_done[rs];
+          bool run = false;
           if (has_cond) {
-            uint32_t blocks = kAllBlocks;
             if (!dense) {
-              ok = wait_bar(cx, &sh->gate_done[jj % kNP], (jj / kNP) & 1, 10);
+              ok = wait_bar_warp(cx, &sh->gate_done[jj % kNP], (jj / kNP) & 1, 10);
               if (!ok) break;
-              blocks = slot_blocks(sh, jj % kNP);
+              blocks = __shfl_sync(0xffffffffu, slot_blocks(sh, jj % kNP), 0);
             }
             // the R slot's previous user must be done with it even when this job skips the
             // conditional path: otherwise cond_done could run two phases ahead of its waiters
-            ok = wait_bar(cx, &sh->r_free[rs], ((jj / kNR) & 1) ^ 1, 14);
+            ok = wait_bar_warp(cx, &sh->r_free[rs], ((jj / kNR) & 1) ^ 1, 14);
             if (!ok) break;
-            if (blocks) {
-              ptx::tc_fence_after();
-              ok = mi.run_phase(tmem + (uint32_t)((kNP + rs) * NT), true, blocks, jj);
-              if (!ok) break;
-            } else if (P.share_a) {
-              ptx::mbar_arrive(&sh->a_empty[jj % P.na]);   // the job's patch is not needed again
-            }
+            run = blocks != 0u;
+            if (!run && P.share_a && lane == 0) ptx::mbar_arrive(&sh->a_empty[jj % P.na]);   // the job's patch is not needed again
           } else {
-            ok = wait_bar(cx, &sh->r_free[rs], ((jj / kNR) & 1) ^ 1, 15);
+            ok = wait_bar_warp(cx, &sh->r_free[rs], ((jj / kNR) & 1) ^ 1, 15);
             if (!ok) break;
           }
-          ptx::umma_commit(&sh->cond_done[rs]);
+          if (!run) {
+            ptx::umma_commit_if(mi.lead, done);
+            continue;
+          }
+          CG_PROF_EV(jj, 5);
         }
+        ptx::tc_fence_after();
+        ok = mi.run_phase(d, cond, blocks, jr);
+        if (!ok) break;
+        ptx::umma_commit_if(mi.lead, done);
+        CG_PROF_EV(jr, cond ? 6 : 2);
       }
     }
   } else {
-    // ============================================================ epilogue (8 warps)
-    // Warps w and w+4 share a TMEM lane quadrant and split its 32-column blocks between them.
+    // ============================================================ epilogue (16 warps)
+    // Two groups of eight warps work on different jobs at the same time: warps 4-11 evaluate the
+    // gate of job j while warps 12-19 combine and store job j-1 (or earlier).  Within a group,
+    // warp w works on TMEM lane quadrant w % 4 (its 32 pixel rows) and on one half of the tile's
+    // columns.
+    constexpr int CW = NT / 2;                              // columns per warp: 32 or 64
+    const bool gate_group = warp < kEpiWarp0 + kGroupWarps;
     const int quad = warp & 3;
-    const int half = (warp - kEpiWarp0) >> 2;
+    const int cgi = ((warp - kEpiWarp0) >> 2) & 1;         // column half
+    const int col0 = cgi * CW;
     const int row = quad * 32 + lane;                      // TMEM lane = patch row i
-    const int et = threadIdx.x - kEpiThread0;
+    const int ct = threadIdx.x - kEpiThread0 - kGroupThreads;   // thread index within the combine group
     const int n_loc = P.images_mode ? row / P.ip : 0;
     const int rem = P.images_mode ? row - n_loc * P.ip : row;
     const int h_loc = rem / P.wp;
     const int w_out = rem - h_loc * P.wp;
     const uint32_t t_lane = tmem + ((uint32_t)(quad * 32) << 16);
     unsigned long long st_active = 0, st_rows_valid = 0, st_rows_active = 0;
-    unsigned long long st_blocks_run = 0;                  // et == 0
+    unsigned long long st_blocks_run = 0;                  // ct == 0
     bool ok = true;
 
     // gate of job j: P -> mask words (global + stash), block activity flags
@@ -606,83 +692,109 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       ok = wait_bar(cx, &sh->base_done[slot], (j / kNP) & 1, 11);
       if (!ok) return;
       ptx::tc_fence_after();
+      CG_PROF_T(pt0);
+      if (warp == kEpiWarp0) CG_PROF_EV(j, 3);
+      uint32_t r[CW / 32][32];
+#pragma unroll
+      for (int w = 0; w < CW / 32; ++w)
+        ptx::tmem_ld_nowait<32>(t_lane + (uint32_t)(slot * NT + col0 + w * 32), r[w]);
       int n0, h0;
       job_origin(j, n0, h0);
       const int rows_here = P.images_mode ? L.ho : min(P.r, L.ho - h0);
       const bool valid = (w_out < L.wo) && (h_loc < rows_here) && (n_loc < P.ni) && (n0 + n_loc < L.n);
       const long long m = ((long long)(n0 + n_loc) * L.ho + (h0 + h_loc)) * L.wo + w_out;
-      uint32_t my_blocks = 0;
+      uint32_t* g_words = prm.mask + m * L.words + tile_n * kWords + cgi * (CW / 32);
+      uint32_t* s_words = s_mask + (slot * 128 + row) * kWords + cgi * (CW / 32);
+      uint32_t any = 0;
 #pragma unroll
-      for (int cc = 0; cc < kWords / 2; ++cc) {
-        const int cb = cc * 2 + half;
-        uint32_t r[32];
-        ptx::tmem_ld32(t_lane + (uint32_t)(slot * NT + cb * 32), r);
-        uint32_t word = 0;
+      for (int w = 0; w < CW / 32; ++w) {
+        ptx::tmem_ld_wait<32>(r[w]);
+        // four partial words, so that the bit inserts do not form one dependent chain
+        uint32_t pw[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
           if (I8) {
-            const int4 t4 = *(const int4*)(s_qt + cb * 32 + q * 4);
-            word |= ((int)r[q * 4 + 0] >= t4.x ? 1u : 0u) << (q * 4 + 0);
-            word |= ((int)r[q * 4 + 1] >= t4.y ? 1u : 0u) << (q * 4 + 1);
-            word |= ((int)r[q * 4 + 2] >= t4.z ? 1u : 0u) << (q * 4 + 2);
-            word |= ((int)r[q * 4 + 3] >= t4.w ? 1u : 0u) << (q * 4 + 3);
+            const int4 t4 = *(const int4*)(s_qt + col0 + w * 32 + q * 4);
+            pw[q & 3] |= ((int)r[w][q * 4 + 0] >= t4.x ? 1u : 0u) << (q * 4 + 0);
+            pw[q & 3] |= ((int)r[w][q * 4 + 1] >= t4.y ? 1u : 0u) << (q * 4 + 1);
+            pw[q & 3] |= ((int)r[w][q * 4 + 2] >= t4.z ? 1u : 0u) << (q * 4 + 2);
+            pw[q & 3] |= ((int)r[w][q * 4 + 3] >= t4.w ? 1u : 0u) << (q * 4 + 3);
           } else {
-            const float4 t4 = *(const float4*)(s_t + cb * 32 + q * 4);
-            word |= (__uint_as_float(r[q * 4 + 0]) >= t4.x ? 1u : 0u) << (q * 4 + 0);
-            word |= (__uint_as_float(r[q * 4 + 1]) >= t4.y ? 1u : 0u) << (q * 4 + 1);
-            word |= (__uint_as_float(r[q * 4 + 2]) >= t4.z ? 1u : 0u) << (q * 4 + 2);
-            word |= (__uint_as_float(r[q * 4 + 3]) >= t4.w ? 1u : 0u) << (q * 4 + 3);
+            const float4 t4 = *(const float4*)(s_t + col0 + w * 32 + q * 4);
+            pw[q & 3] |= (__uint_as_float(r[w][q * 4 + 0]) >= t4.x ? 1u : 0u) << (q * 4 + 0);
+            pw[q & 3] |= (__uint_as_float(r[w][q * 4 + 1]) >= t4.y ? 1u : 0u) << (q * 4 + 1);
+            pw[q & 3] |= (__uint_as_float(r[w][q * 4 + 2]) >= t4.z ? 1u : 0u) << (q * 4 + 2);
+            pw[q & 3] |= (__uint_as_float(r[w][q * 4 + 3]) >= t4.w ? 1u : 0u) << (q * 4 + 3);
           }
         }
+        uint32_t word = (pw[0] | pw[1]) | (pw[2] | pw[3]);
         if (!valid) word = 0;
-        s_mask[(slot * 128 + row) * kWords + cb] = word;
+        s_words[w] = word;
         st_active += __popc(word);
-        if (word) my_blocks |= 1u << (cb >> 1);
-        if (valid && prm.mask) prm.mask[m * L.words + tile_n * kWords + cb] = word;
+        any |= word;
+        if (valid && prm.mask) g_words[w] = word;
       }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) my_blocks |= __shfl_xor_sync(0xffffffffu, my_blocks, o);
-      if (lane == 0) sh->warp_blk[slot][warp - kEpiWarp0] = my_blocks;
-      if (half == 0) {
+      // 64-channel column blocks with a firing gate, over the warp
+      const uint32_t fired = __ballot_sync(0xffffffffu, any != 0u);
+      if (lane == 0) sh->warp_blk[slot][warp - kEpiWarp0] = fired ? 1u << (col0 >> 6) : 0u;
+      if (cgi == 0) {
         const uint32_t row_valid = __ballot_sync(0xffffffffu, valid);
         if (lane == 0) st_rows_valid += __popc(row_valid);
       }
       ptx::tc_fence_before();
-      ptx::mbar_arrive(&sh->gate_done[slot]);
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&sh->gate_done[slot]);
+      CG_PROF_T(pt1);
+      CG_PROF_ADD(16, pt0, pt1);
+      if (warp == kEpiWarp0) CG_PROF_EV(j, 4);
     };
 
     // combine of job j: y = f(BN1(P)) or f(BN2(P+R)) by mask bit, staged and stored
     auto combine_pass = [&](int j) {
       const int slot = j % kNP, rslot = j % kNR;
-      ok = wait_bar(cx, &sh->gate_done[slot], (j / kNP) & 1, 12);   // every warp's flags and words
+      CG_PROF_T(pc0);
+      ok = wait_bar(cx, &sh->gate_done[slot], (j / kNP) & 1, 12);   // every gate warp's flags and words
       if (!ok) return;
       const uint32_t blocks = !has_cond ? 0u : (dense ? kAllBlocks : slot_blocks(sh, slot));
-      if (half == 0) {
-        uint32_t any = 0;
+      const uint32_t* s_words = s_mask + (slot * 128 + row) * kWords;
+      uint32_t any = 0;                                              // cgi == 0: any gate of the row
+      if (cgi == 0) {
 #pragma unroll
-        for (int cb = 0; cb < kWords; ++cb) any |= s_mask[(slot * 128 + row) * kWords + cb];
+        for (int cb = 0; cb < kWords; ++cb) any |= s_words[cb];
         const uint32_t row_active = __ballot_sync(0xffffffffu, any != 0);
         if (lane == 0) st_rows_active += __popc(row_active);
       }
+      uint32_t words[CW / 32];                                       // the mask bits of this warp's columns
+#pragma unroll
+      for (int w = 0; w < CW / 32; ++w) words[w] = s_words[cgi * (CW / 32) + w];
       ok = wait_bar(cx, &sh->cond_done[rslot], (j / kNR) & 1, 13);
       if (!ok) return;
       ptx::tc_fence_after();
-      if (et == 0) {
+      if (warp == kEpiWarp0 + kGroupWarps) CG_PROF_EV(j, 7);
+      // the warp's columns go through the registers 16 at a time; the loads of the next 16 are
+      // issued before the current ones are stored.  R is read only where the conditional path
+      // ran and a gate of these rows fired.
+      const bool block_ran = (blocks >> (col0 >> 6)) & 1u;
+      uint32_t p[16], rr[16];
+      const uint32_t t_p = t_lane + (uint32_t)(slot * NT + col0), t_r = t_lane + (uint32_t)((kNP + rslot) * NT + col0);
+      bool have_r = block_ran && __ballot_sync(0xffffffffu, (words[0] & 0xffffu) != 0u) != 0u;
+      ptx::tmem_ld_nowait<16>(t_p, p);
+      if (have_r) ptx::tmem_ld_nowait<16>(t_r, rr);
+      if (ct == 0) {
         ptx::tma_store_wait_read();   // the previous store has finished reading the staging tile
         st_blocks_run += __popc(blocks);
       }
-      if (compact && half == 0) {
+      if (compact && cgi == 0) {
         // rows with a firing gate get a slot in this column tile's list (order is arbitrary)
-        uint32_t any = 0;
-#pragma unroll
-        for (int cb = 0; cb < kWords; ++cb) any |= s_mask[(slot * 128 + row) * kWords + cb];
         const uint32_t act = __ballot_sync(0xffffffffu, any != 0);
         uint32_t base = 0;
         if (lane == 0 && act) base = atomicAdd(&prm.ws_counts[tile_n], (uint32_t)__popc(act));
         base = __shfl_sync(0xffffffffu, base, 0);
         sh->row_idx[row] = any ? (int)(base + __popc(act & ((1u << lane) - 1u))) : -1;
       }
-      ptx::named_bar_sync(1, kEpiThreads);
+      CG_PROF_T(pc1);
+      ptx::named_bar_sync(1, kGroupThreads);
+      CG_PROF_T(pc2);
       // residual rows (the shortcut of a residual block, added before the activation)
       const __nv_bfloat16* res_row = nullptr;
       if (!I8 && prm.residual) {
@@ -691,108 +803,125 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         const int rows_here = P.images_mode ? L.ho : min(P.r, L.ho - h0);
         const bool valid = (w_out < L.wo) && (h_loc < rows_here) && (n_loc < P.ni) && (n0 + n_loc < L.n);
         if (valid)
-          res_row = prm.residual + (((long long)(n0 + n_loc) * L.ho + (h0 + h_loc)) * L.wo + w_out) * L.c_out + tile_n * NT;
+          res_row = prm.residual + (((long long)(n0 + n_loc) * L.ho + (h0 + h_loc)) * L.wo + w_out) * L.c_out + tile_n * NT + col0;
       }
-      int list_idx = -1;
-      long long m_row = 0;
+      uint32_t* rec = nullptr;                              // compact mode: this row's record
       if (compact) {
-        list_idx = sh->row_idx[row];
+        const int list_idx = sh->row_idx[row];
         if (list_idx >= 0) {
-          int n0, h0;
-          job_origin(j, n0, h0);
-          m_row = ((long long)(n0 + n_loc) * L.ho + (h0 + h_loc)) * L.wo + w_out;
-          if (half == 0) prm.ws_list[(long long)tile_n * L.m + list_idx] = (uint32_t)m_row;
+          rec = prm.ws_rows + ((long long)tile_n * L.m + list_idx) * (NT + 4);
+          if (cgi == 0) {
+            int n0, h0;
+            job_origin(j, n0, h0);
+            const long long m_row = ((long long)(n0 + n_loc) * L.ho + (h0 + h_loc)) * L.wo + w_out;
+            prm.ws_list[(long long)tile_n * L.m + list_idx] = (uint32_t)m_row;
+          }
+#pragma unroll
+          for (int w = 0; w < CW / 32; ++w) rec[NT + cgi * (CW / 32) + w] = words[w];
         }
       }
 #pragma unroll
-      for (int cc = 0; cc < kWords / 2; ++cc) {
-        const int cb = cc * 2 + half;
-        const uint32_t word = s_mask[(slot * 128 + row) * kWords + cb];
-        uint32_t p[32], rr[32];
-        ptx::tmem_ld32(t_lane + (uint32_t)(slot * NT + cb * 32), p);
-        if (compact && list_idx >= 0) {
-          uint32_t* rec = prm.ws_rows + ((long long)tile_n * L.m + list_idx) * (NT + 4);
+      for (int sc = 0; sc < CW / 16; ++sc) {
+      const int colS = col0 + sc * 16;                     // first column of this sub-chunk
+      const uint32_t bits = words[sc >> 1] >> ((sc & 1) * 16);   // its mask bits
+      ptx::tmem_ld_wait<16>(p);
+      if (have_r) {
+        ptx::tmem_ld_wait<16>(rr);
+      } else {
 #pragma unroll
-          for (int q = 0; q < 8; ++q)
-            *(uint4*)(rec + cb * 32 + q * 4) = make_uint4(p[q * 4], p[q * 4 + 1], p[q * 4 + 2], p[q * 4 + 3]);
-          rec[NT + cb] = word;
-        }
-        const bool have_r = ((blocks >> (cb >> 1)) & 1u) && __ballot_sync(0xffffffffu, word != 0) != 0;
-        if (have_r) {
-          ptx::tmem_ld32(t_lane + (uint32_t)((kNP + rslot) * NT + cb * 32), rr);
-        } else {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) rr[i] = 0u;
-        }
-        if (I8) {
-          // quantised layer: z = acc*mul + off (64-bit), q = (z + 2^(S-1)) >> S, clamp to int8;
-          // 32 channels = 32 bytes = two 16-byte pieces of a 128-channel staging row
-          uint8_t* st = s_y + (size_t)(cb >> 2) * P.stage_rows * 128 + (size_t)row * 128;
-          const long long half_ulp = 1ll << (L.shift - 1);
-          const int lo = L.relu ? 0 : -128;
-#pragma unroll
-          for (int q = 0; q < 2; ++q) {
-            uint32_t packed[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              uint32_t w4 = 0;
-#pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                const int jx = q * 16 + e * 4 + k;
-                const int c = cb * 32 + jx;
-                const bool f = (word >> jx) & 1u;
-                const long long acc = f ? (long long)(int)p[jx] + (long long)(int)rr[jx] : (long long)(int)p[jx];
-                const long long z = acc * (long long)(f ? s_qm2[c] : s_qm1[c]) + (f ? s_qo2[c] : s_qo1[c]);
-                long long qv = (z + half_ulp) >> L.shift;
-                qv = qv < lo ? lo : (qv > 127 ? 127 : qv);
-                w4 |= ((uint32_t)qv & 0xffu) << (8 * k);
-              }
-              packed[e] = w4;
-            }
-            const int c16 = (cb & 3) * 2 + q;
-            *(uint4*)(st + ((c16 ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-          }
-        } else {
-          uint8_t* st = s_y + (size_t)(cb >> 1) * P.stage_rows * 128 + (size_t)row * 128;
-  #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            uint32_t packed[4];
-            uint4 res4 = make_uint4(0u, 0u, 0u, 0u);
-            if (res_row) res4 = *(const uint4*)(res_row + cb * 32 + q * 8);
-            const uint32_t resw[4] = {res4.x, res4.y, res4.z, res4.w};
-  #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int jx = q * 8 + e * 2;
-              const int c = cb * 32 + jx;
-              const float2 a1 = *(const float2*)(s_a1 + c), b1 = *(const float2*)(s_b1 + c);
-              const float2 a2 = *(const float2*)(s_a2 + c), b2 = *(const float2*)(s_b2 + c);
-              const bool f0 = (word >> jx) & 1u, f1 = (word >> (jx + 1)) & 1u;
-              const float p0 = __uint_as_float(p[jx]), p1 = __uint_as_float(p[jx + 1]);
-              // Eq. 1: the full sum P+R where the gate fired, the partial sum elsewhere; then the
-              // batch norm of that path (Section 4) as one multiply and one add
-              const float s0 = f0 ? __fadd_rn(p0, __uint_as_float(rr[jx])) : p0;
-              const float s1 = f1 ? __fadd_rn(p1, __uint_as_float(rr[jx + 1])) : p1;
-              float v0 = __fadd_rn(__fmul_rn(f0 ? a2.x : a1.x, s0), f0 ? b2.x : b1.x);
-              float v1 = __fadd_rn(__fmul_rn(f1 ? a2.y : a1.y, s1), f1 ? b2.y : b1.y);
-              if (res_row) {
-                v0 = __fadd_rn(v0, __uint_as_float(resw[e] << 16));
-                v1 = __fadd_rn(v1, __uint_as_float(resw[e] & 0xffff0000u));
-              }
-              if (L.relu) { v0 = v0 > 0.f ? v0 : 0.f; v1 = v1 > 0.f ? v1 : 0.f; }
-              const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
-              packed[e] = *(const uint32_t*)&h2;
-            }
-            const int c16 = (cb & 1) * 4 + q;
-            *(uint4*)(st + ((c16 ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-          }
-              }
+        for (int i = 0; i < 16; ++i) rr[i] = 0u;
       }
+      if (rec) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          *(uint4*)(rec + colS + q * 4) = make_uint4(p[q * 4], p[q * 4 + 1], p[q * 4 + 2], p[q * 4 + 3]);
+      }
+      if (I8) {
+        // quantised layer: z = acc*mul + off (64-bit), q = (z + 2^(S-1)) >> S, clamp to int8;
+        // 32 channels = 32 bytes = two 16-byte pieces of a 128-channel staging row
+        uint8_t* st = s_y + (size_t)(colS >> 7) * P.stage_rows * 128 + (size_t)row * 128;
+        const long long half_ulp = 1ll << (L.shift - 1);
+        const int lo = L.relu ? 0 : -128;
+        {
+          constexpr int q = 0;
+          uint32_t packed[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            uint32_t w4 = 0;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const int jx = q * 16 + e * 4 + k;
+              const int c = colS + jx;
+              const bool f = (bits >> jx) & 1u;
+              const long long acc = f ? (long long)(int)p[jx] + (long long)(int)rr[jx] : (long long)(int)p[jx];
+              const long long z = acc * (long long)(f ? s_qm2[c] : s_qm1[c]) + (f ? s_qo2[c] : s_qo1[c]);
+              long long qv = (z + half_ulp) >> L.shift;
+              qv = qv < lo ? lo : (qv > 127 ? 127 : qv);
+              w4 |= ((uint32_t)qv & 0xffu) << (8 * k);
+            }
+            packed[e] = w4;
+          }
+          const int c16 = ((colS & 127) >> 4) + q;
+          *(uint4*)(st + ((c16 ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        }
+      } else {
+        uint8_t* st = s_y + (size_t)(colS >> 6) * P.stage_rows * 128 + (size_t)row * 128;
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          float4 k[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) k[i] = s_k[colS + q * 8 + i];
+          uint4 res4 = make_uint4(0u, 0u, 0u, 0u);
+          if (res_row) res4 = *(const uint4*)(res_row + sc * 16 + q * 8);
+          const uint32_t resw[4] = {res4.x, res4.y, res4.z, res4.w};
+          uint32_t packed[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int jx = q * 8 + e * 2;
+            const float4 k0 = k[e * 2], k1 = k[e * 2 + 1];
+            const bool f0 = (bits >> jx) & 1u, f1 = (bits >> (jx + 1)) & 1u;
+            const float p0 = __uint_as_float(p[jx]), p1 = __uint_as_float(p[jx + 1]);
+            // Eq. 1: the full sum P+R where the gate fired, the partial sum elsewhere, each
+            // under the batch norm of its path (Section 4) as one fused multiply-add
+            float v0 = f0 ? fmaf(k0.z, p0 + __uint_as_float(rr[jx]), k0.w) : fmaf(k0.x, p0, k0.y);
+            float v1 = f1 ? fmaf(k1.z, p1 + __uint_as_float(rr[jx + 1]), k1.w) : fmaf(k1.x, p1, k1.y);
+            if (res_row) {
+              v0 += __uint_as_float(resw[e] << 16);
+              v1 += __uint_as_float(resw[e] & 0xffff0000u);
+            }
+            if (L.relu) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
+            packed[e] = *(const uint32_t*)&h2;
+          }
+          const int c16 = ((colS & 63) >> 3) + q;
+          *(uint4*)(st + ((c16 ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        }
+      }
+      if (sc + 1 < CW / 16) {
+        const uint32_t nbits = (words[(sc + 1) >> 1] >> (((sc + 1) & 1) * 16)) & 0xffffu;
+        have_r = block_ran && __ballot_sync(0xffffffffu, nbits != 0u) != 0u;
+        ptx::tmem_ld_nowait<16>(t_p + (sc + 1) * 16, p);
+        if (have_r) ptx::tmem_ld_nowait<16>(t_r + (sc + 1) * 16, rr);
+      }
+      }
+      CG_PROF_T(pcb);
+      CG_PROF_ADD(25, pc2, pcb);
       ptx::tc_fence_before();
-      ptx::mbar_arrive(&sh->p_free[slot]);
-      ptx::mbar_arrive(&sh->r_free[rslot]);
+      __syncwarp();
+      if (lane == 0) {
+        ptx::mbar_arrive(&sh->p_free[slot]);
+        ptx::mbar_arrive(&sh->r_free[rslot]);
+      }
       ptx::fence_proxy_async();
-      ptx::named_bar_sync(1, kEpiThreads);
-      if (et == 0) {
+      CG_PROF_T(pc3);
+      ptx::named_bar_sync(1, kGroupThreads);
+      CG_PROF_T(pc4);
+      CG_PROF_ADD(17, pc0, pc1);
+      CG_PROF_ADD(18, pc1, pc2);
+      CG_PROF_ADD(19, pc2, pc3);
+      CG_PROF_ADD(20, pc3, pc4);
+      if (warp == kEpiWarp0 + kGroupWarps) CG_PROF_EV(j, 8);
+      if (ct == 0) {
         int n0, h0;
         job_origin(j, n0, h0);
         constexpr int kStoreCh = I8 ? 128 : 64;   // channels per 128-byte staging row
@@ -803,24 +932,24 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       }
     };
 
-    for (int j = 0; j < jobs && ok; ++j) {
-      gate_pass(j);
-      if (j >= 1 && ok) combine_pass(j - 1);
+    if (gate_group) {
+      for (int j = 0; j < jobs && ok; ++j) gate_pass(j);
+    } else {
+      for (int j = 0; j < jobs && ok; ++j) combine_pass(j);
+      if (ct == 0) ptx::tma_store_wait_all();
     }
-    if (jobs > 0 && ok) combine_pass(jobs - 1);
-    if (et == 0) ptx::tma_store_wait_all();
 
     // counters of this CTA
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) st_active += __shfl_xor_sync(0xffffffffu, st_active, o);
     if (lane == 0 && ok) {
       atomicAdd(&prm.counters[CNT_ACTIVE], st_active);
-      if (half == 0) {
-        atomicAdd(&prm.counters[CNT_ROWS_TOTAL], st_rows_valid);
-        atomicAdd(&prm.counters[CNT_ROWS_ACTIVE], st_rows_active);
+      if (cgi == 0) {
+        if (gate_group) atomicAdd(&prm.counters[CNT_ROWS_TOTAL], st_rows_valid);
+        else atomicAdd(&prm.counters[CNT_ROWS_ACTIVE], st_rows_active);
       }
     }
-    if (et == 0 && ok) {
+    if (ct == 0 && ok) {
       const unsigned long long k_p = (unsigned long long)taps * L.c_p, k_r = (unsigned long long)taps * L.c_r;
       if (blockIdx.x == 0) atomicAdd(&prm.counters[CNT_CALLS], 1ull);
       atomicAdd(&prm.counters[CNT_TILES_TOTAL], (unsigned long long)kBlocks * jobs);
@@ -830,6 +959,9 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
                 (unsigned long long)kBM * NT * k_p * jobs + (unsigned long long)kBM * 64ull * st_blocks_run * k_r);
     }
   }
+#ifdef CG_PROF
+  if (blockIdx.x == 0 && lane == 0) atomicAdd(&g_prof[warp * 32 + 31], (unsigned long long)(clock64() - prof_t0));
+#endif
   // ---------------------------------------------------------------- teardown
   // (the idle lanes of the single-thread warps wait here, at the hardware barrier)
   ptx::tc_fence_before();
@@ -838,6 +970,12 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     __syncwarp();
     ptx::tmem_dealloc(tmem, 512);
   }
+#ifdef CG_PROF
+  if (blockIdx.x == 0 && threadIdx.x == 32) {
+    atomicAdd(&g_prof[23 * 32 + 0], (unsigned long long)(prof_t0 - prof_k0));
+    atomicAdd(&g_prof[23 * 32 + 1], (unsigned long long)(clock64() - prof_k0));
+  }
+#endif
 }
 
 // ------------------------------------------------------------------------------------------
@@ -894,7 +1032,7 @@ template <int NT>
 __global__ void __launch_bounds__(kCpThreads, 1)
 tc_compact_cond_kernel(const __grid_constant__ CUtensorMap map_wc, const __grid_constant__ CpParams prm) {
   extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
   const LayerDims& L = prm.L;
   const TcPlan& P = prm.P;
   constexpr int kWords = NT / 32;
@@ -1398,5 +1536,18 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
   }
   return (int)cudaGetLastError();
 }
+
+#ifdef CG_PROF
+// Profiling build only: copies the wait-cycle table to the host and clears it.
+extern "C" int cg_prof_read(unsigned long long* host_out) {
+  cudaError_t e = cudaMemcpyFromSymbol(host_out, g_prof, sizeof(g_prof));
+  if (e != cudaSuccess) return (int)e;
+  static unsigned long long zeros[24 * 32];
+  return (int)cudaMemcpyToSymbol(g_prof, zeros, sizeof(g_prof));
+}
+extern "C" int cg_prof_timeline(unsigned long long* host_out) {
+  return (int)cudaMemcpyFromSymbol(host_out, g_tl, sizeof(g_tl));
+}
+#endif
 
 }  // namespace cg
