@@ -49,6 +49,7 @@ constexpr int kBM = 128;            // MMA M: patch rows per job
 constexpr int kSpinLimit = 1 << 21; // try_wait polls before a wait gives up ...
 constexpr long long kWaitCycles = 2000000000ll;   // ... or about one second of SM clocks, whichever is first
 constexpr int kMaxWTiles = 192;     // weight tiles per job, both phases
+constexpr int kStageTiles = 3;      // weight tiles per ring stage (the taps of a 3x3 filter row)
 
 struct TcParams {
   LayerDims L;
@@ -214,6 +215,8 @@ struct MmaIssuer {
   // per phase
   uint32_t d_tmem, idesc, a_grp, b_lo, acc, blk_off_b;
   int a_first, b_held;
+  int st_tile;            // rolled path: tiles used of the current stage
+  uint32_t st_base;       // ... and its first tile
   bool ok;
   bool share, release;   // shared patch ring: slot by job index; release: this issuer frees patches
   uint32_t lead;         // 1 in the lane that issues the tcgen05 instructions (the whole warp runs this code)
@@ -264,19 +267,21 @@ struct MmaIssuer {
     if (!release) return;
     for (int pl = 0; pl < planes; ++pl) ptx::umma_commit_if(lead, &sh->a_empty[a_first + pl]);
   }
-  // Next weight tile.  Resident weights: tiles follow one another from b_lo on (b_lo includes
-  // the column-block offset).  Ring: wait for the slot.
+  // Next three weight tiles (a stage).  Resident weights: tiles follow one another from b_lo
+  // on (b_lo includes the column-block offset).  Ring: the weight producer fills a ring of
+  // stages of up to three consecutive tiles of a phase, one barrier pair per stage, so that the
+  // issuer pays one wait and one commit per filter row instead of per tap.
   template <bool RES>
-  __device__ __forceinline__ uint32_t acquire_b() {
-    if (RES) { const uint32_t b = b_lo; b_lo += kWTile; return b; }
+  __device__ __forceinline__ uint32_t acquire_stage() {
+    if (RES) { const uint32_t b = b_lo; b_lo += kStageTiles * kWTile; return b; }
     ok = ok && wait_bar_warp(cx, &sh->b_full[bs], bpar, 8);
     b_held = bs;
-    const uint32_t b = b_base_lo + (uint32_t)bs * kWTile + blk_off_b;
+    const uint32_t b = b_base_lo + (uint32_t)bs * (kStageTiles * kWTile) + blk_off_b;
     if (++bs == nb) { bs = 0; bpar ^= 1; }
     return b;
   }
   template <bool RES>
-  __device__ __forceinline__ void release_b() {
+  __device__ __forceinline__ void release_stage() {
     if (!RES) ptx::umma_commit_if(lead, &sh->b_empty[b_held]);
   }
   // 3x3: K steps [KS0, KS1) of every tap of the next chunk in the ring, one weight tile per tap
@@ -288,15 +293,16 @@ struct MmaIssuer {
     uint32_t a_row = a_grp + f0, step = f1 - f0;
 #pragma unroll 1
     for (int r = 0; r < 3; ++r) {
+      const uint32_t b_row = acquire_stage<RES>();   // the three taps of a filter row = one stage
+      if (!RES && !ok) return;
 #pragma unroll
       for (int sx = 0; sx < 3; ++sx) {
-        const uint32_t b_t = acquire_b<RES>();
-        if (!RES && !ok) return;
+        const uint32_t b_t = b_row + sx * kWTile;
         const uint32_t a_t = a_row + (sx == 0 ? c0 : sx == 1 ? c1 : c2);
 #pragma unroll
         for (int ks = KS0; ks < KS1; ++ks) mma(a_t + ks * 2, b_t + (ks - KS0) * 2);
-        release_b<RES>();
       }
+      release_stage<RES>();
       a_row += step;
       step = f2 - f1;
     }
@@ -308,39 +314,52 @@ struct MmaIssuer {
     constexpr int TPT = 4 / KP;
     acquire_a();
     if (!ok) return;
-    uint32_t b_t = 0;
+    uint32_t b_row = 0;
 #pragma unroll
     for (int t = 0; t < 9; ++t) {
-      if (t % TPT == 0) b_t = acquire_b<RES>();
+      const int tile = t / TPT;                          // (compile-time: the loop is unrolled)
+      if (t % TPT == 0 && tile % kStageTiles == 0) b_row = acquire_stage<RES>();
       if (!RES && !ok) return;
+      const uint32_t b_t = b_row + (uint32_t)(tile % kStageTiles) * kWTile;
       const uint32_t a_t = a_grp + (t / 3 == 0 ? f0 : t / 3 == 1 ? f1 : f2) + (t % 3 == 0 ? c0 : t % 3 == 1 ? c1 : c2);
 #pragma unroll
       for (int ks = 0; ks < KP; ++ks) mma(a_t + ks * 2, b_t + ((t % TPT) * KP + ks) * 2);
-      if (t % TPT == TPT - 1 || t == 8) release_b<RES>();
+      if ((t % TPT == TPT - 1 && tile % kStageTiles == kStageTiles - 1) || t == 8) release_stage<RES>();
     }
     release_a();
+  }
+  // rolled path: the current tile is done; a stage is released when its last tile is
+  __device__ __forceinline__ void next_tile() {
+    if (++st_tile == kStageTiles) {
+      if (!resident) release_stage<false>();
+      st_tile = 0;
+    }
   }
   // any kernel size (stride 1): K steps [ks0, ks1) of every tap of the next chunk, a weight
   // tile covering `tpt` taps.  Rolled; slow to issue, small in code.
   __device__ __forceinline__ void chunk_taps_any(int ks0, int ks1, int tpt) {
     acquire_a();
     if (!ok) return;
-    int in_tile = 0;
+    int in_tile = 0;          // taps done with the current weight tile
     uint32_t b_t = 0;
     for (int r = 0; r < kh; ++r) {
       const uint32_t a_row = a_grp + (uint32_t)r * row_lo;
       for (int sx = 0; sx < kw; ++sx) {
         if (in_tile == 0) {
-          b_t = resident ? acquire_b<true>() : acquire_b<false>();
-          if (!ok) return;
+          // next tile of the phase: a new stage every kStageTiles tiles
+          if (st_tile == 0) {
+            st_base = resident ? acquire_stage<true>() : acquire_stage<false>();
+            if (!ok) return;
+          }
+          b_t = st_base + (uint32_t)st_tile * kWTile;
         }
         const uint32_t a_t = a_row + (uint32_t)sx * 8u;
         const uint32_t b_k = b_t + (uint32_t)((in_tile * (ks1 - ks0) - ks0) * 2);
         for (int ks = ks0; ks < ks1; ++ks) mma(a_t + ks * 2, b_k + ks * 2);
-        if (++in_tile == tpt) { if (!resident) release_b<false>(); in_tile = 0; }
+        if (++in_tile == tpt) { in_tile = 0; next_tile(); }
       }
     }
-    if (in_tile != 0 && !resident) release_b<false>();
+    if (in_tile != 0) next_tile();
     release_a();
   }
   // Chunks and K ranges of a phase.
@@ -391,7 +410,13 @@ struct MmaIssuer {
     if (kh == 3 && kw == 3) {
       if (resident) phase3<true>(cond); else phase3<false>(cond);
     } else {
+      st_tile = 0;
       phase_any(cond);
+      // a phase's last stage may hold fewer than kStageTiles tiles
+      if (ok && st_tile != 0) {
+        if (!resident) release_stage<false>();
+        st_tile = 0;
+      }
     }
     return ok;
   }
@@ -571,14 +596,17 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         int bs = 0;            // ring slot and the parity of its "empty" barrier
         uint32_t bpar = 1;
         bool ok = true;
+        // the tiles of a phase, in stages of up to kStageTiles tiles on one barrier
         auto load_tiles = [&](const CUtensorMap* map, int t0, int n) {
-          for (int bt = 0; bt < n && ok; ++bt) {
+          for (int g = 0; g < n && ok; g += kStageTiles) {
             ok = wait_bar_warp(cx, &sh->b_empty[bs], bpar, 3);
             if (!ok) return;
+            const int cnt = min(kStageTiles, n - g);
             if (lane == 0) {
-              ptx::mbar_expect_tx(&sh->b_full[bs], w_tile_bytes);
-              ptx::tma_load_2d(s_b + (size_t)bs * w_tile_bytes, map, &sh->b_full[bs], s_wx[t0 + bt],
-                               tile_n * NT);
+              ptx::mbar_expect_tx(&sh->b_full[bs], (uint32_t)cnt * w_tile_bytes);
+              for (int k = 0; k < cnt; ++k)
+                ptx::tma_load_2d(s_b + (size_t)(bs * kStageTiles + k) * w_tile_bytes, map, &sh->b_full[bs],
+                                 s_wx[t0 + g + k], tile_n * NT);
             }
             if (++bs == P.nb) { bs = 0; bpar ^= 1; }
           }
@@ -603,15 +631,22 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     // One thread issues the base path of job j+1 and then the conditional path of job j; when
     // the patch ring is split (resident weights), warp 3 takes the conditional path instead, so
     // the per-job bookkeeping of the two paths runs in parallel.
+    // Conditional phases: one issuer -> warp 1; two issuers -> warp 3, except that with a
+    // shared patch (single-chunk layers: 9 base and 27 conditional MMAs per job) warp 1 also
+    // takes the conditional phase of every third job, which balances the two issue streams
+    // (3 x 9 + 27 = 2 x 27 MMAs per three jobs).
     const bool do_base = warp == 1;
-    const bool do_cond = P.issuers == 2 ? warp == 3 : warp == 1;
-    if (jobs > 0 && (do_base || do_cond)) {   // (the whole warp, convergent; lane 0 issues)
+    auto cond_is_mine = [&](int jj) {
+      if (P.issuers != 2) return warp == 1;
+      if (P.share_a && jj % 3 == 2) return warp == 1;
+      return warp == 3;
+    };
+    if (jobs > 0 && (warp == 1 || P.issuers == 2)) {   // (the whole warp, convergent; lane 0 issues)
       MmaIssuer<NT, I8> mi;
       mi.lead = lane == 0 ? 1u : 0u;
       if (P.split_a) mi.init(sh, cx, s_a, s_b, P, L, do_base ? 0 : P.split_a, do_base ? P.split_a : P.na - P.split_a);
       else mi.init(sh, cx, s_a, s_b, P, L, 0, P.na);
       mi.share = P.share_a != 0;
-      mi.release = !(P.share_a && do_base);   // a shared patch is released by the conditional issuer
       bool ok = true;
       if (P.resident) ok = wait_bar_warp(cx, &sh->w_ready, 0, 6);
       // steps 2j (base path of job j) and 2j+1 (conditional path of job j-1), through ONE
@@ -630,7 +665,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
           d = tmem + (uint32_t)(ps * NT); jr = j; done = &sh->base_done[ps];
           CG_PROF_EV(j, 1);
         } else {
-          if (!do_cond || j < 1) continue;
+          if (j < 1 || !cond_is_mine(j - 1)) continue;
           const int jj = j - 1;
           const int rs = jj % kNR;
           d = tmem + (uint32_t)((kNP + rs) * NT); jr = jj; done = &sh->cond_done[rs];
@@ -658,6 +693,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
           CG_PROF_EV(jj, 5);
         }
         ptx::tc_fence_after();
+        mi.release = !(P.share_a && !cond);   // a shared patch is released by the conditional phase
         ok = mi.run_phase(d, cond, blocks, jr);
         if (!ok) break;
         ptx::umma_commit_if(mi.lead, done);
@@ -1367,14 +1403,17 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
     } else {
       // streamed weights are latency-bound (bytes in flight per SM), so the weight ring gets
       // the shared memory that three patch buffers (stride 1) or one set of planes leave
+      // (nb counts ring stages of kStageTiles tiles: three stages if they fit, else two)
       bool found = false;
-      const int na_want = P.planes == 1 ? 3 : P.planes;
-      for (nb = 8; nb >= 3 && !found; --nb) {
-        if (fixed + nb * w_tile + (size_t)na_want * P.patch_bytes > limit) continue;
-        na = (int)((limit - fixed - nb * w_tile) / P.patch_bytes);
-        if (na > na_max) na = na_max;
-        found = true;
-        break;
+      for (int na_want = P.planes == 1 ? 3 : P.planes; na_want >= (P.planes == 1 ? 2 : P.planes) && !found; --na_want) {
+        for (nb = 3; nb >= 2; --nb) {
+          const size_t ring = (size_t)nb * kStageTiles * w_tile;
+          if (fixed + ring + (size_t)na_want * P.patch_bytes > limit) continue;
+          na = (int)((limit - fixed - ring) / P.patch_bytes);
+          if (na > na_max) na = na_max;
+          found = true;
+          break;
+        }
       }
       if (!found) continue;
     }
@@ -1382,7 +1421,7 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
     if (P.planes == 4) na = na / 4 * 4;
     if (na < P.planes) continue;
     size_t off = 0;
-    P.off_b = (unsigned)off; off += resident ? w_all : nb * w_tile;
+    P.off_b = (unsigned)off; off += resident ? w_all : (size_t)nb * kStageTiles * w_tile;
     P.off_a = (unsigned)off; off += (size_t)na * P.patch_bytes;
     P.off_y = (unsigned)off; off += align_up((size_t)(nt * eb / 128) * P.stage_rows * 128, 1024);
     P.off_consts = (unsigned)off; off += align_up((size_t)8 * nt * 4, 128);

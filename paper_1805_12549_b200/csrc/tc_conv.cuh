@@ -30,7 +30,7 @@ struct TcPlan {
                         // conditional path
   int share_a;          // 2 issuers, 1: one input chunk serves both paths, so job j's patch stays
                         // in slot j % na from its base MMAs until its conditional MMAs are done
-  int nb;               // weight-tile ring depth (0 when the weights are resident)
+  int nb;               // weight ring depth in stages of three tiles (0 when the weights are resident)
   int resident;         // 1: all weight tiles of a column tile stay in shared memory
   int box_h;            // patch box rows: r + 2*pad (rows mode) or h + pad (images mode)
   int box_pixels;       // wp * box_h * ni
