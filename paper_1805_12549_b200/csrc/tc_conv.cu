@@ -27,7 +27,8 @@
 // Weights stay resident in shared memory when they fit, otherwise they stream through a ring.
 //
 // Warp roles: 0 = patch (A) producer, 1 = MMA issuer (owns TMEM), 2 = weight (B) producer,
-// 3 = second MMA issuer (conditional path, resident weights), 4-19 = epilogue.  Every mbarrier wait is bounded; on expiry the CTA records
+// 3 = second MMA issuer (conditional path, resident weights), 4-19 = epilogue, 20 = third MMA
+// issuer (single-chunk layers).  Every mbarrier wait is bounded; on expiry the CTA records
 // CG_ERR_DEVICE_TIMEOUT with the id of the wait and leaves.
 #include <cstring>
 
@@ -38,7 +39,8 @@ namespace cg {
 
 namespace {
 
-constexpr int kThreads = 640;       // 4 single-thread warps + 16 epilogue warps
+constexpr int kThreads = 672;       // 4 producer/issuer warps + 16 epilogue warps + a third MMA issuer
+constexpr int kIssuer3Warp = 20;    // third MMA issuer (single-chunk layers)
 constexpr int kEpiWarp0 = 4;        // warps 0-3: patch producer, MMA issuer, weight producer, second MMA issuer
 constexpr int kEpiThread0 = kEpiWarp0 * 32;
 constexpr int kEpiThreads = 512;
@@ -500,7 +502,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     ptx::prefetch_tensormap(&map_wc); ptx::prefetch_tensormap(&map_y);
   }
   if (warp == 1) ptx::tmem_alloc(&sh->tmem_base, 512);
-  if (warp >= kEpiWarp0) {
+  if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiWarps) {
     const int et = threadIdx.x - kEpiThread0;
     // zero the rows behind the TMA box of every patch buffer: they stand for the right padding
     // of the last patch row and are never written again
@@ -626,22 +628,24 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         }
       }
     }
-  } else if (warp == 1 || warp == 3) {
+  } else if (warp == 1 || warp == 3 || warp == kIssuer3Warp) {
     // ============================================================ MMA issuer(s)
     // One thread issues the base path of job j+1 and then the conditional path of job j; when
     // the patch ring is split (resident weights), warp 3 takes the conditional path instead, so
     // the per-job bookkeeping of the two paths runs in parallel.
-    // Conditional phases: one issuer -> warp 1; two issuers -> warp 3, except that with a
-    // shared patch (single-chunk layers: 9 base and 27 conditional MMAs per job) warp 1 also
-    // takes the conditional phase of every third job, which balances the two issue streams
-    // (3 x 9 + 27 = 2 x 27 MMAs per three jobs).
+    // Conditional phases: one issuer -> warp 1 does both paths; two issuers (resident weights,
+    // several input chunks) -> warp 3; three issuers (resident weights, a single input chunk whose
+    // patch serves both paths: 9 base and 27 conditional MMAs per job) -> warps 3 and 20 take
+    // alternate jobs, so that two conditional phases are issued at the same time and warp 1 is
+    // free to start the base path of the next job as soon as its patch has landed.
     const bool do_base = warp == 1;
     auto cond_is_mine = [&](int jj) {
-      if (P.issuers != 2) return warp == 1;
-      if (P.share_a && jj % 3 == 2) return warp == 1;
-      return warp == 3;
+      if (P.issuers == 1) return warp == 1;
+      if (P.issuers == 2) return warp == 3;
+      return (jj & 1) ? warp == kIssuer3Warp : warp == 3;
     };
-    if (jobs > 0 && (warp == 1 || P.issuers == 2)) {   // (the whole warp, convergent; lane 0 issues)
+    const bool have_role = warp == 1 || (warp == 3 && P.issuers >= 2) || (warp == kIssuer3Warp && P.issuers == 3);
+    if (jobs > 0 && have_role) {   // (the whole warp, convergent; lane 0 issues)
       MmaIssuer<NT, I8> mi;
       mi.lead = lane == 0 ? 1u : 0u;
       if (P.split_a) mi.init(sh, cx, s_a, s_b, P, L, do_base ? 0 : P.split_a, do_base ? P.split_a : P.na - P.split_a);
@@ -1434,7 +1438,7 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
     const bool two = resident && P.cond_tiles > 0 && P.cond_mode != CG_COND_COMPACT;
     P.share_a = (two && P.chunks == 1 && P.planes == 1) ? 1 : 0;
     P.split_a = (two && !P.share_a && na >= 2 * P.planes && (na / 2) % P.planes == 0) ? na / 2 : 0;
-    P.issuers = (P.share_a || P.split_a) ? 2 : 1;
+    P.issuers = P.share_a ? 3 : (P.split_a ? 2 : 1);
     P.smem_bytes = (unsigned)(off + 1024);
     P.valid = 1;
     *plan = P;

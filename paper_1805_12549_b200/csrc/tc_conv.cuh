@@ -24,8 +24,9 @@ struct TcPlan {
   int planes;           // patch buffers per chunk: 1 (stride 1) or 4 (stride 2: the input's
                         // even/odd row x even/odd column sub-images)
   int na;               // patch buffers in the ring
-  int issuers;          // MMA-issuing threads: 1, or 2 (base path / conditional path) when the
-                        // weights are resident
+  int issuers;          // MMA-issuing threads: 1; 2 (base path / conditional path) when the
+                        // weights are resident; 3 (base / conditional of even jobs / of odd jobs)
+                        // when in addition one input chunk serves both paths
   int split_a;          // 2 issuers, > 0: slots [0, split_a) serve the base path and the rest the
                         // conditional path
   int share_a;          // 2 issuers, 1: one input chunk serves both paths, so job j's patch stays
