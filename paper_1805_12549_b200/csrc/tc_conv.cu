@@ -27,8 +27,8 @@
 // Weights stay resident in shared memory when they fit, otherwise they stream through a ring.
 //
 // Warp roles: 0 = patch (A) producer, 1 = MMA issuer (owns TMEM), 2 = weight (B) producer,
-// 3 = second MMA issuer (conditional path, resident weights), 4-19 = epilogue, 20 = third MMA
-// issuer (single-chunk layers).  Every mbarrier wait is bounded; on expiry the CTA records
+// 3 = second MMA issuer (conditional path, resident weights), 4-19 = epilogue; on single-chunk
+// layers warp 2 becomes a third MMA issuer once it has loaded the resident weights.  Every mbarrier wait is bounded; on expiry the CTA records
 // CG_ERR_DEVICE_TIMEOUT with the id of the wait and leaves.
 #include <cstring>
 
@@ -39,8 +39,9 @@ namespace cg {
 
 namespace {
 
-constexpr int kThreads = 672;       // 4 producer/issuer warps + 16 epilogue warps + a third MMA issuer
-constexpr int kIssuer3Warp = 20;    // third MMA issuer (single-chunk layers)
+constexpr int kThreads = 640;       // 4 producer/issuer warps + 16 epilogue warps
+constexpr int kIssuer3Warp = 2;     // third MMA issuer (single-chunk layers): the weight producer's warp, which has
+                                    // nothing to do once resident weights are loaded
 constexpr int kEpiWarp0 = 4;        // warps 0-3: patch producer, MMA issuer, weight producer, second MMA issuer
 constexpr int kEpiThread0 = kEpiWarp0 * 32;
 constexpr int kEpiThreads = 512;
@@ -583,7 +584,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         }
       }
     }
-  } else if (warp == 2) {
+  } else if (warp == 2 && P.issuers != 3) {
     // ============================================================ weight (B) producer
     if (jobs > 0) {   // (the whole warp, convergent; lane 0 issues the copies)
       if (P.resident) {
@@ -635,7 +636,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     // the per-job bookkeeping of the two paths runs in parallel.
     // Conditional phases: one issuer -> warp 1 does both paths; two issuers (resident weights,
     // several input chunks) -> warp 3; three issuers (resident weights, a single input chunk whose
-    // patch serves both paths: 9 base and 27 conditional MMAs per job) -> warps 3 and 20 take
+    // patch serves both paths: 9 base and 27 conditional MMAs per job) -> warps 3 and 2 take
     // alternate jobs, so that two conditional phases are issued at the same time and warp 1 is
     // free to start the base path of the next job as soon as its patch has landed.
     const bool do_base = warp == 1;
@@ -646,6 +647,14 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     };
     const bool have_role = warp == 1 || (warp == 3 && P.issuers >= 2) || (warp == kIssuer3Warp && P.issuers == 3);
     if (jobs > 0 && have_role) {   // (the whole warp, convergent; lane 0 issues)
+      if (warp == kIssuer3Warp && lane == 0) {
+        // (three issuers imply resident weights: this warp loads them once, then issues MMAs)
+        ptx::mbar_expect_tx(&sh->w_ready, (uint32_t)(P.base_tiles + P.cond_tiles) * w_tile_bytes);
+        for (int bt = 0; bt < P.base_tiles + P.cond_tiles; ++bt)
+          ptx::tma_load_2d(s_b + (size_t)bt * w_tile_bytes, bt < P.base_tiles ? &map_wb : &map_wc,
+                           &sh->w_ready, s_wx[bt], tile_n * NT);
+      }
+      __syncwarp();
       MmaIssuer<NT, I8> mi;
       mi.lead = lane == 0 ? 1u : 0u;
       if (P.split_a) mi.init(sh, cx, s_a, s_b, P, L, do_base ? 0 : P.split_a, do_base ? P.split_a : P.na - P.split_a);
