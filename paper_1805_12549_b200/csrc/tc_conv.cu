@@ -106,6 +106,7 @@ struct Shared {
   uint64_t a_full[8], a_empty[8];
   uint64_t b_full[8], b_empty[8];
   uint64_t w_ready;
+  uint64_t setup_done;       // the epilogue warps have zeroed the patch tails
   uint64_t base_done[4], gate_done[4], p_free[4];   // per P accumulator slot
   uint64_t cond_done[4], r_free[4];                 // per R accumulator slot
   uint32_t tmem_base;
@@ -489,6 +490,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     for (int i = 0; i < P.na; ++i) { ptx::mbar_init(&sh->a_full[i], 1); ptx::mbar_init(&sh->a_empty[i], 1); }
     for (int i = 0; i < P.nb; ++i) { ptx::mbar_init(&sh->b_full[i], 1); ptx::mbar_init(&sh->b_empty[i], 1); }
     ptx::mbar_init(&sh->w_ready, 1);
+    ptx::mbar_init(&sh->setup_done, kEpiWarps);
     for (int i = 0; i < 4; ++i) {
       ptx::mbar_init(&sh->base_done[i], 1);
       ptx::mbar_init(&sh->gate_done[i], kGroupWarps);   // one arrival per warp of the group
@@ -503,18 +505,29 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     ptx::prefetch_tensormap(&map_wc); ptx::prefetch_tensormap(&map_y);
   }
   if (warp == 1) ptx::tmem_alloc(&sh->tmem_base, 512);
+  if (warp == 2) {
+    // K coordinate of every weight tile, for the weight loads
+    for (int bt = lane; bt < P.base_tiles + P.cond_tiles; bt += 32)
+      s_wx[bt] = (bt < P.base_tiles ? base_tile(L, P.ck, bt) : cond_tile(L, P.ck, bt - P.base_tiles)).x;
+  }
+  // Only the barriers, the TMEM address and the tile coordinates are needed before the first
+  // copies can be issued: the rest of the set-up (below, epilogue warps) overlaps those copies.
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
   if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiWarps) {
     const int et = threadIdx.x - kEpiThread0;
     // zero the rows behind the TMA box of every patch buffer: they stand for the right padding
-    // of the last patch row and are never written again
+    // of the last patch row and are never written again; the MMA issuers wait for setup_done
     const int tail0 = P.box_pixels * 128, tail1 = P.patch_rows * 128;
     for (int q = 0; q < P.na; ++q) {
       uint8_t* base = s_a + (size_t)q * P.patch_bytes;
       for (int o = tail0 + et * 16; o < tail1; o += kEpiThreads * 16) *(uint4*)(base + o) = make_uint4(0, 0, 0, 0);
     }
-    // K coordinate of every weight tile, for the weight producer
-    for (int bt = et; bt < P.base_tiles + P.cond_tiles; bt += kEpiThreads)
-      s_wx[bt] = (bt < P.base_tiles ? base_tile(L, P.ck, bt) : cond_tile(L, P.ck, bt - P.base_tiles)).x;
+    ptx::fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) ptx::mbar_arrive(&sh->setup_done);
+    // per-channel constants of this column tile, for the epilogue warps themselves
     for (int c = et; c < NT; c += kEpiThreads) {
       const int cg_ = tile_n * NT + c;
       if (I8) {
@@ -526,11 +539,8 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         s_t[c] = k.t; s_k[c] = make_float4(k.a1, k.b1, k.a2, k.b2);
       }
     }
-    ptx::fence_proxy_async();
+    ptx::named_bar_sync(2, kEpiThreads);
   }
-  ptx::tc_fence_before();
-  __syncthreads();
-  ptx::tc_fence_after();
   const uint32_t tmem = sh->tmem_base;
 #ifdef CG_PROF
   const long long prof_t0 = clock64();
@@ -660,8 +670,8 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       if (P.split_a) mi.init(sh, cx, s_a, s_b, P, L, do_base ? 0 : P.split_a, do_base ? P.split_a : P.na - P.split_a);
       else mi.init(sh, cx, s_a, s_b, P, L, 0, P.na);
       mi.share = P.share_a != 0;
-      bool ok = true;
-      if (P.resident) ok = wait_bar_warp(cx, &sh->w_ready, 0, 6);
+      bool ok = wait_bar_warp(cx, &sh->setup_done, 0, 5);
+      if (ok && P.resident) ok = wait_bar_warp(cx, &sh->w_ready, 0, 6);
       // steps 2j (base path of job j) and 2j+1 (conditional path of job j-1), through ONE
       // inlined copy of the issue loop
       for (int s = 0; s < 2 * (jobs + 1) && ok; ++s) {
