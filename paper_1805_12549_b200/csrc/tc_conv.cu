@@ -1573,7 +1573,9 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
     if (e != cudaSuccess) return (int)e;
     attr_set[which] = true;
   }
-  kernels[which]<<<grid, kThreads, P.smem_bytes, stream>>>(ms->x[0], ms->x[1], ms->x[2], ms->x[3], ms->wb,
+  // Every layer asks for the same (maximum) amount of dynamic shared memory: consecutive layer
+  // kernels then never differ in the SM's shared-memory configuration.
+  kernels[which]<<<grid, kThreads, 227 * 1024, stream>>>(ms->x[0], ms->x[1], ms->x[2], ms->x[3], ms->wb,
                                                            ms->wc, ms->y, prm);
   if (compact) {
     // second kernel: gathered conditional path over the listed rows
