@@ -301,6 +301,17 @@ __device__ __forceinline__ void tmem_ld_wait<32>(uint32_t* r) {
                : "memory");
 }
 
+// Programmatic dependent launch.  launch_dependents: the next kernel in the stream may be
+// scheduled once every CTA of this grid has executed this (or exited).  wait: blocks until the
+// kernels this grid depends on have completed and their memory is visible (returns at once when
+// the grid was launched without the attribute).
+__device__ __forceinline__ void grid_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void grid_dependency_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 __device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }

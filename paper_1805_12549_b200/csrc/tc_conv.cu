@@ -438,6 +438,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
                      const __grid_constant__ TcParams prm) {
   extern __shared__ uint8_t smem_raw[];
   CG_PROF_T(prof_k0);
+  ptx::grid_launch_dependents();   // the next kernel in the stream may start as SMs become free
   // 1024-byte alignment as an offset from the array, so that every pointer below is still known
   // to point into shared memory (shared-memory loads and stores, not generic ones)
   uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -515,6 +516,9 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
+  // everything above touched only this CTA's own state; from here on global memory is read and
+  // written, so the kernel that ran before this one in the stream must be complete
+  ptx::grid_dependency_wait();
   if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiWarps) {
     const int et = threadIdx.x - kEpiThread0;
     // zero the rows behind the TMA box of every patch buffer: they stand for the right padding
@@ -1574,9 +1578,26 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
     attr_set[which] = true;
   }
   // Every layer asks for the same (maximum) amount of dynamic shared memory: consecutive layer
-  // kernels then never differ in the SM's shared-memory configuration.
-  kernels[which]<<<grid, kThreads, 227 * 1024, stream>>>(ms->x[0], ms->x[1], ms->x[2], ms->x[3], ms->wb,
-                                                           ms->wc, ms->y, prm);
+  // kernels then never differ in the SM's shared-memory configuration.  The launch is a
+  // programmatic dependent launch: the CTAs of this kernel may start while the last CTAs of the
+  // previous kernel in the stream still run; they set up their barriers and TMEM and then wait
+  // (griddepcontrol.wait) for that kernel to finish before they touch global memory.
+  {
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3((unsigned)kThreads, 1, 1);
+    cfg.dynamicSmemBytes = 227 * 1024;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernels[which], ms->x[0], ms->x[1], ms->x[2], ms->x[3], ms->wb,
+                                             ms->wc, ms->y, prm);
+    if (e != cudaSuccess) return (int)e;
+  }
   if (compact) {
     // second kernel: gathered conditional path over the listed rows
     CpParams cp;
