@@ -29,6 +29,31 @@ METRIC = "gated-conv images/sec at measured gate density"
 UNIT = "images/s"
 
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the layer kernel,
+# from the ncu captures summarised under profiles/.  It is reported only while the kernel sources
+# still hash to what they were when the counters were taken.
+TRAFFIC = {
+    "source_sha": "",
+    "bytes_per_launch": {},
+}
+
+
+def kernel_source_sha():
+    import glob
+    import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_1805_12549_b200", "csrc")
+    for path in sorted(glob.glob(os.path.join(csrc, "*.cu")) + glob.glob(os.path.join(csrc, "*.cuh"))):
+        h.update(open(path, "rb").read())
+    return h.hexdigest()[:16]
+
+
+def measured_traffic(layer_name):
+    if TRAFFIC["source_sha"] != kernel_source_sha():
+        return None
+    return TRAFFIC["bytes_per_launch"].get(layer_name)
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -303,7 +328,8 @@ def run_ours(args):
         roof = {"bound": "tensor", "achieved": dp["gated_tflops"], "peak": peaks["bf16_tflops"],
                 "unit": "TFLOP/s"}
     roof["frac"] = round(roof["achieved"] / roof["peak"], 4)
-    roof["traffic"] = None
+    roof["traffic"] = measured_traffic(dp["layer"])
+    roof["algorithmic_bytes"] = dl.algorithmic_bytes
     roof["kernel"] = f"tc_gated_conv_kernel ({dp['layer']})"
     roof["peak_source"] = f"of {peaks['source']}"
     roof["us_per_launch"] = dp["us"]

@@ -39,15 +39,16 @@ namespace cg {
 
 namespace {
 
-constexpr int kThreads = 640;       // 4 producer/issuer warps + 16 epilogue warps
+constexpr int kThreads = 768;       // 4 producer/issuer warps + 4 gate warps + 16 combine warps
 constexpr int kIssuer3Warp = 2;     // third MMA issuer (single-chunk layers): the weight producer's warp, which has
                                     // nothing to do once resident weights are loaded
 constexpr int kEpiWarp0 = 4;        // warps 0-3: patch producer, MMA issuer, weight producer, second MMA issuer
 constexpr int kEpiThread0 = kEpiWarp0 * 32;
-constexpr int kEpiThreads = 512;
-constexpr int kEpiWarps = kEpiThreads / 32;
-constexpr int kGroupWarps = kEpiWarps / 2;   // gate group, combine group
-constexpr int kGroupThreads = kGroupWarps * 32;
+constexpr int kGateWarps = 4;       // gate group: one warp per TMEM lane quadrant, all columns
+constexpr int kCombWarps = 16;      // combine group: quadrant x quarter of the columns
+constexpr int kEpiWarps = kGateWarps + kCombWarps;
+constexpr int kEpiThreads = kEpiWarps * 32;
+constexpr int kCombThreads = kCombWarps * 32;
 constexpr int kBM = 128;            // MMA M: patch rows per job
 constexpr int kSpinLimit = 1 << 21; // try_wait polls before a wait gives up ...
 constexpr long long kWaitCycles = 2000000000ll;   // ... or about one second of SM clocks, whichever is first
@@ -111,7 +112,7 @@ struct Shared {
   uint64_t cond_done[4], r_free[4];                 // per R accumulator slot
   uint32_t tmem_base;
   uint32_t abort_flag;
-  uint32_t warp_blk[4][8];   // per job slot, per epilogue warp: column blocks with a firing gate
+  uint32_t warp_blk[4][kGateWarps];   // per job slot, per epilogue warp: column blocks with a firing gate
   int row_idx[128];          // compact mode: list slot of each pixel row of the job being combined
 };
 
@@ -123,7 +124,7 @@ struct Ctx {
 #ifdef CG_PROF
 // Profiling build only: cycles that each warp of CTA 0 spent inside every bounded wait
 // ([warp][site]), and the cycles of its role loops ([warp][31]).
-__device__ unsigned long long g_prof[24 * 32];
+__device__ unsigned long long g_prof[25 * 32];
 __device__ unsigned long long g_tl[16 * 16];   // [job][event] clock stamps of CTA 0
 #define CG_PROF_EV(j, ev) \
   do { if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && (j) < 16) g_tl[(j) * 16 + (ev)] = (unsigned long long)clock64(); } while (0)
@@ -183,7 +184,7 @@ __device__ __forceinline__ uint32_t slot_blocks(const Shared* sh, int slot) {
   const volatile uint32_t* w = sh->warp_blk[slot];
   uint32_t b = 0;
 #pragma unroll
-  for (int i = 0; i < kGroupWarps; ++i) b |= w[i];
+  for (int i = 0; i < kGateWarps; ++i) b |= w[i];
   return b;
 }
 
@@ -494,10 +495,10 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     ptx::mbar_init(&sh->setup_done, kEpiWarps);
     for (int i = 0; i < 4; ++i) {
       ptx::mbar_init(&sh->base_done[i], 1);
-      ptx::mbar_init(&sh->gate_done[i], kGroupWarps);   // one arrival per warp of the group
-      ptx::mbar_init(&sh->p_free[i], kGroupWarps);
+      ptx::mbar_init(&sh->gate_done[i], kGateWarps);   // one arrival per warp of the group
+      ptx::mbar_init(&sh->p_free[i], kCombWarps);
       ptx::mbar_init(&sh->cond_done[i], 1);
-      ptx::mbar_init(&sh->r_free[i], kGroupWarps);
+      ptx::mbar_init(&sh->r_free[i], kCombWarps);
     }
     sh->abort_flag = 0;
     ptx::fence_mbar_init();
@@ -728,18 +729,19 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       }
     }
   } else {
-    // ============================================================ epilogue (16 warps)
-    // Two groups of eight warps work on different jobs at the same time: warps 4-11 evaluate the
-    // gate of job j while warps 12-19 combine and store job j-1 (or earlier).  Within a group,
-    // warp w works on TMEM lane quadrant w % 4 (its 32 pixel rows) and on one half of the tile's
-    // columns.
-    constexpr int CW = NT / 2;                              // columns per warp: 32 or 64
-    const bool gate_group = warp < kEpiWarp0 + kGroupWarps;
+    // ============================================================ epilogue (20 warps)
+    // Two groups work on different jobs at the same time: warps 4-7 evaluate the gate of job j
+    // (one warp per TMEM lane quadrant, all columns of the tile), warps 8-23 combine and store job
+    // j-1 or earlier (quadrant x quarter of the columns).  The combine pass is the long one and
+    // is latency-bound -- its shared-memory accesses queue behind the operand fetches of the
+    // MMAs -- so it gets four warps per scheduler.
+    constexpr int CW = NT / 4;                              // columns per combine warp: 16 or 32
+    const bool gate_group = warp < kEpiWarp0 + kGateWarps;
     const int quad = warp & 3;
-    const int cgi = ((warp - kEpiWarp0) >> 2) & 1;         // column half
+    const int cgi = gate_group ? 0 : (warp - kEpiWarp0 - kGateWarps) >> 2;   // column quarter
     const int col0 = cgi * CW;
     const int row = quad * 32 + lane;                      // TMEM lane = patch row i
-    const int ct = threadIdx.x - kEpiThread0 - kGroupThreads;   // thread index within the combine group
+    const int ct = threadIdx.x - kEpiThread0 - kGateWarps * 32;   // thread index within the combine group
     const int n_loc = P.images_mode ? row / P.ip : 0;
     const int rem = P.images_mode ? row - n_loc * P.ip : row;
     const int h_loc = rem / P.wp;
@@ -757,50 +759,50 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       ptx::tc_fence_after();
       CG_PROF_T(pt0);
       if (warp == kEpiWarp0) CG_PROF_EV(j, 3);
-      uint32_t r[CW / 32][32];
-#pragma unroll
-      for (int w = 0; w < CW / 32; ++w)
-        ptx::tmem_ld_nowait<32>(t_lane + (uint32_t)(slot * NT + col0 + w * 32), r[w]);
+      // the tile's columns go through the registers 32 at a time; the next 32 are loaded while
+      // the current ones are compared
+      uint32_t r[2][32];
+      ptx::tmem_ld_nowait<32>(t_lane + (uint32_t)(slot * NT), r[0]);
       int n0, h0;
       job_origin(j, n0, h0);
       const int rows_here = P.images_mode ? L.ho : min(P.r, L.ho - h0);
       const bool valid = (w_out < L.wo) && (h_loc < rows_here) && (n_loc < P.ni) && (n0 + n_loc < L.n);
       const long long m = ((long long)(n0 + n_loc) * L.ho + (h0 + h_loc)) * L.wo + w_out;
-      uint32_t* g_words = prm.mask + m * L.words + tile_n * kWords + cgi * (CW / 32);
-      uint32_t* s_words = s_mask + (slot * 128 + row) * kWords + cgi * (CW / 32);
-      uint32_t any = 0;
+      uint32_t* g_words = prm.mask + m * L.words + tile_n * kWords;
+      uint32_t* s_words = s_mask + (slot * 128 + row) * kWords;
+      uint32_t fired_blocks = 0;
 #pragma unroll
-      for (int w = 0; w < CW / 32; ++w) {
-        ptx::tmem_ld_wait<32>(r[w]);
+      for (int w = 0; w < kWords; ++w) {
+        ptx::tmem_ld_wait<32>(r[w & 1]);
+        if (w + 1 < kWords) ptx::tmem_ld_nowait<32>(t_lane + (uint32_t)(slot * NT + (w + 1) * 32), r[(w + 1) & 1]);
         // four partial words, so that the bit inserts do not form one dependent chain
         uint32_t pw[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
           if (I8) {
-            const int4 t4 = *(const int4*)(s_qt + col0 + w * 32 + q * 4);
-            pw[q & 3] |= ((int)r[w][q * 4 + 0] >= t4.x ? 1u : 0u) << (q * 4 + 0);
-            pw[q & 3] |= ((int)r[w][q * 4 + 1] >= t4.y ? 1u : 0u) << (q * 4 + 1);
-            pw[q & 3] |= ((int)r[w][q * 4 + 2] >= t4.z ? 1u : 0u) << (q * 4 + 2);
-            pw[q & 3] |= ((int)r[w][q * 4 + 3] >= t4.w ? 1u : 0u) << (q * 4 + 3);
+            const int4 t4 = *(const int4*)(s_qt + w * 32 + q * 4);
+            pw[q & 3] |= ((int)r[w & 1][q * 4 + 0] >= t4.x ? 1u : 0u) << (q * 4 + 0);
+            pw[q & 3] |= ((int)r[w & 1][q * 4 + 1] >= t4.y ? 1u : 0u) << (q * 4 + 1);
+            pw[q & 3] |= ((int)r[w & 1][q * 4 + 2] >= t4.z ? 1u : 0u) << (q * 4 + 2);
+            pw[q & 3] |= ((int)r[w & 1][q * 4 + 3] >= t4.w ? 1u : 0u) << (q * 4 + 3);
           } else {
-            const float4 t4 = *(const float4*)(s_t + col0 + w * 32 + q * 4);
-            pw[q & 3] |= (__uint_as_float(r[w][q * 4 + 0]) >= t4.x ? 1u : 0u) << (q * 4 + 0);
-            pw[q & 3] |= (__uint_as_float(r[w][q * 4 + 1]) >= t4.y ? 1u : 0u) << (q * 4 + 1);
-            pw[q & 3] |= (__uint_as_float(r[w][q * 4 + 2]) >= t4.z ? 1u : 0u) << (q * 4 + 2);
-            pw[q & 3] |= (__uint_as_float(r[w][q * 4 + 3]) >= t4.w ? 1u : 0u) << (q * 4 + 3);
+            const float4 t4 = *(const float4*)(s_t + w * 32 + q * 4);
+            pw[q & 3] |= (__uint_as_float(r[w & 1][q * 4 + 0]) >= t4.x ? 1u : 0u) << (q * 4 + 0);
+            pw[q & 3] |= (__uint_as_float(r[w & 1][q * 4 + 1]) >= t4.y ? 1u : 0u) << (q * 4 + 1);
+            pw[q & 3] |= (__uint_as_float(r[w & 1][q * 4 + 2]) >= t4.z ? 1u : 0u) << (q * 4 + 2);
+            pw[q & 3] |= (__uint_as_float(r[w & 1][q * 4 + 3]) >= t4.w ? 1u : 0u) << (q * 4 + 3);
           }
         }
         uint32_t word = (pw[0] | pw[1]) | (pw[2] | pw[3]);
         if (!valid) word = 0;
         s_words[w] = word;
         st_active += __popc(word);
-        any |= word;
         if (valid && prm.mask) g_words[w] = word;
+        if (__ballot_sync(0xffffffffu, word != 0u)) fired_blocks |= 1u << (w >> 1);
       }
       // 64-channel column blocks with a firing gate, over the warp
-      const uint32_t fired = __ballot_sync(0xffffffffu, any != 0u);
-      if (lane == 0) sh->warp_blk[slot][warp - kEpiWarp0] = fired ? 1u << (col0 >> 6) : 0u;
-      if (cgi == 0) {
+      if (lane == 0) sh->warp_blk[slot][warp - kEpiWarp0] = fired_blocks;
+      {
         const uint32_t row_valid = __ballot_sync(0xffffffffu, valid);
         if (lane == 0) st_rows_valid += __popc(row_valid);
       }
@@ -827,20 +829,20 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         const uint32_t row_active = __ballot_sync(0xffffffffu, any != 0);
         if (lane == 0) st_rows_active += __popc(row_active);
       }
-      uint32_t words[CW / 32];                                       // the mask bits of this warp's columns
-#pragma unroll
-      for (int w = 0; w < CW / 32; ++w) words[w] = s_words[cgi * (CW / 32) + w];
+      // the mask word that holds this warp's 16 or 32 columns, and their position in it
+      const uint32_t wv = s_words[col0 >> 5];
+      const int wshift = col0 & 31;
       ok = wait_bar(cx, &sh->cond_done[rslot], (j / kNR) & 1, 13);
       if (!ok) return;
       ptx::tc_fence_after();
-      if (warp == kEpiWarp0 + kGroupWarps) CG_PROF_EV(j, 7);
+      if (warp == kEpiWarp0 + kGateWarps) CG_PROF_EV(j, 7);
       // the warp's columns go through the registers 16 at a time; the loads of the next 16 are
       // issued before the current ones are stored.  R is read only where the conditional path
       // ran and a gate of these rows fired.
       const bool block_ran = (blocks >> (col0 >> 6)) & 1u;
       uint32_t p[16], rr[16];
       const uint32_t t_p = t_lane + (uint32_t)(slot * NT + col0), t_r = t_lane + (uint32_t)((kNP + rslot) * NT + col0);
-      bool have_r = block_ran && __ballot_sync(0xffffffffu, (words[0] & 0xffffu) != 0u) != 0u;
+      bool have_r = block_ran && __ballot_sync(0xffffffffu, ((wv >> wshift) & 0xffffu) != 0u) != 0u;
       ptx::tmem_ld_nowait<16>(t_p, p);
       if (have_r) ptx::tmem_ld_nowait<16>(t_r, rr);
       if (ct == 0) {
@@ -856,7 +858,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         sh->row_idx[row] = any ? (int)(base + __popc(act & ((1u << lane) - 1u))) : -1;
       }
       CG_PROF_T(pc1);
-      ptx::named_bar_sync(1, kGroupThreads);
+      ptx::named_bar_sync(1, kCombThreads);
       CG_PROF_T(pc2);
       // residual rows (the shortcut of a residual block, added before the activation)
       const __nv_bfloat16* res_row = nullptr;
@@ -879,14 +881,13 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
             const long long m_row = ((long long)(n0 + n_loc) * L.ho + (h0 + h_loc)) * L.wo + w_out;
             prm.ws_list[(long long)tile_n * L.m + list_idx] = (uint32_t)m_row;
           }
-#pragma unroll
-          for (int w = 0; w < CW / 32; ++w) rec[NT + cgi * (CW / 32) + w] = words[w];
+          if (wshift == 0) rec[NT + (col0 >> 5)] = wv;
         }
       }
 #pragma unroll
       for (int sc = 0; sc < CW / 16; ++sc) {
       const int colS = col0 + sc * 16;                     // first column of this sub-chunk
-      const uint32_t bits = words[sc >> 1] >> ((sc & 1) * 16);   // its mask bits
+      const uint32_t bits = wv >> (wshift + sc * 16);          // its mask bits
       ptx::tmem_ld_wait<16>(p);
       if (have_r) {
         ptx::tmem_ld_wait<16>(rr);
@@ -961,7 +962,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         }
       }
       if (sc + 1 < CW / 16) {
-        const uint32_t nbits = (words[(sc + 1) >> 1] >> (((sc + 1) & 1) * 16)) & 0xffffu;
+        const uint32_t nbits = (wv >> (wshift + (sc + 1) * 16)) & 0xffffu;
         have_r = block_ran && __ballot_sync(0xffffffffu, nbits != 0u) != 0u;
         ptx::tmem_ld_nowait<16>(t_p + (sc + 1) * 16, p);
         if (have_r) ptx::tmem_ld_nowait<16>(t_r + (sc + 1) * 16, rr);
@@ -977,13 +978,13 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       }
       ptx::fence_proxy_async();
       CG_PROF_T(pc3);
-      ptx::named_bar_sync(1, kGroupThreads);
+      ptx::named_bar_sync(1, kCombThreads);
       CG_PROF_T(pc4);
       CG_PROF_ADD(17, pc0, pc1);
       CG_PROF_ADD(18, pc1, pc2);
       CG_PROF_ADD(19, pc2, pc3);
       CG_PROF_ADD(20, pc3, pc4);
-      if (warp == kEpiWarp0 + kGroupWarps) CG_PROF_EV(j, 8);
+      if (warp == kEpiWarp0 + kGateWarps) CG_PROF_EV(j, 8);
       if (ct == 0) {
         int n0, h0;
         job_origin(j, n0, h0);
@@ -1035,8 +1036,8 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   }
 #ifdef CG_PROF
   if (blockIdx.x == 0 && threadIdx.x == 32) {
-    atomicAdd(&g_prof[23 * 32 + 0], (unsigned long long)(prof_t0 - prof_k0));
-    atomicAdd(&g_prof[23 * 32 + 1], (unsigned long long)(clock64() - prof_k0));
+    atomicAdd(&g_prof[24 * 32 + 0], (unsigned long long)(prof_t0 - prof_k0));
+    atomicAdd(&g_prof[24 * 32 + 1], (unsigned long long)(clock64() - prof_k0));
   }
 #endif
 }
@@ -1627,7 +1628,7 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
 extern "C" int cg_prof_read(unsigned long long* host_out) {
   cudaError_t e = cudaMemcpyFromSymbol(host_out, g_prof, sizeof(g_prof));
   if (e != cudaSuccess) return (int)e;
-  static unsigned long long zeros[24 * 32];
+  static unsigned long long zeros[25 * 32];
   return (int)cudaMemcpyToSymbol(g_prof, zeros, sizeof(g_prof));
 }
 extern "C" int cg_prof_timeline(unsigned long long* host_out) {
