@@ -20,15 +20,19 @@
 //
 // The CTA is persistent (one per SM) and software-pipelined over its jobs:
 //   MMA issue order      base(0) | base(1) cond(0) | base(2) cond(1) | ...
-//   epilogue order       gate(0) | gate(1) combine(0) | gate(2) combine(1) | ...
+//   gate group           gate(0) | gate(1) | gate(2) | ...
+//   combine group        combine(0) | combine(1) | ...          (each as soon as its inputs exist)
 // so the tensor pipe works on the next tile's base path while the gate of the current tile is
 // being evaluated.  TMEM (512 columns) holds a ring of P accumulators and a ring of R
 // accumulators: 4 + 4 at NT = 64, 3 + 1 at NT = 128, so the issuer can run ahead of the epilogue.
-// Weights stay resident in shared memory when they fit, otherwise they stream through a ring.
+// Weights stay resident in shared memory when they fit, otherwise they stream through a ring of
+// stages of three tiles (the taps of a filter row).
 //
 // Warp roles: 0 = patch (A) producer, 1 = MMA issuer (owns TMEM), 2 = weight (B) producer,
-// 3 = second MMA issuer (conditional path, resident weights), 4-19 = epilogue; on single-chunk
-// layers warp 2 becomes a third MMA issuer once it has loaded the resident weights.  Every mbarrier wait is bounded; on expiry the CTA records
+// 3 = second MMA issuer (conditional path, resident weights), 4-7 = gate group, 8-23 = combine
+// group; on single-chunk layers warp 2 becomes a third MMA issuer once it has loaded the
+// resident weights.  The producer and issuer warps run convergently and lane 0 issues the
+// copies and MMAs.  Every mbarrier wait is bounded; on expiry the CTA records
 // CG_ERR_DEVICE_TIMEOUT with the id of the wait and leaves.
 #include <cstring>
 
@@ -1027,7 +1031,6 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   if (blockIdx.x == 0 && lane == 0) atomicAdd(&g_prof[warp * 32 + 31], (unsigned long long)(clock64() - prof_t0));
 #endif
   // ---------------------------------------------------------------- teardown
-  // (the idle lanes of the single-thread warps wait here, at the hardware barrier)
   ptx::tc_fence_before();
   __syncthreads();
   if (warp == 1) {
