@@ -119,21 +119,27 @@ def test_two_calls_accumulate_and_are_deterministic():
     g.close()
 
 
-@pytest.mark.parametrize("layer", ["c64@56", "c128@28", "c256@14", "c512@7"])
-def test_full_size_layers_on_sampled_images(layer):
-    """Batch-64 ImageNet ResNet-18 layer shapes in the configuration the benchmark times;
-    images are independent, so the oracle checks a sample of them one by one."""
+@pytest.mark.parametrize("workload,layer", [
+    ("imagenet", "c64@56"), ("imagenet", "c128@28"), ("imagenet", "c256@14"), ("imagenet", "c512@7"),
+    ("imagenet", "c64to128@56s2"), ("imagenet", "c128to256@28s2"), ("imagenet", "c256to512@14s2"),
+    ("cifar", "c64@32"), ("cifar", "c128@16"), ("cifar", "c256@8"), ("cifar", "c512@4")])
+def test_full_size_layers_on_sampled_images(workload, layer):
+    """Every layer shape of the two benchmark workloads (batch-64 ImageNet and batch-256 CIFAR
+    ResNet-18 layers) in the configuration the benchmark times; images are independent, so the
+    oracle checks a sample of them one by one."""
     from paper_1805_12549_b200 import synth
-    ls = {l.name: l for l in synth.imagenet_resnet18_layers(64, 4)}[layer]
-    s = O.Shape(ls.n, ls.hw, ls.hw, ls.c_in, ls.c_out, groups=4)
+    layers = synth.imagenet_resnet18_layers(64, 4) if workload == "imagenet" else synth.cifar_resnet18_layers(256, 4)
+    ls = {l.name: l for l in layers}[layer]
+    s = O.Shape(ls.n, ls.hw, ls.hw, ls.c_in, ls.c_out, stride=ls.stride, groups=4)
     c = K.make_float_case("full", s, "bf16", density=0.3, calib_images=2)
     g = K.GpuCase(c, algo=TENSOR)
+    assert g.conv.uses_tensor_cores
     y, mask, st = g.run()
     g.close()
     assert abs(st.density - 0.3) < 0.04
     words = s.words
     per_img = s.ho * s.wo
-    for n in (0, 17, 40, 63):
+    for n in sorted({0, s.n // 4 + 1, (5 * s.n) // 8, s.n - 1}):
         s1 = O.Shape(**{**s.__dict__, "n": 1})
         c1 = K.Case(c.name, s1, c.dtype, c.x[n:n + 1], c.wb, c.wc, c.bn, c.delta)
         ref = K.run_oracle(c1)
