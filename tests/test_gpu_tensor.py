@@ -232,3 +232,38 @@ def test_residual_input_on_the_tensor_path(s, why):
     c0 = K.make_float_case("tcres", s, "bf16", density=0.3, residual=False)
     ref0 = K.run_oracle(c0)
     assert np.abs(ref.y.astype(np.float64) - ref0.y.astype(np.float64)).max() > 0.1
+
+
+def test_dependent_layers_back_to_back_on_one_stream():
+    """Two layers chained on one stream without any host synchronisation: the second reads the
+    first one's output.  Each call is a programmatic dependent launch (its blocks may start while
+    the previous kernel drains), so this checks that no block touches global memory before the
+    previous kernel has finished: the result must be bit-identical to the same chain run with a
+    device synchronisation after every call, on every one of several repetitions."""
+    import torch
+    s = O.Shape(24, 28, 28, 128, 128, groups=4)
+    c = K.make_float_case("chain", s, "bf16", density=0.3, calib_images=2)
+    g1 = K.GpuCase(c, algo=TENSOR)
+    g2 = K.GpuCase(c, algo=TENSOR)
+    assert g1.conv.uses_tensor_cores
+
+    def chain(sync):
+        g1.y.fill_(0); g2.y.fill_(0); g2.mask.fill_(-1)
+        torch.cuda.synchronize()
+        for _ in range(3):     # the last pass decides; earlier passes keep the queue full
+            g1.conv.forward(g1.x, g1.wb, g1.wc, g1.bn, g1.delta, g1.y, g1.mask, None)
+            if sync:
+                torch.cuda.synchronize()
+            g2.conv.forward(g1.y, g2.wb, g2.wc, g2.bn, g2.delta, g2.y, g2.mask, None)
+            if sync:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        return g2.y.clone(), g2.mask.clone()
+
+    y_ref, m_ref = chain(sync=True)
+    for _ in range(5):
+        y, m = chain(sync=False)
+        assert torch.equal(m, m_ref)
+        assert torch.equal(y.view(torch.int16), y_ref.view(torch.int16))
+    assert g1.conv.stats().device_status == 0 and g2.conv.stats().device_status == 0
+    g1.close(); g2.close()
