@@ -47,7 +47,10 @@ typedef enum { CG_F32 = 0, CG_BF16 = 1, CG_I8 = 2 } cg_dtype;
 typedef enum {
   CG_ALGO_AUTO = 0,   /* tensor-core path when the layer qualifies, else the direct path */
   CG_ALGO_DIRECT = 1, /* CUDA-core direct convolution: any shape, sums in the order (r,s,c_in) */
-  CG_ALGO_TENSOR = 2  /* tcgen05 implicit GEMM; CG_ERR_UNSUPPORTED at create if not eligible */
+  CG_ALGO_TENSOR = 2, /* tcgen05 implicit GEMM; CG_ERR_UNSUPPORTED at create if not eligible */
+  CG_ALGO_TENSOR_ROWS = 3,     /* the pixel-major tcgen05 kernel only (pixels on the MMA's M side) */
+  CG_ALGO_TENSOR_CHANNELS = 4  /* the channel-major tcgen05 kernel only (output channels on the M side).
+                                  AUTO and TENSOR pick between the two by layer shape. */
 } cg_algo;
 
 /* How the tensor-core path treats the conditional path (Eq. 1, second case). */
@@ -189,6 +192,20 @@ int cg_conv_launches_per_forward(cg_conv_t h);
 
 /* 1 if the tensor-core path runs this layer, 0 if the direct path does. */
 int cg_conv_uses_tensor_cores(cg_conv_t h);
+
+/* Which kernel family runs this layer (Section 3.1's two convolutions, gate and combine fused
+ * in all three): the CUDA-core direct kernels, the tcgen05 kernel with pixels on the MMA's M
+ * side, or the tcgen05 kernel with output channels on the M side and pixels on the N side. */
+typedef enum {
+  CG_KERNEL_DIRECT = 0,
+  CG_KERNEL_TENSOR_PIXEL_MAJOR = 1,
+  CG_KERNEL_TENSOR_CHANNEL_MAJOR = 2
+} cg_kernel_id;
+int cg_conv_kernel_id(cg_conv_t h);
+
+/* Writes a one-line description of the tiling chosen for this layer (tile sizes, K stages, ring
+ * depth, grid) into buf; returns the length snprintf would have written, -1 on a NULL argument. */
+int cg_conv_plan_string(cg_conv_t h, char* buf, size_t len);
 
 void cg_conv_destroy(cg_conv_t h);
 

@@ -16,13 +16,14 @@ from . import build as _build
 
 CG_OK = 0
 CG_F32, CG_BF16, CG_I8 = 0, 1, 2
-CG_ALGO_AUTO, CG_ALGO_DIRECT, CG_ALGO_TENSOR = 0, 1, 2
+CG_ALGO_AUTO, CG_ALGO_DIRECT, CG_ALGO_TENSOR, CG_ALGO_TENSOR_ROWS, CG_ALGO_TENSOR_CHANNELS = 0, 1, 2, 3, 4
+CG_KERNEL_DIRECT, CG_KERNEL_TENSOR_PIXEL_MAJOR, CG_KERNEL_TENSOR_CHANNEL_MAJOR = 0, 1, 2
 CG_COND_AUTO, CG_COND_DENSE, CG_COND_SKIP_TILES, CG_COND_COMPACT = 0, 1, 2, 3
 
 EXPORTS = ("cg_conv_create", "cg_conv_workspace_bytes", "cg_conv_forward",
            "cg_conv_host_staging_bytes", "cg_conv_forward_host", "cg_conv_partial_sums",
            "cg_conv_stats", "cg_conv_launches_per_forward", "cg_conv_uses_tensor_cores",
-           "cg_conv_destroy", "cg_status_string", "cg_conv_forward_static")
+           "cg_conv_kernel_id", "cg_conv_plan_string", "cg_conv_destroy", "cg_status_string", "cg_conv_forward_static")
 
 
 class CgConvDesc(C.Structure):
@@ -81,6 +82,10 @@ def lib():
         L.cg_conv_launches_per_forward.argtypes = [C.c_void_p]
         L.cg_conv_uses_tensor_cores.restype = C.c_int
         L.cg_conv_uses_tensor_cores.argtypes = [C.c_void_p]
+        L.cg_conv_kernel_id.restype = C.c_int
+        L.cg_conv_kernel_id.argtypes = [C.c_void_p]
+        L.cg_conv_plan_string.restype = C.c_int
+        L.cg_conv_plan_string.argtypes = [C.c_void_p, C.c_char_p, C.c_size_t]
         L.cg_conv_destroy.restype = None
         L.cg_conv_destroy.argtypes = [C.c_void_p]
         L.cg_conv_forward_static.restype = C.c_int
@@ -220,6 +225,16 @@ def cg_conv_uses_tensor_cores(h) -> bool:
     return bool(lib().cg_conv_uses_tensor_cores(h))
 
 
+def cg_conv_kernel_id(h) -> int:
+    return int(lib().cg_conv_kernel_id(h))
+
+
+def cg_conv_plan_string(h) -> str:
+    buf = C.create_string_buffer(512)
+    lib().cg_conv_plan_string(h, buf, len(buf))
+    return buf.value.decode()
+
+
 class GatedConv:
     """Convenience owner of one handle plus its workspace (still argument marshalling only)."""
 
@@ -259,6 +274,14 @@ class GatedConv:
     @property
     def uses_tensor_cores(self):
         return cg_conv_uses_tensor_cores(self.handle)
+
+    @property
+    def kernel_id(self):
+        return cg_conv_kernel_id(self.handle)
+
+    @property
+    def plan(self):
+        return cg_conv_plan_string(self.handle)
 
     def close(self):
         if self.handle is not None:

@@ -6,6 +6,7 @@
 
 #include "common.cuh"
 #include "tc_conv.cuh"
+#include "tc2_conv.cuh"
 
 struct cg_conv_s {
   cg_conv_desc desc;
@@ -15,6 +16,9 @@ struct cg_conv_s {
   int device;
   unsigned long long* counters;   // device, cg::CNT_SLOTS entries
   cg::TcMaps maps;                // tensor maps cached for the last set of pointers
+  int use_tc2;                    // channel-major tensor-core kernel (tc2_conv.cu)
+  cg::Tc2Plan plan2;
+  cg::Tc2Maps maps2;
 };
 
 namespace {
@@ -37,7 +41,7 @@ cg_status check_desc(const cg_conv_desc* d) {
   if (d->in_dtype == CG_I8 && (d->requant_shift < 1 || d->requant_shift > 31)) return CG_ERR_INVALID_ARG;
   if (d->in_dtype == CG_I8 && d->has_residual) return CG_ERR_INVALID_ARG;
   if (!(d->bn_eps >= 0.f)) return CG_ERR_INVALID_ARG;
-  if (d->algo < CG_ALGO_AUTO || d->algo > CG_ALGO_TENSOR) return CG_ERR_INVALID_ARG;
+  if (d->algo < CG_ALGO_AUTO || d->algo > CG_ALGO_TENSOR_CHANNELS) return CG_ERR_INVALID_ARG;
   if (d->cond_mode < CG_COND_AUTO || d->cond_mode > CG_COND_COMPACT) return CG_ERR_INVALID_ARG;
   if (d->grouping != 0 && d->grouping != 1) return CG_ERR_INVALID_ARG;
   if (d->grouping && d->c_out % d->groups != 0) return CG_ERR_INVALID_ARG;
@@ -105,16 +109,34 @@ cg_status cg_conv_create(cg_conv_t* out, const cg_conv_desc* desc) {
   h->L = make_dims(*desc);
   h->counters = nullptr;
   std::memset(&h->maps, 0, sizeof(h->maps));
+  std::memset(&h->maps2, 0, sizeof(h->maps2));
+  // (which kernels apply is decided before the device is needed, so that an ineligible layer is
+  // reported as such on any machine)
+  const bool have_device = cudaGetDevice(&h->device) == cudaSuccess;
+  int sms = 0;
+  if (!have_device || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess || sms <= 0) sms = 148;
   // the channel-wise gate needs every partial sum of an image before any conditional path: it
   // runs on the direct kernels
-  const bool tc_ok = !(desc->channel_tau > 0.f) &&
-                     cg::tc_plan(h->L, desc->in_dtype, desc->cond_mode, &h->plan);
-  if (desc->algo == CG_ALGO_TENSOR && !tc_ok) { delete h; return CG_ERR_UNSUPPORTED; }
-  h->use_tc = (desc->algo != CG_ALGO_DIRECT) && tc_ok;
-  if (cudaGetDevice(&h->device) != cudaSuccess) { delete h; return CG_ERR_CUDA; }
+  const bool want_tc = desc->algo != CG_ALGO_DIRECT && !(desc->channel_tau > 0.f);
+  // Two tensor-core kernels.  Measured on B200 (batch 64-256 ResNet-18 shapes), the channel-major
+  // kernel is the faster one for 128 output channels and for 256 channels on 8x8 images, where the
+  // pixel-major kernel's whole-image tiles are half padding; elsewhere the pixel-major kernel wins.
+  // Each also takes the layers only it can run.
+  const bool prefer2 = h->L.c_out == 128 || (h->L.c_out == 256 && h->L.ho * h->L.wo <= 64);
+  const bool allow1 = desc->algo != CG_ALGO_TENSOR_CHANNELS, allow2 = desc->algo != CG_ALGO_TENSOR_ROWS;
+  bool ok1 = false, ok2 = false;
+  if (want_tc && allow2 && (prefer2 || !allow1)) ok2 = cg::tc2_plan(h->L, desc->in_dtype, desc->cond_mode, sms, &h->plan2);
+  if (want_tc && allow1 && !ok2) ok1 = cg::tc_plan(h->L, desc->in_dtype, desc->cond_mode, &h->plan);
+  if (want_tc && allow2 && !ok1 && !ok2) ok2 = cg::tc2_plan(h->L, desc->in_dtype, desc->cond_mode, sms, &h->plan2);
+  h->use_tc2 = ok2;
+  const bool tc_ok = ok1;
+  const bool must_tc = desc->algo >= CG_ALGO_TENSOR;
+  if (must_tc && !tc_ok && !h->use_tc2) { delete h; return CG_ERR_UNSUPPORTED; }
+  if (!have_device) { delete h; return CG_ERR_CUDA; }
+  h->use_tc = tc_ok || h->use_tc2;
   if (h->use_tc && !cg::tc_device_ok(h->device)) {
-    if (desc->algo == CG_ALGO_TENSOR) { delete h; return CG_ERR_UNSUPPORTED; }
-    h->use_tc = 0;
+    if (must_tc) { delete h; return CG_ERR_UNSUPPORTED; }
+    h->use_tc = 0; h->use_tc2 = 0;
   }
   if (cudaMalloc(&h->counters, cg::CNT_SLOTS * sizeof(unsigned long long)) != cudaSuccess) {
     delete h; return CG_ERR_CUDA;
@@ -135,16 +157,40 @@ void cg_conv_destroy(cg_conv_t h) {
 size_t cg_conv_workspace_bytes(cg_conv_t h) {
   if (!h) return 0;
   if (h->L.channel_tau > 0.f) return cg::channel_gate_workspace_bytes(h->L);
-  return h->use_tc ? cg::tc_workspace_bytes(h->L, h->plan) : 0;
+  return (h->use_tc && !h->use_tc2) ? cg::tc_workspace_bytes(h->L, h->plan) : 0;
 }
 
 int cg_conv_launches_per_forward(cg_conv_t h) {
   if (!h) return 0;
   if (h->L.channel_tau > 0.f) return 2;
-  return (h->use_tc && h->plan.cond_mode == CG_COND_COMPACT) ? 2 : 1;
+  return (h->use_tc && !h->use_tc2 && h->plan.cond_mode == CG_COND_COMPACT) ? 2 : 1;
 }
 
 int cg_conv_uses_tensor_cores(cg_conv_t h) { return h ? h->use_tc : 0; }
+
+int cg_conv_plan_string(cg_conv_t h, char* buf, size_t len) {
+  if (!h || !buf || len == 0) return -1;
+  if (h->use_tc2) {
+    const cg::Tc2Plan& P = h->plan2;
+    return std::snprintf(buf, len,
+                         "channel-major tcgen05: %d channel tile(s) x %d pixel tiles of %d sub-tile(s) x %d stacked rows "
+                         "(%d pixels, MMA N=%d), %d K stages (%d base), weight ring %d, lead %d, grid %d",
+                         P.tiles_c, P.jobs_m, P.nsub, P.r, P.np, P.nmma, P.ns, P.nb, P.ring, P.lead, P.grid);
+  }
+  if (h->use_tc) {
+    const cg::TcPlan& P = h->plan;
+    return std::snprintf(buf, len,
+                         "pixel-major tcgen05: %d row tiles x %d column tiles of %d, %s weights, %d patch buffers, %d issuer(s)",
+                         P.tiles_m, P.tiles_n, P.nt, P.resident ? "resident" : "streamed", P.na, P.issuers);
+  }
+  return std::snprintf(buf, len, "direct CUDA-core kernels");
+}
+
+int cg_conv_kernel_id(cg_conv_t h) {
+  if (!h) return -1;
+  if (h->L.channel_tau > 0.f) return CG_KERNEL_DIRECT;
+  return h->use_tc2 ? CG_KERNEL_TENSOR_CHANNEL_MAJOR : (h->use_tc ? CG_KERNEL_TENSOR_PIXEL_MAJOR : CG_KERNEL_DIRECT);
+}
 
 cg_status cg_conv_forward(cg_conv_t h, const void* x, const void* w_base, const void* w_cond,
                           const cg_bn_params* bn, const float* delta, const void* residual,
@@ -160,13 +206,20 @@ cg_status cg_conv_forward(cg_conv_t h, const void* x, const void* w_base, const 
     return CG_ERR_ALIGNMENT;
   const size_t need = cg_conv_workspace_bytes(h);
   if (need > 0 && (!workspace || workspace_bytes < need)) return CG_ERR_WORKSPACE;
+  // the kernels that use the workspace access it in 16-byte pieces and clear its first 256 bytes
+  if (need > 0 && !aligned(workspace, 256)) return CG_ERR_ALIGNMENT;
+  int cur = -1;
+  if (cudaGetDevice(&cur) != cudaSuccess) return CG_ERR_CUDA;
+  if (cur != h->device) return CG_ERR_INVALID_ARG;         // a handle belongs to the device it was created on
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   int err;
-  if (h->use_tc) {
+  if (h->use_tc2) {
+    err = cg::launch_tc2(h->L, h->plan2, &h->maps2, x, w_base, w_cond, *bn, delta, residual, y,
+                         mask_out, h->counters, stream);
+  } else if (h->use_tc) {
     err = cg::launch_tc(h->L, h->plan, h->desc.in_dtype, &h->maps, x, w_base, w_cond, *bn, delta,
                         residual, y, mask_out, workspace, h->counters, stream);
   } else if (h->L.channel_tau > 0.f) {
-    if (!aligned(workspace, 256)) return CG_ERR_ALIGNMENT;
     err = cg::launch_direct_channel_gate(h->L, h->desc.in_dtype, x, w_base, w_cond, *bn, delta,
                                          residual, y, mask_out, workspace, h->counters, stream);
   } else {

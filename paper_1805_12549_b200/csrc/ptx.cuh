@@ -248,6 +248,11 @@ __device__ __forceinline__ void tmem_ld_wait16(uint32_t* a, uint32_t* b) {
                : "memory");
 }
 
+// Waits for every TMEM load of this thread (the loaded registers are not used afterwards).
+__device__ __forceinline__ void tmem_ld_wait_all() {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
 // N = 16 or 32 columns for the warp's 32 lanes, without waiting: several loads can be in flight.
 // Every use of the registers must come after tmem_ld_wait<N>() on the same array.
 template <int N>

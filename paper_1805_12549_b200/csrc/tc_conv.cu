@@ -822,8 +822,10 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     auto combine_pass = [&](int j) {
       const int slot = j % kNP, rslot = j % kNR;
       CG_PROF_T(pc0);
+      // A wait that gives up must not keep its thread from the group barrier below, where the
+      // sibling warps (whose waits may still have succeeded) are going to arrive: the decision to
+      // leave is taken after that barrier, from the CTA-wide flag, by all of them together.
       ok = wait_bar(cx, &sh->gate_done[slot], (j / kNP) & 1, 12);   // every gate warp's flags and words
-      if (!ok) return;
       const uint32_t blocks = !has_cond ? 0u : (dense ? kAllBlocks : slot_blocks(sh, slot));
       const uint32_t* s_words = s_mask + (slot * 128 + row) * kWords;
       uint32_t any = 0;                                              // cgi == 0: any gate of the row
@@ -836,8 +838,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       // the mask word that holds this warp's 16 or 32 columns, and their position in it
       const uint32_t wv = s_words[col0 >> 5];
       const int wshift = col0 & 31;
-      ok = wait_bar(cx, &sh->cond_done[rslot], (j / kNR) & 1, 13);
-      if (!ok) return;
+      ok = ok && wait_bar(cx, &sh->cond_done[rslot], (j / kNR) & 1, 13);
       ptx::tc_fence_after();
       if (warp == kEpiWarp0 + kGateWarps) CG_PROF_EV(j, 7);
       // the warp's columns go through the registers 16 at a time; the loads of the next 16 are
@@ -863,6 +864,11 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       }
       CG_PROF_T(pc1);
       ptx::named_bar_sync(1, kCombThreads);
+      if (*(volatile uint32_t*)&sh->abort_flag) {   // (the same for every thread of the group)
+        ptx::tmem_ld_wait_all();
+        ok = false;
+        return;
+      }
       CG_PROF_T(pc2);
       // residual rows (the shortcut of a residual block, added before the activation)
       const __nv_bfloat16* res_row = nullptr;
@@ -1031,6 +1037,12 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   if (blockIdx.x == 0 && lane == 0) atomicAdd(&g_prof[warp * 32 + 31], (unsigned long long)(clock64() - prof_t0));
 #endif
   // ---------------------------------------------------------------- teardown
+  if (*(volatile uint32_t*)&sh->abort_flag) {
+    // a wait gave up somewhere: let copies and MMAs that are still in flight finish (they take
+    // microseconds) before the CTA's shared memory and TMEM go back
+    const long long t_drain = clock64();
+    while (clock64() - t_drain < 4000000ll) {}
+  }
   ptx::tc_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -1328,15 +1340,22 @@ bool encode(CUtensorMap* map, int elem_bytes, void* base, int rank, const cuuint
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-int sm_count() {
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-      sms = 148;
+constexpr int kMaxDevices = 64;
+
+int current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+  return dev;
+}
+
+int sm_count(int dev) {
+  static int sms[kMaxDevices] = {};
+  if (sms[dev] == 0) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+    sms[dev] = v;
   }
-  return sms;
+  return sms[dev];
 }
 
 }  // namespace
@@ -1463,7 +1482,9 @@ bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
     // resident weights: the base and the conditional path get their own MMA issuer and their own
     // half of the patch ring
     const bool two = resident && P.cond_tiles > 0 && P.cond_mode != CG_COND_COMPACT;
-    P.share_a = (two && P.chunks == 1 && P.planes == 1) ? 1 : 0;
+    // (three issuers only at NT = 64: with a single R accumulator two conditional issuers would
+    // alternate on one r_free/cond_done barrier pair and could run a whole phase apart)
+    P.share_a = (two && P.chunks == 1 && P.planes == 1 && nt == 64) ? 1 : 0;
     P.split_a = (two && !P.share_a && na >= 2 * P.planes && (na / 2) % P.planes == 0) ? na / 2 : 0;
     P.issuers = P.share_a ? 3 : (P.split_a ? 2 : 1);
     P.smem_bytes = (unsigned)(off + 1024);
@@ -1564,7 +1585,9 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
     if (e != cudaSuccess) return (int)e;
   }
   // persistent grid: one CTA per SM, a multiple of the number of column tiles
-  const int sms = sm_count();
+  const int dev = current_device();
+  if (dev < 0) return (int)cudaErrorInvalidDevice;
+  const int sms = sm_count(dev);
   int grid = sms - sms % P.tiles_n;
   if (grid < P.tiles_n) grid = P.tiles_n;
   if (grid > P.tiles_m * P.tiles_n) grid = P.tiles_m * P.tiles_n;
@@ -1574,12 +1597,12 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
   const int which = P.elem_bytes == 1 ? 2 : (P.nt == 128 ? 1 : 0);
   const Kernel kernels[3] = {tc_gated_conv_kernel<64, false>, tc_gated_conv_kernel<128, false>,
                              tc_gated_conv_kernel<128, true>};
-  static bool attr_set[3] = {false, false, false};
-  if (!attr_set[which]) {
+  static bool attr_set[kMaxDevices][3] = {};   // (the attribute is per device)
+  if (!attr_set[dev][which]) {
     const cudaError_t e = cudaFuncSetAttribute(kernels[which], cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                227 * 1024);
     if (e != cudaSuccess) return (int)e;
-    attr_set[which] = true;
+    attr_set[dev][which] = true;
   }
   // Every layer asks for the same (maximum) amount of dynamic shared memory: consecutive layer
   // kernels then never differ in the SM's shared-memory configuration.  The launch is a
@@ -1615,11 +1638,11 @@ int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, c
     const int grid2 = (int)(items < sms ? items : sms);
     typedef void (*Kernel2)(CUtensorMap, CpParams);
     const Kernel2 k2 = P.nt == 128 ? (Kernel2)tc_compact_cond_kernel<128> : (Kernel2)tc_compact_cond_kernel<64>;
-    static bool attr2[2] = {false, false};
-    if (!attr2[P.nt == 128]) {
+    static bool attr2[kMaxDevices][2] = {};
+    if (!attr2[dev][P.nt == 128]) {
       const cudaError_t e = cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
       if (e != cudaSuccess) return (int)e;
-      attr2[P.nt == 128] = true;
+      attr2[dev][P.nt == 128] = true;
     }
     k2<<<grid2, kCpThreads, smem2, stream>>>(ms->wc, cp);
   }

@@ -149,7 +149,41 @@ class GpuCase:
             self.params[k] = torch.from_numpy(np.ascontiguousarray(v)).cuda()
         self.bn = B.make_bn(self.params)
         self.delta = None if c.delta is None else torch.from_numpy(c.delta).cuda()
-        self.y, self.mask = self.conv.alloc_outputs()
+        # y, mask and the workspace sit inside larger buffers whose margins hold a known pattern:
+        # a kernel that writes outside its tensors is caught by check_guards() after every run
+        self.y, self._y_buf = self._guarded(self.conv.desc.n * self.conv.ho * self.conv.wo * s.c_out,
+                                            self.B._TORCH_DTYPE[dt])
+        self.y = self.y.view(self.conv.desc.n, self.conv.ho, self.conv.wo, s.c_out)
+        self.mask, self._m_buf = self._guarded(self.conv.m * self.conv.words, torch.int32)
+        self.mask = self.mask.view(self.conv.m, self.conv.words)
+        self._ws_buf = None
+        if self.conv.workspace is not None:
+            n = self.conv.workspace.numel()
+            ws, self._ws_buf = self._guarded(n, torch.uint8)
+            self.conv.workspace = ws
+
+    GUARD = 4096      # bytes of pattern before and after each tensor
+    PATTERN = 0x5A
+
+    def _guarded(self, numel, dtype):
+        torch = self.torch
+        esz = torch.empty(0, dtype=dtype).element_size()
+        nbytes = numel * esz
+        pad = (-nbytes) % 256
+        buf = torch.full((self.GUARD + nbytes + pad + self.GUARD,), self.PATTERN, dtype=torch.uint8, device="cuda")
+        inner = buf[self.GUARD:self.GUARD + nbytes].view(dtype)
+        return inner, buf
+
+    def check_guards(self):
+        for name, buf, t in (("y", self._y_buf, self.y), ("mask", self._m_buf, self.mask),
+                             ("workspace", self._ws_buf, self.conv.workspace)):
+            if buf is None:
+                continue
+            nbytes = t.numel() * t.element_size()
+            head = buf[:self.GUARD]
+            tail = buf[self.GUARD + nbytes:]
+            assert bool((head == self.PATTERN).all()), f"write in front of {name}"
+            assert bool((tail == self.PATTERN).all()), f"write behind {name}"
 
     def run(self, with_mask=True):
         self.y.fill_(0)
@@ -158,6 +192,7 @@ class GpuCase:
                           self.mask if with_mask else None, self.res)
         st = self.conv.stats()
         self.torch.cuda.synchronize()
+        self.check_guards()
         y = self.y.float().cpu().numpy() if self.c.dtype != "i8" else self.y.cpu().numpy()
         mask = self.mask.cpu().numpy().view(np.uint32)
         return y, mask, st
