@@ -5,7 +5,10 @@
                     [--workload cifar|imagenet] [--density D] [--rho R] [--cond-mode M]
 
 One step = one forward pass of every gated 3x3 layer shape of the workload over one batch
-of synthetic activations (ReLU of box-smoothed Gaussian noise, bf16).  Prints ONE JSON line.
+of synthetic activations (ReLU of box-smoothed Gaussian noise, bf16).  Prints ONE JSON line:
+the headline value on --workload, every layer at the target density and with all gates open
+(`speedup_vs_density1` against `flop_reduction`), and, at one GPU, extra blocks for the ImageNet
+shapes, G = 8, a density sweep, cross-channel correlated inputs and the int8 layers.
 Under torchrun each rank runs the same layers on its own batch (weak scaling, no collective
 on the data path); the time is the max over ranks.
 """
@@ -142,58 +145,106 @@ def whole_job_rate(images_per_rank, world, ms_per_step):
 
 
 # ------------------------------------------------------------------------------- our arm
+CALIB_IMAGES = 4     # gate statistics and Delta come from the first images of the batch (both arms)
+
+
+def calibrate(p, density, eps=1e-5):
+    """Gate statistics = per-channel mean/variance of the partial sums `p` [pixels, c_out] (what a
+    trained network's running statistics would hold); Delta = one scalar per layer at the quantile
+    of the normalised partial sums that gives the target density.  Used by both arms, on the
+    partial sums of the first CALIB_IMAGES images."""
+    p = np.asarray(p, np.float64)
+    mean = p.mean(0).astype(np.float32)
+    var = np.maximum(p.var(0), 1e-6).astype(np.float32)
+    p_hat = (p - mean) / np.sqrt(var.astype(np.float64) + eps)
+    return mean, var, p_hat.ravel()
+
+
+def delta_for(p_hat, density):
+    if density >= 1.0:
+        return float("-inf")
+    if density <= 0.0:
+        return float("inf")
+    return float(np.quantile(p_hat, 1.0 - density))
+
+
 class LayerBench:
     """Device buffers, calibrated gate parameters and the handle of one layer shape."""
 
     SETS = 4   # x/y/mask buffer sets rotated so that no step finds its tensors in L2
 
-    def __init__(self, shape, density, rho, cond_mode, rank):
+    def __init__(self, shape, rho, cond_mode, rank, dtype="bf16", host=False):
         import torch
         from paper_1805_12549_b200 import binding as B, synth
-        self.B, self.torch, self.shape = B, torch, shape
+        self.B, self.torch, self.shape, self.dtype = B, torch, shape, dtype
         s = shape
         key = ("bench", s.name, rank)
-        x = synth.bf16_bits(synth.smoothed_noise((key, "x"), s.n, s.hw, s.hw, s.c_in, rho=rho))
-        wb, wc = synth.kaiming_weights(key, s.c_out, 3, 3, s.c_in, s.groups)
-        bn = synth.bn_params(key, s.c_out)
         dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
-        bf = lambda a: dev(synth.bf16_bits(a).view(np.int16)).view(torch.bfloat16)
-        x0 = dev(x.view(np.int16)).view(torch.bfloat16)
-        self.x_host = x0.cpu().pin_memory()
-        self.xs = [x0] + [torch.roll(x0, k, dims=0).contiguous() for k in range(1, self.SETS)]
-        self.wb, self.wc = bf(wb), bf(wc)
-        self.conv = B.GatedConv(s.n, s.hw, s.hw, s.c_in, s.c_out, k=3, stride=s.stride, pad=1,
-                                groups=s.groups, dtype=B.CG_BF16, cond_mode=cond_mode)
-        self.params = {k: dev(v) for k, v in bn.items()}
-        # gate statistics = per-channel mean/variance of the partial sums over this batch
-        # (what a trained network's running statistics would hold); Delta = one scalar per
-        # layer at the quantile of the normalised partial sums that gives the target density
-        p = torch.empty((self.conv.m, s.c_out), dtype=torch.float32, device="cuda")
-        B.cg_conv_partial_sums(self.conv.handle, x0, self.wb, p)
-        torch.cuda.synchronize()
-        mean, var = p.mean(dim=0), p.var(dim=0, unbiased=False).clamp_min(1e-6)
-        self.params["gate_mean"], self.params["gate_var"] = mean.contiguous(), var.contiguous()
-        if density >= 1.0:
-            dval = float("-inf")
+        calib = min(CALIB_IMAGES, s.n)
+        if dtype == "bf16":
+            x = synth.bf16_bits(synth.smoothed_noise((key, "x"), s.n, s.hw, s.hw, s.c_in, rho=rho))
+            wb, wc = synth.kaiming_weights(key, s.c_out, 3, 3, s.c_in, s.groups)
+            bf = lambda a: dev(synth.bf16_bits(a).view(np.int16)).view(torch.bfloat16)
+            x0 = dev(x.view(np.int16)).view(torch.bfloat16)
+            self.wb, self.wc = bf(wb), bf(wc)
+            self.conv = B.GatedConv(s.n, s.hw, s.hw, s.c_in, s.c_out, k=3, stride=s.stride, pad=1,
+                                    groups=s.groups, dtype=B.CG_BF16, cond_mode=cond_mode)
+            self.params = {k: dev(v) for k, v in synth.bn_params(key, s.c_out).items()}
+            cal = B.GatedConv(calib, s.hw, s.hw, s.c_in, s.c_out, k=3, stride=s.stride, pad=1,
+                              groups=s.groups, dtype=B.CG_BF16, algo=B.CG_ALGO_DIRECT)
+            p = torch.empty((cal.m, s.c_out), dtype=torch.float32, device="cuda")
+            B.cg_conv_partial_sums(cal.handle, x0[:calib].contiguous(), self.wb, p)
+            torch.cuda.synchronize()
+            mean, var, self.p_hat = calibrate(p.cpu().numpy(), None)
+            cal.close()
+            self.params["gate_mean"], self.params["gate_var"] = dev(mean), dev(var)
+            self.delta = torch.zeros((s.c_out,), dtype=torch.float32, device="cuda")
+            el = 2
         else:
-            p_hat = ((p - mean) / torch.sqrt(var + 1e-5)).flatten()
-            idx = torch.randint(0, p_hat.numel(), (min(p_hat.numel(), 4_000_000),), device="cuda")
-            dval = float(torch.quantile(p_hat[idx], 1.0 - density))
-        del p
-        self.delta = torch.full((s.c_out,), dval, dtype=torch.float32, device="cuda")
+            x0 = dev(synth.int8_activations(key, s.n, s.hw, s.hw, s.c_in))
+            wb, wc = synth.int8_weights(key, s.c_out, 3, 3, s.c_in, s.groups)
+            self.wb, self.wc = dev(wb), dev(wc)
+            self.conv = B.GatedConv(s.n, s.hw, s.hw, s.c_in, s.c_out, k=3, stride=s.stride, pad=1,
+                                    groups=s.groups, dtype=B.CG_I8, requant_shift=24, cond_mode=cond_mode)
+            cal = B.GatedConv(calib, s.hw, s.hw, s.c_in, s.c_out, k=3, stride=s.stride, pad=1,
+                              groups=s.groups, dtype=B.CG_I8, requant_shift=24, algo=B.CG_ALGO_DIRECT)
+            p = torch.empty((cal.m, s.c_out), dtype=torch.int32, device="cuda")
+            B.cg_conv_partial_sums(cal.handle, x0[:calib].contiguous(), self.wb, p)
+            torch.cuda.synchronize()
+            self.p_int = p.cpu().numpy().astype(np.float64)
+            cal.close()
+            sigma_base = self.p_int.std() + 1.0
+            q = synth.int8_requant(key, s.c_out, 24, sigma_base, sigma_base * np.sqrt(s.groups))
+            self.params = {k: dev(v) for k, v in q.items()}
+            self.params["q_gate_thr"] = torch.zeros((s.c_out,), dtype=torch.int32, device="cuda")
+            self.delta = None
+            el = 1
+        self.xs = [x0] + [torch.roll(x0, k, dims=0).contiguous() for k in range(1, self.SETS)]
         self.bn = B.make_bn(self.params)
         self.ys, self.masks = zip(*[self.conv.alloc_outputs() for _ in range(self.SETS)])
-        self.y_host = torch.empty(self.ys[0].shape, dtype=torch.bfloat16).pin_memory()
-        self.mask_host = torch.empty(self.masks[0].shape, dtype=torch.int32).pin_memory()
-        self.staging = torch.empty(B.cg_conv_host_staging_bytes(self.conv.handle),
-                                   dtype=torch.uint8, device="cuda")
-        el = 2
+        if host:
+            self.x_host = x0.cpu().pin_memory()
+            self.y_host = torch.empty(self.ys[0].shape, dtype=self.ys[0].dtype).pin_memory()
+            self.mask_host = torch.empty(self.masks[0].shape, dtype=torch.int32).pin_memory()
+            self.staging = torch.empty(B.cg_conv_host_staging_bytes(self.conv.handle),
+                                       dtype=torch.uint8, device="cuda")
         self.bytes_x = s.n * s.hw * s.hw * s.c_in * el
         self.bytes_y = self.conv.m * s.c_out * el
         self.bytes_mask = self.conv.m * self.conv.words * 4
         self.bytes_w = s.c_out * 9 * s.c_in * el
         self.algorithmic_bytes = self.bytes_x + self.bytes_y + self.bytes_mask + self.bytes_w
         self.stats = None
+
+    def set_density(self, density):
+        """Rewrites Delta (or the integer thresholds) in place: captured graphs read the new values."""
+        if self.dtype == "bf16":
+            self.delta.fill_(delta_for(self.p_hat, density))
+        else:
+            if density >= 1.0:
+                thr = np.full(self.shape.c_out, np.iinfo(np.int32).min, np.int64)
+            else:
+                thr = np.ceil(np.quantile(self.p_int, 1.0 - density, axis=0))
+            self.params["q_gate_thr"].copy_(self.torch.from_numpy(thr.astype(np.int32)))
 
     def forward(self, i):
         k = i % self.SETS
@@ -203,6 +254,126 @@ class LayerBench:
     def forward_host(self):
         self.B.cg_conv_forward_host(self.conv.handle, self.x_host, self.wb, self.wc, self.bn,
                                     self.delta, None, self.y_host, self.mask_host, self.staging)
+
+    def close(self):
+        self.conv.close()
+
+
+class Plain:
+    def __init__(self, fn):
+        self.fn = fn
+
+    def replay(self):
+        self.fn()
+
+
+def capture(fn, no_graph):
+    """Launches go through CUDA graphs (one graph = the captured calls on fixed buffer sets), so
+    the device, not the Python caller, sets the pace."""
+    import torch
+    if no_graph:
+        return Plain(fn)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        fn()
+    return g
+
+
+def time_layer(lb, reps, no_graph):
+    """Average device time of one launch of the layer kernel (CUDA events on the launching
+    stream), the buffer sets rotating so that no launch finds its tensors in L2."""
+    import torch
+    stream = torch.cuda.current_stream()
+    g = capture(lambda: [lb.forward(k) for k in range(LayerBench.SETS)], no_graph)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g.replay()
+    torch.cuda.synchronize()
+    lb.conv.stats()
+    e0.record(stream)
+    for _ in range(reps):
+        g.replay()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    st = lb.conv.stats()
+    return e0.elapsed_time(e1) / (reps * LayerBench.SETS), st
+
+
+def layer_record(lb, d_ms, st, peaks):
+    el_flops = 2.0 * st.gated_macs / max(st.calls, 1)
+    t_tensor = el_flops / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = lb.algorithmic_bytes / (peaks["hbm_gbs"] * 1e9)
+    rec = {
+        "layer": lb.shape.name, "us": round(d_ms * 1e3, 2), "density": round(st.density, 4),
+        "kernel": ["direct", "tcgen05 pixel-major", "tcgen05 channel-major"][lb.conv.kernel_id],
+        "gated_tflops": round(el_flops / (d_ms * 1e-3) / 1e12, 1),
+        "gbs": round(lb.algorithmic_bytes / (d_ms * 1e-3) / 1e9, 1),
+        "roof_us": round(max(t_tensor, t_hbm) * 1e6, 2),
+        "roof_frac": round(max(t_tensor, t_hbm) / (d_ms * 1e-3), 3),
+        "bound": "tensor" if t_tensor > t_hbm else "hbm",
+        "flop_reduction": round(st.dense_macs / max(st.gated_macs, 1), 3),
+        "executed_over_gated": round(st.executed_macs / max(st.gated_macs, 1), 3),
+        "blocks_skipped": f"{st.tiles_skipped}/{st.tiles_total}",
+    }
+    if lb.dtype != "bf16":
+        # no measured int8 tensor peak on this machine: the fraction is against the HBM side only
+        rec["roof_us"] = round(t_hbm * 1e6, 2)
+        rec["roof_frac"] = round(t_hbm / (d_ms * 1e-3), 3)
+        rec["bound"] = "hbm (no int8 tensor peak measured)"
+    return rec
+
+
+def with_density1(lb, rec, reps, no_graph, peaks, target):
+    """The same layer with every gate open (Delta = -inf): the method's own claim is the ratio."""
+    lb.set_density(1.0)
+    d1_ms, st1 = time_layer(lb, reps, no_graph)
+    lb.set_density(target)
+    rec["us_density1"] = round(d1_ms * 1e3, 2)
+    rec["speedup_vs_density1"] = round(d1_ms * 1e3 / rec["us"], 3)
+    dense_flops = 2.0 * st1.dense_macs / max(st1.calls, 1)
+    rec["dense_frac_of_tensor_peak_at_density1"] = round(
+        dense_flops / (d1_ms * 1e-3) / (peaks["bf16_tflops"] * 1e12), 3)
+    rec["executed_over_dense_at_density1"] = round(st1.executed_macs / max(st1.dense_macs, 1), 3)
+    return rec
+
+
+# Extra measurement blocks of the default run (each: every layer shape, one launch configuration
+# per density; kernel times only).  The headline value stays on the workload given by --workload.
+EXTRA_BLOCKS = [
+    {"workload": "imagenet", "groups": 4, "rho": 0.0, "dtype": "bf16", "densities": [0.1, 0.3, 0.6, 1.0]},
+    {"workload": "imagenet", "groups": 8, "rho": 0.0, "dtype": "bf16", "densities": [0.3, 1.0]},
+    {"workload": "imagenet", "groups": 4, "rho": 0.5, "dtype": "bf16", "densities": [0.1, 0.3]},
+    {"workload": "imagenet", "groups": 4, "rho": 0.0, "dtype": "i8", "densities": [0.3, 1.0]},
+]
+
+
+def run_block(block, args, peaks, rank):
+    from paper_1805_12549_b200 import synth
+    if block["workload"] == "imagenet":
+        name = "imagenet_resnet18_gated_3x3_layers"
+        shapes = synth.imagenet_resnet18_layers(64, block["groups"], transitions=block["dtype"] == "bf16")
+    else:
+        name = "cifar_resnet18_gated_3x3_layers"
+        shapes = synth.cifar_resnet18_layers(256, block["groups"])
+    out = {"workload": name, "batch": shapes[0].n, "groups": block["groups"], "rho": block["rho"],
+           "dtype": block["dtype"], "densities": {}}
+    per_density = {d: [] for d in block["densities"]}
+    for s in shapes:
+        lb = LayerBench(s, block["rho"], args.cond_mode, rank, dtype=block["dtype"])
+        for d in block["densities"]:
+            lb.set_density(d)
+            ms, st = time_layer(lb, 3, args.no_graph)
+            per_density[d].append(layer_record(lb, ms, st, peaks))
+        lb.close()
+        del lb
+    t1 = sum(r["us"] for r in per_density[1.0]) if 1.0 in per_density else None
+    for d in block["densities"]:
+        recs = per_density[d]
+        tot = sum(r["us"] for r in recs)
+        entry = {"us_all_layers": round(tot, 2), "layers": recs}
+        if t1 is not None:
+            entry["speedup_vs_density1"] = round(t1 / tot, 3)
+        out["densities"][str(d)] = entry
+    return out
 
 
 def run_ours(args):
@@ -219,7 +390,9 @@ def run_ours(args):
     if args.layers:
         keep = set(args.layers.split(","))
         shapes = [s for s in shapes if s.name in keep]
-    layers = [LayerBench(s, args.density, args.rho, args.cond_mode, rank) for s in shapes]
+    layers = [LayerBench(s, args.rho, args.cond_mode, rank, host=True) for s in shapes]
+    for lb in layers:
+        lb.set_density(args.density)
     stream = torch.cuda.current_stream()
 
     def step(i):
@@ -232,29 +405,10 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    # Launches go through CUDA graphs (one graph = one step on one buffer set), so the
-    # device, not the Python caller, sets the pace.
-    class Plain:
-        def __init__(self, fn):
-            self.fn = fn
-
-        def replay(self):
-            self.fn()
-
-    def capture(fn):
-        if args.no_graph:
-            return Plain(fn)
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g):
-            fn()
-        return g
-
     for i in range(LayerBench.SETS):
         step(i)                                   # first calls encode the tensor maps
     torch.cuda.synchronize()
-    step_graphs = [capture(lambda k=k: step(k)) for k in range(LayerBench.SETS)]
-    layer_graphs = [capture(lambda lb=lb: [lb.forward(k) for k in range(LayerBench.SETS)])
-                    for lb in layers]
+    step_graphs = [capture(lambda k=k: step(k), args.no_graph) for k in range(LayerBench.SETS)]
 
     # warm-up (at least W steps and about a second of load, so the clock samples are under load)
     sampler = ClockSampler(local) if rank == 0 else None
@@ -277,7 +431,6 @@ def run_ours(args):
         step_graphs[i % LayerBench.SETS].replay()
     e1.record(stream)
     torch.cuda.synchronize()
-    t1 = time.time()
     ms_total = max_over_ranks(e0.elapsed_time(e1))
     for lb in layers:
         lb.stats = lb.conv.stats()
@@ -285,43 +438,16 @@ def run_ours(args):
     batch = shapes[0].n
     value = whole_job_rate(batch, world, ms_step)
 
-    # per-layer kernel durations: the same launches, one layer at a time, back to back
+    # per-layer kernel durations at the target density and with every gate open
     reps = max(1, args.steps // LayerBench.SETS)
-    layer_ms = []
-    for g in layer_graphs:
-        g.replay()
-        torch.cuda.synchronize()
-        e0.record(stream)
-        for _ in range(reps):
-            g.replay()
-        e1.record(stream)
-        torch.cuda.synchronize()
-        layer_ms.append(e0.elapsed_time(e1) / (reps * LayerBench.SETS))
+    per_layer = []
+    for lb in layers:
+        d_ms, st = time_layer(lb, reps, args.no_graph)
+        rec = layer_record(lb, d_ms, st, peaks)
+        per_layer.append(with_density1(lb, rec, reps, args.no_graph, peaks, args.density))
     t1 = time.time()
     clocks = sampler.stop(t_load0, t1) if sampler else None
-    for lb in layers:
-        lb.conv.stats()
-
-    per_layer = []
-    for j, lb in enumerate(layers):
-        d_ms = layer_ms[j]
-        st = lb.stats
-        dens = st.density
-        flops = 2.0 * st.gated_macs / max(st.calls, 1)
-        t_tensor = flops / (peaks["bf16_tflops"] * 1e12)
-        t_hbm = lb.algorithmic_bytes / (peaks["hbm_gbs"] * 1e9)
-        per_layer.append({
-            "layer": lb.shape.name, "us": round(d_ms * 1e3, 2), "density": round(dens, 4),
-            "tensor_cores": bool(lb.conv.uses_tensor_cores),
-            "gated_tflops": round(flops / (d_ms * 1e-3) / 1e12, 1),
-            "gbs": round(lb.algorithmic_bytes / (d_ms * 1e-3) / 1e9, 1),
-            "roof_us": round(max(t_tensor, t_hbm) * 1e6, 2),
-            "roof_frac": round(max(t_tensor, t_hbm) / (d_ms * 1e-3), 3),
-            "bound": "tensor" if t_tensor > t_hbm else "hbm",
-            "flop_reduction": round(st.dense_macs / max(st.gated_macs, 1), 3),
-            "executed_over_gated": round(st.executed_macs / max(st.gated_macs, 1), 3),
-            "blocks_skipped": f"{st.tiles_skipped}/{st.tiles_total}",
-        })
+    speedup = round(sum(r["us_density1"] for r in per_layer) / sum(r["us"] for r in per_layer), 3)
     dom = max(range(len(layers)), key=lambda j: per_layer[j]["us"])
     dl, dp = layers[dom], per_layer[dom]
     if dp["bound"] == "hbm":
@@ -332,7 +458,7 @@ def run_ours(args):
     roof["frac"] = round(roof["achieved"] / roof["peak"], 4)
     roof["traffic"] = measured_traffic(dp["layer"])
     roof["algorithmic_bytes"] = dl.algorithmic_bytes
-    roof["kernel"] = f"tc_gated_conv_kernel ({dp['layer']})"
+    roof["kernel"] = f"{dp['kernel']} ({dp['layer']})"
     roof["peak_source"] = f"of {peaks['source']}"
     roof["us_per_launch"] = dp["us"]
 
@@ -353,6 +479,17 @@ def run_ours(args):
     e2e = {"value": round(whole_job_rate(batch, world, ms_e2e / e2e_steps), 1), "unit": UNIT,
            "h2d_bytes_per_step": sum(lb.bytes_x for lb in layers),
            "d2h_bytes_per_step": sum(lb.bytes_y + lb.bytes_mask for lb in layers)}
+    launches = args.steps * sum(lb.B.cg_conv_launches_per_forward(lb.conv.handle) for lb in layers)
+    for lb in layers:
+        lb.close()
+    del layers, step_graphs
+    torch.cuda.empty_cache()
+
+    blocks = []
+    if rank == 0 and world == 1 and not args.no_extra:
+        for block in EXTRA_BLOCKS:
+            blocks.append(run_block(block, args, peaks, rank))
+            torch.cuda.empty_cache()
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -367,12 +504,12 @@ def run_ours(args):
             "config": {"workload": wname, "batch_per_gpu": batch, "groups": 4,
                        "target_density": args.density, "rho": args.rho,
                        "cond_mode": args.cond_mode,
+                       "calibration": f"gate statistics and Delta from the first {CALIB_IMAGES} images",
                        "l2": f"x/y/mask rotate over {LayerBench.SETS} buffer sets per layer "
                              "(total > L2)", "parallelism": f"batch x{world}, no collective"},
-            "clocks": clocks, "e2e": e2e,
-            "gpu_launches": args.steps * sum(lb.B.cg_conv_launches_per_forward(lb.conv.handle)
-                                             for lb in layers),
-            "roofline": roof, "cpu_baseline": cpu, "layers": per_layer,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+            "speedup_vs_density1": speedup,
+            "roofline": roof, "cpu_baseline": cpu, "layers": per_layer, "blocks": blocks,
         }
         print(json.dumps(out))
     if world > 1:
@@ -381,29 +518,27 @@ def run_ours(args):
 
 # ------------------------------------------------------------------------------- oracle arm
 def oracle_layer_inputs(s, density, rho, images):
-    """The same seeded layer as LayerBench, cut to `images` images, calibrated by the oracle."""
+    """The same seeded layer as LayerBench, cut to `images` images; gate statistics and Delta from
+    the oracle's partial sums of the first CALIB_IMAGES images (the direct kernels that calibrate
+    the other arm reproduce these sums bit for bit)."""
     from oracle import oracle as O
     from paper_1805_12549_b200 import synth
     key = ("bench", s.name, 0)
     chunk = 16
-    n_gen = ((images + chunk - 1) // chunk) * chunk
-    x = synth.bf16_round(synth.smoothed_noise((key, "x"), min(n_gen, s.n), s.hw, s.hw, s.c_in,
-                                              rho=rho))[:images]
+    n_need = max(images, min(CALIB_IMAGES, s.n))
+    n_gen = ((n_need + chunk - 1) // chunk) * chunk
+    x_all = synth.bf16_round(synth.smoothed_noise((key, "x"), min(n_gen, s.n), s.hw, s.hw, s.c_in,
+                                                  rho=rho))
     wb, wc = synth.kaiming_weights(key, s.c_out, 3, 3, s.c_in, s.groups)
     wb, wc = synth.bf16_round(wb), synth.bf16_round(wc)
     bn = synth.bn_params(key, s.c_out)
+    calib = min(CALIB_IMAGES, s.n)
     sh = O.Shape(images, s.hw, s.hw, s.c_in, s.c_out, stride=s.stride, groups=s.groups)
-    one = O.Shape(1, s.hw, s.hw, s.c_in, s.c_out, stride=s.stride, groups=s.groups)
-    probe = O.gated_conv(one, x[:1], wb, wc, bn, np.full(s.c_out, np.inf, np.float32))
-    p = probe.p.reshape(-1, s.c_out).astype(np.float64)
-    bn["gate_mean"] = p.mean(0).astype(np.float32)
-    bn["gate_var"] = np.maximum(p.var(0), 1e-6).astype(np.float32)
-    if density >= 1.0:
-        dval = -np.inf
-    else:
-        p_hat = (p - bn["gate_mean"]) / np.sqrt(bn["gate_var"] + 1e-5)
-        dval = float(np.quantile(p_hat, 1.0 - density))
-    return sh, x, wb, wc, bn, np.full(s.c_out, dval, np.float32)
+    cs = O.Shape(calib, s.hw, s.hw, s.c_in, s.c_out, stride=s.stride, groups=s.groups)
+    probe = O.gated_conv(cs, x_all[:calib], wb, wc, bn, np.full(s.c_out, np.inf, np.float32))
+    bn["gate_mean"], bn["gate_var"], p_hat = calibrate(probe.p.reshape(-1, s.c_out), None)
+    dval = delta_for(p_hat, density)
+    return sh, x_all[:images], wb, wc, bn, np.full(s.c_out, dval, np.float32)
 
 
 def cpu_baseline(args, shapes):
@@ -478,6 +613,8 @@ def main():
     ap.add_argument("--cond-mode", type=int, default=0)
     ap.add_argument("--cpu-images", type=int, default=None)
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-extra", action="store_true",
+                    help="skip the extra blocks (ImageNet shapes, G = 8, density sweep, int8)")
     ap.add_argument("--layers", default=None,
                     help="comma-separated layer names to keep (e.g. c64@56,c256@14)")
     ap.add_argument("--no-graph", action="store_true",
@@ -485,8 +622,19 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
-    else:
-        run_ours(args)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started plainly with --gpus N: run N ranks, one per GPU (each shards nothing and
+        # exchanges nothing on the data path; only the timing is reduced over the ranks)
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+               f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1", "--master-port",
+               str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.call(cmd))
+    run_ours(args)
 
 
 if __name__ == "__main__":

@@ -157,13 +157,15 @@ void cg_conv_destroy(cg_conv_t h) {
 size_t cg_conv_workspace_bytes(cg_conv_t h) {
   if (!h) return 0;
   if (h->L.channel_tau > 0.f) return cg::channel_gate_workspace_bytes(h->L);
-  return (h->use_tc && !h->use_tc2) ? cg::tc_workspace_bytes(h->L, h->plan) : 0;
+  if (h->use_tc2) return cg::tc2_workspace_bytes(h->L, h->plan2);
+  return h->use_tc ? cg::tc_workspace_bytes(h->L, h->plan) : 0;
 }
 
 int cg_conv_launches_per_forward(cg_conv_t h) {
   if (!h) return 0;
   if (h->L.channel_tau > 0.f) return 2;
-  return (h->use_tc && !h->use_tc2 && h->plan.cond_mode == CG_COND_COMPACT) ? 2 : 1;
+  if (h->use_tc2) return h->plan2.pad8 ? 2 : 1;
+  return (h->use_tc && h->plan.cond_mode == CG_COND_COMPACT) ? 2 : 1;
 }
 
 int cg_conv_uses_tensor_cores(cg_conv_t h) { return h ? h->use_tc : 0; }
@@ -215,7 +217,7 @@ cg_status cg_conv_forward(cg_conv_t h, const void* x, const void* w_base, const 
   int err;
   if (h->use_tc2) {
     err = cg::launch_tc2(h->L, h->plan2, &h->maps2, x, w_base, w_cond, *bn, delta, residual, y,
-                         mask_out, h->counters, stream);
+                         mask_out, workspace, h->counters, stream);
   } else if (h->use_tc) {
     err = cg::launch_tc(h->L, h->plan, h->desc.in_dtype, &h->maps, x, w_base, w_cond, *bn, delta,
                         residual, y, mask_out, workspace, h->counters, stream);

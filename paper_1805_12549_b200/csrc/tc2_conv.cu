@@ -595,13 +595,44 @@ bool encode2(CUtensorMap* map, void* base, int rank, const cuuint64_t* dims,
 
 size_t align_up2(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Base slices of 8 channels (G = 8 at 64 input channels) are half of the 16-channel K step of a
+// bf16 MMA.  The weights are copied into scratch memory with the K steps made whole: W_base gets 8
+// zero channels behind its 8 per tap (the base path then reads input channels [0,16) and multiplies
+// the upper 8 by zero), W_cond gets 8 zero channels in front (the conditional path reads every
+// channel and multiplies the first 8 by zero).  The sums are unchanged.
+__global__ void tc2_repack_kernel(const __nv_bfloat16* __restrict__ wb, const __nv_bfloat16* __restrict__ wc,
+                                  __nv_bfloat16* __restrict__ wb16, __nv_bfloat16* __restrict__ wcf, int rows,
+                                  int c_in) {
+  // rows = c_out * taps
+  const int total = rows * (16 + c_in);
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+    const int row = i / (16 + c_in), c = i - row * (16 + c_in);
+    if (c < 16) {
+      wb16[(size_t)row * 16 + c] = c < 8 ? wb[(size_t)row * 8 + c] : __float2bfloat16_rn(0.f);
+    } else {
+      const int cc = c - 16;
+      wcf[(size_t)row * c_in + cc] = cc < 8 ? __float2bfloat16_rn(0.f) : wc[(size_t)row * (c_in - 8) + cc - 8];
+    }
+  }
+}
+
 }  // namespace
+
+size_t tc2_workspace_bytes(const LayerDims& L, const Tc2Plan& P) {
+  if (!P.valid || !P.pad8) return 0;
+  const size_t rows = (size_t)L.c_out * L.kh * L.kw;
+  return align_up2(rows * 16 * 2, 256) + align_up2(rows * (size_t)L.c_in * 2, 256);
+}
 
 // K stages of a job in the order the MMA issuer consumes them (and the weight producer loads
 // them).  Base path: when c_p >= 64 one stage per (64-channel chunk, filter tap); when c_p is 16
 // or 32 a stage covers 64/c_p taps of chunk 0.  Conditional path: one stage per (chunk, tap);
 // when c_p < 64 chunk 0 comes first and only its K steps behind the base channels are used.
-static int build_stages(const LayerDims& L, int wp, Tc2Stage* st, int* nb_out) {
+static int build_stages(const LayerDims& L0, int wp, int pad8, Tc2Stage* st, int* nb_out) {
+  // (pad8: the weights are repacked so that the base path reads 16 channels per tap, the upper 8
+  // with zero weights, and the conditional path reads every channel, the first 8 with zero weights)
+  LayerDims L = L0;
+  if (pad8) { L.c_p = 16; L.c_r = L.c_in; }
   const int taps = L.kh * L.kw;
   const int chunks = L.c_in / 64;
   int n = 0;
@@ -638,6 +669,9 @@ static int build_stages(const LayerDims& L, int wp, Tc2Stage* st, int* nb_out) {
     if (L.c_p >= 64) {
       for (int q = L.c_p / 64; q < chunks; ++q)
         for (int t = 0; t < taps; ++t) full_stage(t * L.c_r + 64 * q - L.c_p, 1, q, t, 0);
+    } else if (pad8) {
+      for (int q = 0; q < chunks; ++q)
+        for (int t = 0; t < taps; ++t) full_stage(t * L.c_r + 64 * q, 1, q, t, 0);
     } else {
       for (int t = 0; t < taps; ++t) full_stage(t * L.c_r - L.c_p, 1, 0, t, L.c_p / 16);
       for (int q = 1; q < chunks; ++q)
@@ -663,7 +697,8 @@ bool tc2_plan(const LayerDims& L, int in_dtype, int cond_mode, int sms, Tc2Plan*
   if (L.grouping || L.stride != 1) return false;
   if (L.kh != L.kw || L.kh != 2 * L.pad + 1) return false;
   if (L.c_in % 64 != 0 || L.c_out % 32 != 0) return false;
-  if (!(L.c_p == 16 || L.c_p == 32 || L.c_p % 64 == 0)) return false;
+  if (!(L.c_p == 8 || L.c_p == 16 || L.c_p == 32 || L.c_p % 64 == 0)) return false;
+  P.pad8 = L.c_p == 8 ? 1 : 0;
   if (cond_mode == CG_COND_COMPACT) return false;
   if (L.c_in / 64 > 255) return false;
   P.wp = L.w + L.pad;
@@ -672,7 +707,7 @@ bool tc2_plan(const LayerDims& L, int in_dtype, int cond_mode, int sms, Tc2Plan*
   if ((long long)L.n * L.ho * L.wo * L.c_out >= (1ll << 32) - 1) return false;   // y is indexed in 32 bits
   P.chunks = L.c_in / 64;
   P.tiles_c = (L.c_out + 127) / 128;
-  P.ns = build_stages(L, P.wp, P.st, &P.nb);
+  P.ns = build_stages(L, P.wp, P.pad8, P.st, &P.nb);
   if (P.ns > kTc2MaxStages) return false;
   // the largest tap offset must fit the 16-bit table entries
   if (((L.kh - 1) * P.wp + L.kw) * 8 + 8 > 65535) return false;
@@ -746,10 +781,22 @@ bool tc2_plan(const LayerDims& L, int in_dtype, int cond_mode, int sms, Tc2Plan*
 }
 
 int launch_tc2(const LayerDims& L, const Tc2Plan& P, Tc2Maps* maps, const void* x,
-               const void* w_base, const void* w_cond, const cg_bn_params& bn, const float* delta,
-               const void* residual, void* y, uint32_t* mask, unsigned long long* counters,
+               const void* w_base_in, const void* w_cond_in, const cg_bn_params& bn, const float* delta,
+               const void* residual, void* y, uint32_t* mask, void* workspace, unsigned long long* counters,
                cudaStream_t stream) {
   if (!P.valid) return (int)cudaErrorInvalidValue;
+  const void* w_base = w_base_in;
+  const void* w_cond = w_cond_in;
+  int c_p = L.c_p, c_r = L.c_r;
+  if (P.pad8) {
+    if (!workspace) return (int)cudaErrorInvalidValue;
+    const size_t rows = (size_t)L.c_out * L.kh * L.kw;
+    __nv_bfloat16* wb16 = static_cast<__nv_bfloat16*>(workspace);
+    __nv_bfloat16* wcf = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + align_up2(rows * 16 * 2, 256));
+    tc2_repack_kernel<<<64, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(w_base_in),
+                                              static_cast<const __nv_bfloat16*>(w_cond_in), wb16, wcf, (int)rows, L.c_in);
+    w_base = wb16; w_cond = wcf; c_p = 16; c_r = L.c_in;
+  }
   const void* wc_key = w_cond ? w_cond : w_base;
   Tc2MapSet* ms = nullptr;
   for (int i = 0; i < Tc2Maps::kEntries; ++i) {
@@ -775,14 +822,14 @@ int launch_tc2(const LayerDims& L, const Tc2Plan& P, Tc2Maps* maps, const void* 
       }
     }
     {
-      cuuint64_t dims[2] = {(cuuint64_t)taps * L.c_p, (cuuint64_t)L.c_out};
-      cuuint64_t str[1] = {(cuuint64_t)taps * L.c_p * 2};
+      cuuint64_t dims[2] = {(cuuint64_t)taps * c_p, (cuuint64_t)L.c_out};
+      cuuint64_t str[1] = {(cuuint64_t)taps * c_p * 2};
       cuuint32_t box[2] = {64, (cuuint32_t)P.w_rows};
       if (!encode2(&ms->wb, const_cast<void*>(w_base), 2, dims, str, box)) return (int)cudaErrorInvalidValue;
     }
-    if (L.c_r > 0) {
-      cuuint64_t dims[2] = {(cuuint64_t)taps * L.c_r, (cuuint64_t)L.c_out};
-      cuuint64_t str[1] = {(cuuint64_t)taps * L.c_r * 2};
+    if (c_r > 0) {
+      cuuint64_t dims[2] = {(cuuint64_t)taps * c_r, (cuuint64_t)L.c_out};
+      cuuint64_t str[1] = {(cuuint64_t)taps * c_r * 2};
       cuuint32_t box[2] = {64, (cuuint32_t)P.w_rows};
       if (!encode2(&ms->wc, const_cast<void*>(w_cond), 2, dims, str, box)) return (int)cudaErrorInvalidValue;
     } else {

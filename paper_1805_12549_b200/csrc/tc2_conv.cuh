@@ -51,6 +51,7 @@ struct Tc2Plan {
   int patch_bytes;
   int patch_box_rows;    // stacked rows loaded per patch: r + 2*pad
   int cond_mode;
+  int pad8;              // c_p = 8: the weights are repacked into the workspace with whole K steps
   int use_img;           // whole images are loaded by single copies (small images)
   int grid;
   unsigned off_w, off_p, off_tab, off_bar, smem_bytes;
@@ -69,9 +70,10 @@ struct Tc2Maps {
 };
 
 bool tc2_plan(const LayerDims& L, int in_dtype, int cond_mode, int sms, Tc2Plan* plan);
+size_t tc2_workspace_bytes(const LayerDims& L, const Tc2Plan& plan);
 int launch_tc2(const LayerDims& L, const Tc2Plan& plan, Tc2Maps* maps, const void* x,
                const void* w_base, const void* w_cond, const cg_bn_params& bn, const float* delta,
-               const void* residual, void* y, uint32_t* mask, unsigned long long* counters,
-               cudaStream_t stream);
+               const void* residual, void* y, uint32_t* mask, void* workspace,
+               unsigned long long* counters, cudaStream_t stream);
 
 }  // namespace cg

@@ -31,6 +31,8 @@ SHAPES = [
     (O.Shape(2, 12, 12, 64, 96, kh=5, kw=5, pad=2, groups=2), "5x5 kernel, pad 2, 96 output channels"),
     (O.Shape(40, 28, 28, 128, 128, groups=4), "several jobs per CTA"),
     (O.Shape(256, 4, 4, 128, 128, groups=4), "many small images per pixel tile"),
+    (O.Shape(3, 56, 56, 64, 64, groups=8), "G = 8 at 64 channels: c_p = 8, weights repacked into the workspace"),
+    (O.Shape(2, 17, 9, 64, 128, groups=8), "c_p = 8, odd extents, 128 output channels"),
 ]
 
 
