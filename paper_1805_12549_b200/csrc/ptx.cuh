@@ -253,6 +253,37 @@ __device__ __forceinline__ void tmem_ld_wait_all() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// 16 TMEM lanes x 16 columns in the accumulator-fragment layout: thread t of the warp gets, from the
+// lanes [base, base+16) of the address,
+//   r[0], r[1] = lane base + t/4,     columns col + 2*(t%4), + 1
+//   r[2], r[3] = lane base + 8 + t/4, the same columns
+//   r[4..7]    = the same for columns col + 8 + ...
+// (no wait: follow with tmem_ld_wait16 on the registers of two such loads).
+__device__ __forceinline__ void tmem_ld_frag16(uint32_t taddr, uint32_t* r) {
+  asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr));
+}
+// Stores 8 registers of every thread into 8 consecutive columns of the thread's TMEM lane.
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* r) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr),
+               "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
+// Waits until the TMEM stores of this thread have completed.
+__device__ __forceinline__ void tmem_st_wait() {
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+// Four 8x8 matrices of 16-bit elements, each given as accumulator fragments (thread t holds
+// M[t/4][2*(t%4)], M[t/4][2*(t%4)+1] in one register), stored TRANSPOSED: row j of matrix i (eight
+// elements, 16 bytes) goes to the shared-memory address that thread 8*i + j passes, and holds
+// column j of the fragments.
+__device__ __forceinline__ void stmatrix_x4_trans(uint32_t smem_addr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3) {
+  asm volatile("stmatrix.sync.aligned.m8n8.x4.trans.shared.b16 [%0], {%1,%2,%3,%4};" ::"r"(smem_addr), "r"(r0), "r"(r1),
+               "r"(r2), "r"(r3)
+               : "memory");
+}
+
 // N = 16 or 32 columns for the warp's 32 lanes, without waiting: several loads can be in flight.
 // Every use of the registers must come after tmem_ld_wait<N>() on the same array.
 template <int N>

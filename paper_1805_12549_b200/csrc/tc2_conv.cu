@@ -48,7 +48,7 @@ namespace {
 constexpr int kThreads2 = 640;
 constexpr int kEpiWarp0 = 4;
 constexpr int kEpiWarps = 16;
-constexpr int kPatchEntries = 3;
+constexpr int kPatchEntries = 3;                  // at most; a plan may use two
 constexpr int kMaxRing = 12;
 constexpr int kMaxBoxes = 32;
 constexpr int kSpinLimit2 = 1 << 21;
@@ -84,6 +84,13 @@ struct Ctx2 {
   unsigned long long* counters;
 };
 
+// A wait ran out: record the error and where, and make every role of the CTA leave its loop.
+__device__ __noinline__ void give_up2(Shared2* sh, unsigned long long* counters, int site) {
+  if (atomicCAS(&counters[CNT_STATUS], 0ull, (unsigned long long)CG_ERR_DEVICE_TIMEOUT) == 0ull)
+    atomicExch(&counters[CNT_SITE], (unsigned long long)site);
+  atomicExch(&sh->abort_flag, 1u);
+}
+
 __device__ __noinline__ bool wait2_slow(Shared2* sh, unsigned long long* counters, uint64_t* bar,
                                         uint32_t parity, int site) {
   const long long t0 = clock64();
@@ -94,9 +101,7 @@ __device__ __noinline__ bool wait2_slow(Shared2* sh, unsigned long long* counter
       if (clock64() - t0 > kWaitCycles2) break;
     }
   }
-  if (atomicCAS(&counters[CNT_STATUS], 0ull, (unsigned long long)CG_ERR_DEVICE_TIMEOUT) == 0ull)
-    atomicExch(&counters[CNT_SITE], (unsigned long long)site);
-  atomicExch(&sh->abort_flag, 1u);
+  give_up2(sh, counters, site);
   return false;
 }
 
@@ -114,114 +119,204 @@ __device__ __forceinline__ void set_max_regs_dec() {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
 }
 
-__device__ __forceinline__ uint32_t bf16_bits(float v) {
-  return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v));
-}
-
-__device__ __forceinline__ void st_global_b16(__nv_bfloat16* p, uint32_t bits) {
-  asm volatile("st.global.b16 [%0], %1;" ::"l"(p), "h"((unsigned short)bits) : "memory");
-}
-
-// What an epilogue thread keeps of a sub-tile between its gate pass and its combine pass.
-// A warp handles the 16-pixel pieces pg, pg+4, pg+8, pg+12 of the sub-tile (q = 0..3); lane l of
-// 32-lane group g stands for pixel l%16 of piece q = 2g + l/16.
-struct Keep {
-  uint32_t dbits[2];     // [g] gate decisions of this thread's channel, bit = lane slot of the pixel
-  uint32_t off[2];       // [g] element offset of this lane's pixel row in y (m * c_out), ~0u if padding
+// Folded per-channel constants of the four channels an epilogue thread sees in the fragment
+// layout: channels ch0 + 8*ci + lane/4, ci = 0..3, of the warp's 32.
+struct Consts4 {
+  float kt[4], ka1[4], kb1[4], ka2[4], kb2[4];
 };
 
-// 32 x 32 bit transpose across the warp: in, lane L holds bit p = value(L, p); out, lane p holds
-// bit L = value(L, p).
-__device__ __forceinline__ uint32_t warp_bit_transpose(uint32_t x, int lane) {
+// What an epilogue thread keeps of a sub-tile between its gate pass and its combine pass.  Lane l
+// of 32-lane group g stands for pixel l%16 of the warp's piece 2g + l/16.
+struct Keep {
+  uint32_t off[2];       // [g] output pixel index m of this lane's column, ~0u if padding
+  uint32_t fired;        // a gate fired in one of the warp's pieces
+};
+
+constexpr int kTilePitch = 80;                    // bytes per pixel row of a warp's staging tile (64 + 16: no bank conflicts)
+constexpr int kEpiTileBytes = 16 * kTilePitch;    // 16 pixels x 32 channels of bf16
+constexpr uint32_t kOpen = 0xffffu;               // bf16 pattern that marks "gate open" in y between the two passes:
+                                                  // a negative NaN, which max(v, lo) never yields
+
+// Output pixel index of this lane's column for both 32-lane groups (~0u: a pad position).
+__device__ __forceinline__ void pixel_offsets(const LayerDims& L, const Tc2Plan& P, int gx, int pg, int lane, Keep& kp) {
+  const int pieces = P.nmma >> 4;
 #pragma unroll
-  for (int k = 16; k >= 1; k >>= 1) {
-    const uint32_t m = k == 16 ? 0x0000ffffu : k == 8 ? 0x00ff00ffu : k == 4 ? 0x0f0f0f0fu : k == 2 ? 0x33333333u : 0x55555555u;
-    const uint32_t y = __shfl_xor_sync(0xffffffffu, x, k);
-    x = (lane & k) ? (((y >> k) & m) | (x & ~m)) : ((x & m) | ((y & m) << k));
+  for (int g = 0; g < 2; ++g) {
+    const int pc = pg + 4 * (2 * g + (lane >> 4));
+    const int j = pc * 16 + (lane & 15);
+    uint32_t off = ~0u;
+    if (pc < pieces && j < P.np) {
+      // (exact for these small non-negative integers: the quotient of (x + 0.5) / d never sits
+      // within 2^-12 of an integer)
+      const int dj = (int)(((float)j + 0.5f) * P.inv_wp);
+      const int gr = gx + dj, w = j - dj * P.wp;
+      const int n = (int)(((float)gr + 0.5f) * P.inv_hp), h = gr - n * P.hp;
+      if (w < L.wo && h < L.ho && n < L.n) off = (uint32_t)((n * L.ho + h) * L.wo + w);
+    }
+    kp.off[g] = off;
   }
-  return x;
 }
 
-// One pass of an epilogue warp over its pieces of a sub-tile (TMEM columns from t_cols on).
-//   gate pass (kCombine = false), Eq. 2/3 and Eq. 1's first case: d = (P >= t), collected per
-//   channel and transposed across the warp into the pixels' mask words; y = f(a1*P + b1) is stored
-//   where d = 0.
-//   combine pass (kCombine = true), Eq. 1's second case: y = f(a2*(P+R) + b2) stored where d = 1.
-// Every output element is written exactly once, by the pass that owns its case, straight from the
-// registers (32 consecutive channels of a pixel = one 64-byte segment per warp store): the
-// shared-memory bandwidth that the MMAs leave is too scarce for a staging tile.
-template <bool kCombine, bool kHasRes>
-__device__ __forceinline__ void epi_pass(const Tc2Params& prm, Keep& kp, uint32_t t_cols, int gx, int pg,
-                                         int lane, int word_idx, float kt, float ka, float kb, float lo,
-                                         __nv_bfloat16* y_ch, const __nv_bfloat16* res_ch,
-                                         unsigned long long& st_active, unsigned long long& st_words,
-                                         unsigned long long& st_words_on, bool& fired) {
+// The warp's 16 pixels x 32 channels, as packed bf16 pairs pk[ci][octet] in the fragment layout
+// of the 16x256b TMEM load, go into the staging tile pixel-major: afterwards lane l finds eight
+// consecutive channels of a pixel (16 bytes) at vector_at(l) and vector_at(l + 32).
+__device__ __forceinline__ void transpose_piece(const uint32_t (&pk)[4][2], uint8_t* s_tile, int lane) {
+  // thread 8*i + j gives the address of pixel row j, channels 8*i..8*i+7
+  const uint32_t row_addr = ptx::smem_u32(s_tile + (lane & 7) * kTilePitch + (lane >> 3) * 16);
+  ptx::stmatrix_x4_trans(row_addr, pk[0][0], pk[1][0], pk[2][0], pk[3][0]);
+  ptx::stmatrix_x4_trans(row_addr + 8 * kTilePitch, pk[0][1], pk[1][1], pk[2][1], pk[3][1]);
+  __syncwarp();
+}
+__device__ __forceinline__ uint4 vector_at(const uint8_t* s_tile, int vidx) {   // pixel vidx/4, channels 8*(vidx%4)..
+  return *(const uint4*)(s_tile + (vidx >> 2) * kTilePitch + (vidx & 3) * 16);
+}
+// per 16-bit half: 0xffff where the half of v is the "gate open" mark, else 0
+__device__ __forceinline__ uint32_t open_halves(uint32_t v) { return __vcmpeq2(v, 0xffffffffu); }
+
+// Gate pass of one warp over its pieces of a sub-tile (Eq. 2, 3 and Eq. 1's first case):
+// d = (P >= t).  Where d = 0 the output f(a1*P + b1) is final; where d = 1 the "gate open" mark
+// is written in its place.  A piece goes through the staging tile to y as 16-byte vectors, and
+// the lane that stores a vector reads the eight decisions off it for the pixel's mask word.
+template <bool kHasRes>
+__device__ __forceinline__ void gate_pass(const Tc2Params& prm, Keep& kp, const Consts4& kc, uint32_t t_acc,
+                                          int gx, int pg, int lane, int word_idx, float lo, __nv_bfloat16* y_q,
+                                          const __nv_bfloat16* res_q, uint8_t* s_tile, unsigned long long& st_active,
+                                          unsigned long long& st_words, unsigned long long& st_words_on) {
   const LayerDims& L = prm.L;
   const Tc2Plan& P = prm.P;
   const int pieces = P.nmma >> 4;
-  if (!kCombine) {
-#pragma unroll
-    for (int g = 0; g < 2; ++g) {
-      // y offset of this lane's pixel of the group
-      const int pc = pg + 4 * (2 * g + (lane >> 4));
-      const int j = pc * 16 + (lane & 15);
-      uint32_t off = ~0u;
-      if (pc < pieces && j < P.np) {
-        // (exact for these small non-negative integers: the quotient of (x + 0.5) / d never sits
-        // within 2^-12 of an integer)
-        const int dj = (int)(((float)j + 0.5f) * P.inv_wp);
-        const int gr = gx + dj, w = j - dj * P.wp;
-        const int n = (int)(((float)gr + 0.5f) * P.inv_hp), h = gr - n * P.hp;
-        if (w < L.wo && h < L.ho && n < L.n) off = (uint32_t)((n * L.ho + h) * L.wo + w) * (uint32_t)L.c_out;
-      }
-      kp.off[g] = off;
-      kp.dbits[g] = 0u;
-    }
-  }
+  pixel_offsets(L, P, gx, pg, lane, kp);
+  bool fired = false;
 #pragma unroll 1
   for (int q = 0; q < 4; ++q) {
     const int piece = pg + 4 * q;
     if (piece >= pieces) break;                              // (uniform over the warp)
     const int slot0 = (q & 1) * 16;
     const uint32_t offs = (q >> 1) ? kp.off[1] : kp.off[0];
-    const uint32_t bits = ((q >> 1) ? kp.dbits[1] : kp.dbits[0]) >> slot0;
-    uint32_t v[16];
-    ptx::tmem_ld_nowait<16>(t_cols + (uint32_t)(piece * 16), v);
-    ptx::tmem_ld_wait<16>(v);
-    uint32_t newbits = 0u;
+    uint32_t r0[8], r1[8];                                   // channels 0-15 / 16-31 of the quadrant
+    ptx::tmem_ld_frag16(t_acc + (uint32_t)(piece * 16), r0);
+    ptx::tmem_ld_frag16(t_acc + (16u << 16) + (uint32_t)(piece * 16), r1);
+    ptx::tmem_ld_wait16(r0, r1);
+    uint32_t pk[4][2];
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      const uint32_t oj = __shfl_sync(0xffffffffu, offs, slot0 + j);
-      const float a = __uint_as_float(v[j]);
-      bool d;
-      if (!kCombine) {
-        d = a >= kt;                                         // Eq. 2: a tie fires, NaN does not
-        if (d) newbits |= 1u << j;
-      } else {
-        d = (bits >> j) & 1u;
+    for (int ci = 0; ci < 4; ++ci) {
+#pragma unroll
+      for (int oct = 0; oct < 2; ++oct) {
+        float yv[2];
+        bool d[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const float a = __uint_as_float((ci >> 1) ? r1[4 * oct + 2 * (ci & 1) + e] : r0[4 * oct + 2 * (ci & 1) + e]);
+          d[e] = a >= kc.kt[ci];                             // Eq. 2: a tie fires, NaN does not
+          float v = fmaf(kc.ka1[ci], a, kc.kb1[ci]);         // BN1 of the partial sum (Section 4)
+          if (kHasRes) {
+            const uint32_t oj = __shfl_sync(0xffffffffu, offs, slot0 + 8 * oct + 2 * (lane & 3) + e);
+            if (oj != ~0u) v += __bfloat162float(res_q[(size_t)oj * L.c_out + 8 * ci + (lane >> 2)]);
+          }
+          yv[e] = fmaxf(v, lo);
+        }
+        const __nv_bfloat162 h2 = __floats2bfloat162_rn(yv[0], yv[1]);
+        uint32_t w = *(const uint32_t*)&h2;
+        if (d[0]) w |= kOpen;
+        if (d[1]) w |= kOpen << 16;
+        pk[ci][oct] = w;
       }
-      float yv = fmaf(ka, a, kb);                            // the batch norm of the path (Section 4)
-      if (kHasRes && oj != ~0u) yv += __bfloat162float(res_ch[oj]);
-      yv = fmaxf(yv, lo);
-      if (oj != ~0u && d == kCombine) st_global_b16(y_ch + oj, bf16_bits(yv));
     }
-    if (!kCombine) {
-      if (q >> 1) kp.dbits[1] |= newbits << slot0; else kp.dbits[0] |= newbits << slot0;
+    transpose_piece(pk, s_tile, lane);
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int vidx = lane + 32 * k;
+      const uint32_t oj = __shfl_sync(0xffffffffu, offs, slot0 + (vidx >> 2));
+      const uint4 val = vector_at(s_tile, vidx);
+      // decisions of the vector's eight channels, one bit each
+      const uint32_t t = (open_halves(val.x) & 0x00020001u) | (open_halves(val.y) & 0x00080004u) |
+                         (open_halves(val.z) & 0x00200010u) | (open_halves(val.w) & 0x00800040u);
+      uint32_t word = ((t | (t >> 16)) & 0xffu) << (8 * (lane & 3));
+      word |= __shfl_xor_sync(0xffffffffu, word, 1);
+      word |= __shfl_xor_sync(0xffffffffu, word, 2);
+      if (oj != ~0u) {
+        *(uint4*)(y_q + (size_t)oj * L.c_out + (vidx & 3) * 8) = val;
+        if ((lane & 3) == 0) {
+          if (prm.mask) prm.mask[(size_t)oj * L.words + word_idx] = word;
+          st_active += __popc(word);
+          st_words += 1;
+          if (word) { st_words_on += 1; fired = true; }
+        }
+      }
     }
+    __syncwarp();
   }
-  if (!kCombine) {
-    // mask words: lane l gets the decisions of all 32 channels for pixel slot l of each group
+  kp.fired = __any_sync(0xffffffffu, fired) ? 1u : 0u;
+}
+
+// Combine pass (Eq. 1's second case): f(a2*(P+R) + b2) replaces the "gate open" marks the gate
+// pass left in y; vectors without a mark are left alone.  The thread that stores a vector here
+// stored the same vector in the gate pass, so it reads back its own write.
+template <bool kHasRes>
+__device__ __forceinline__ void combine_pass(const Tc2Params& prm, const Keep& kp, const Consts4& kc, uint32_t t_acc,
+                                             int pg, int lane, float lo, __nv_bfloat16* y_q,
+                                             const __nv_bfloat16* res_q, uint8_t* s_tile) {
+  const LayerDims& L = prm.L;
+  const Tc2Plan& P = prm.P;
+  const int pieces = P.nmma >> 4;
+  if (!kp.fired) return;                                     // (uniform over the warp: no mark in its pieces)
+#pragma unroll 1
+  for (int q = 0; q < 4; ++q) {
+    const int piece = pg + 4 * q;
+    if (piece >= pieces) break;
+    const int slot0 = (q & 1) * 16;
+    const uint32_t offs = (q >> 1) ? kp.off[1] : kp.off[0];
+    // what the gate pass left, requested first: the loads travel while the new values are made
+    uint4 old[2];
+    uint4* dst[2];
 #pragma unroll
-    for (int g = 0; g < 2; ++g) {
-      if (pg + 8 * g >= pieces) break;
-      const uint32_t word = warp_bit_transpose(kp.dbits[g], lane);
-      if (kp.off[g] != ~0u) {
-        if (prm.mask) prm.mask[(size_t)(kp.off[g] / (uint32_t)L.c_out) * L.words + word_idx] = word;
-        st_active += __popc(word);
-        st_words += 1;
-        if (word) { st_words_on += 1; fired = true; }
+    for (int k = 0; k < 2; ++k) {
+      const int vidx = lane + 32 * k;
+      const uint32_t oj = __shfl_sync(0xffffffffu, offs, slot0 + (vidx >> 2));
+      dst[k] = oj != ~0u ? (uint4*)(y_q + (size_t)oj * L.c_out + (vidx & 3) * 8) : nullptr;
+      old[k] = make_uint4(0u, 0u, 0u, 0u);
+      if (dst[k]) old[k] = *dst[k];
+    }
+    uint32_t r0[8], r1[8];
+    ptx::tmem_ld_frag16(t_acc + (uint32_t)(piece * 16), r0);
+    ptx::tmem_ld_frag16(t_acc + (16u << 16) + (uint32_t)(piece * 16), r1);
+    ptx::tmem_ld_wait16(r0, r1);
+    uint32_t pk[4][2];
+#pragma unroll
+    for (int ci = 0; ci < 4; ++ci) {
+#pragma unroll
+      for (int oct = 0; oct < 2; ++oct) {
+        float yv[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const float a = __uint_as_float((ci >> 1) ? r1[4 * oct + 2 * (ci & 1) + e] : r0[4 * oct + 2 * (ci & 1) + e]);
+          float v = fmaf(kc.ka2[ci], a, kc.kb2[ci]);         // BN2 of the full sum P + R
+          if (kHasRes) {
+            const uint32_t oj = __shfl_sync(0xffffffffu, offs, slot0 + 8 * oct + 2 * (lane & 3) + e);
+            if (oj != ~0u) v += __bfloat162float(res_q[(size_t)oj * L.c_out + 8 * ci + (lane >> 2)]);
+          }
+          yv[e] = fmaxf(v, lo);
+        }
+        const __nv_bfloat162 h2 = __floats2bfloat162_rn(yv[0], yv[1]);
+        pk[ci][oct] = *(const uint32_t*)&h2;
       }
     }
+    transpose_piece(pk, s_tile, lane);
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const uint4 nw = vector_at(s_tile, lane + 32 * k);
+      const uint32_t mx = open_halves(old[k].x), my = open_halves(old[k].y), mz = open_halves(old[k].z),
+                     mw = open_halves(old[k].w);
+      if (dst[k] && ((mx | my) | (mz | mw))) {
+        uint4 out;
+        out.x = (nw.x & mx) | (old[k].x & ~mx);
+        out.y = (nw.y & my) | (old[k].y & ~my);
+        out.z = (nw.z & mz) | (old[k].z & ~mz);
+        out.w = (nw.w & mw) | (old[k].w & ~mw);
+        *dst[k] = out;
+      }
+    }
+    __syncwarp();
   }
 }
 
@@ -280,7 +375,7 @@ tc2_gated_conv_kernel(const __grid_constant__ CUtensorMap map_r1,
     // loaded stacked row; no copy ever writes them
     const int et = threadIdx.x - kEpiWarp0 * 32;
     const int n16 = L.pad * 8;                              // 16-byte pieces per buffer
-    for (int i = et; i < kPatchEntries * n16; i += kEpiWarps * 32)
+    for (int i = et; i < P.entries * n16; i += kEpiWarps * 32)
       *(uint4*)(s_p + (size_t)(i / n16) * P.patch_bytes + (size_t)(i % n16) * 16) = make_uint4(0, 0, 0, 0);
     ptx::fence_proxy_async();
   }
@@ -354,7 +449,7 @@ tc2_gated_conv_kernel(const __grid_constant__ CUtensorMap map_r1,
                 ptx::tma_load_4d(base + sh->box_dst[i], mp, &sh->p_full[slot], chunk * 64, 0, sh->box_h[i], sh->box_n[i]);
               }
               __syncwarp();
-              if (++slot == kPatchEntries) { slot = 0; par ^= 1u; }
+              if (++slot == P.entries) { slot = 0; par ^= 1u; }
             }
           }
         }
@@ -444,7 +539,7 @@ tc2_gated_conv_kernel(const __grid_constant__ CUtensorMap map_r1,
                 ok = wait2(cx, &sh->p_full[entry], ppar, 15 + X);
                 if (!ok) break;
                 pnext += P.nsub;
-                if (pnext >= kPatchEntries) { pnext -= kPatchEntries; ppar ^= 1u; }
+                if (pnext >= P.entries) { pnext -= P.entries; ppar ^= 1u; }
                 b_lo = p_lo0 + (uint32_t)entry * p_step;
               }
             }
@@ -485,23 +580,31 @@ tc2_gated_conv_kernel(const __grid_constant__ CUtensorMap map_r1,
     }
     __syncwarp();
   } else {
-    // ============================================================ epilogue: thread = channel
+    // ============================================================ epilogue
+    // A warp owns one TMEM lane quadrant (32 channels) and every fourth 16-pixel piece of a
+    // sub-tile; it reads the accumulators in the 16x256b fragment layout, where a thread holds
+    // four channels x four pixels of a piece.
     const int quad = warp & 3;
     const int pg = (warp - kEpiWarp0) >> 2;
-    const int ch = tile_c * 128 + quad * 32 + lane;
-    const bool ch_valid = tile_c * 128 + quad * 32 < L.c_out;     // (uniform over the warp)
-    float kt = 0.f, ka1 = 0.f, kb1 = 0.f, ka2 = 0.f, kb2 = 0.f;
-    if (ch_valid && jobs > 0) {
-      const ChannelConsts k = fold_channel(prm.bn, prm.delta, L.eps, ch);
-      kt = k.t; ka1 = k.a1; kb1 = k.b1; ka2 = k.a2; kb2 = k.b2;
+    const int ch0 = tile_c * 128 + quad * 32;
+    const bool ch_valid = ch0 < L.c_out;                      // (uniform over the warp; c_out is a multiple of 32)
+    Consts4 kc;
+#pragma unroll
+    for (int ci = 0; ci < 4; ++ci) {
+      kc.kt[ci] = 0.f; kc.ka1[ci] = 0.f; kc.kb1[ci] = 0.f; kc.ka2[ci] = 0.f; kc.kb2[ci] = 0.f;
+      if (ch_valid && jobs > 0) {
+        const ChannelConsts k = fold_channel(prm.bn, prm.delta, L.eps, ch0 + 8 * ci + (lane >> 2));
+        kc.kt[ci] = k.t; kc.ka1[ci] = k.a1; kc.kb1[ci] = k.b1; kc.ka2[ci] = k.a2; kc.kb2[ci] = k.b2;
+      }
     }
     const float lo = L.relu ? 0.f : -__int_as_float(0x7f800000);   // f = ReLU, or the identity
     const uint32_t t_lane = tmem + ((uint32_t)(quad * 32) << 16);
     const int word_idx = tile_c * 4 + quad;
-    __nv_bfloat16* y_ch = prm.y + ch;
-    const __nv_bfloat16* res_ch = kHasRes ? prm.residual + ch : nullptr;
+    __nv_bfloat16* y_q = prm.y + ch0;
+    const __nv_bfloat16* res_q = kHasRes ? prm.residual + ch0 : nullptr;
+    uint8_t* s_tile = smem + P.off_epi + (warp - kEpiWarp0) * kEpiTileBytes;
     unsigned long long st_active = 0, st_words = 0, st_words_on = 0;
-    Keep keep0 = {{0u, 0u}, {~0u, ~0u}}, keep1 = keep0;
+    Keep keep0 = {{~0u, ~0u}, 0u}, keep1 = keep0;
     bool ok = true;
     for (int jb = 0; jb < jobs && ok; ++jb) {
       const uint32_t par = (uint32_t)jb & 1u;
@@ -515,21 +618,18 @@ tc2_gated_conv_kernel(const __grid_constant__ CUtensorMap map_r1,
         ok = wait2(cx, comb ? &sh->cond_done[X] : &sh->base_done[X], par, 20 + e);
         if (!ok) break;
         ptx::tc_fence_after();
-        const uint32_t t_cols = t_lane + (uint32_t)(X * 256);
+        const uint32_t t_acc = t_lane + (uint32_t)(X * 256);
         Keep kx = X ? keep1 : keep0;
-        bool fired = false;
         if (ch_valid) {
           if (!comb)
-            epi_pass<false, kHasRes>(prm, kx, t_cols, g0 + X * P.r, pg, lane, word_idx, kt, ka1, kb1, lo, y_ch, res_ch,
-                                     st_active, st_words, st_words_on, fired);
+            gate_pass<kHasRes>(prm, kx, kc, t_acc, g0 + X * P.r, pg, lane, word_idx, lo, y_q, res_q, s_tile, st_active,
+                               st_words, st_words_on);
           else
-            epi_pass<true, kHasRes>(prm, kx, t_cols, g0 + X * P.r, pg, lane, word_idx, kt, ka2, kb2, lo, y_ch, res_ch,
-                                    st_active, st_words, st_words_on, fired);
+            combine_pass<kHasRes>(prm, kx, kc, t_acc, pg, lane, lo, y_q, res_q, s_tile);
         }
         if (!comb) {
           if (X) keep1 = kx; else keep0 = kx;
-          const bool any_fired = __any_sync(0xffffffffu, fired);
-          if (lane == 0) sh->fired[X][warp - kEpiWarp0] = any_fired ? 1u : 0u;
+          if (lane == 0) sh->fired[X][warp - kEpiWarp0] = ch_valid ? kx.fired : 0u;
         }
         ptx::tc_fence_before();
         __syncwarp();
@@ -741,11 +841,19 @@ bool tc2_plan(const LayerDims& L, int in_dtype, int cond_mode, int sms, Tc2Plan*
         const int runs = P.use_img ? 2 : box_rows / P.hp + 2;
         if (runs * per_run + images + 4 > kMaxBoxes) continue;
       }
-      const size_t fixed = kPatchEntries * patch_bytes + bar_bytes + (P.w_rows < 128 ? 128 * 128 : 0) +
-                           kTc2MaxStages * sizeof(Tc2Stage);   // (+ slack behind a ring of narrow tiles)
+      // shared memory: patch entries (three, so that the next input-channel chunk of a sub-tile
+      // loads while the current one is read; two where that leaves the weight ring too short),
+      // staging tiles, stage table, barriers; the rest is the weight ring
       const int min_ring = nsub == 2 ? 5 : 3;
-      if (fixed + (size_t)min_ring * P.w_stage_bytes > limit) continue;
-      int ring = (int)((limit - fixed) / P.w_stage_bytes);
+      int entries = 0, ring = 0;
+      for (int en = kPatchEntries; en >= 2 && entries == 0; --en) {
+        const size_t fixed = en * patch_bytes + bar_bytes + (P.w_rows < 128 ? 128 * 128 : 0) +
+                             kTc2MaxStages * sizeof(Tc2Stage) + (size_t)kEpiWarps * 1280;
+        if (fixed + (size_t)min_ring * P.w_stage_bytes > limit) continue;
+        entries = en;
+        ring = (int)((limit - fixed) / P.w_stage_bytes);
+      }
+      if (entries == 0) continue;
       if (ring > kMaxRing) ring = kMaxRing;
       int lead = nsub == 2 ? ring - 3 : 0;
       if (lead > 4) lead = 4;
@@ -764,14 +872,15 @@ bool tc2_plan(const LayerDims& L, int in_dtype, int cond_mode, int sms, Tc2Plan*
         best = est;
         P.r = r; P.nsub = nsub; P.np = np; P.nmma = nmma; P.jobs_m = (int)jobs_m;
         P.patch_rows = patch_rows; P.patch_bytes = (int)patch_bytes; P.patch_box_rows = r + 2 * L.pad;
-        P.ring = ring; P.lead = lead; P.grid = grid;
+        P.ring = ring; P.entries = entries; P.lead = lead; P.grid = grid;
       }
     }
   }
   if (best >= 1e299) return false;
   size_t off = 0;
   P.off_w = (unsigned)off; off += align_up2((size_t)P.ring * P.w_stage_bytes + (P.w_rows < 128 ? 128 * 128 : 0), 1024);
-  P.off_p = (unsigned)off; off += (size_t)kPatchEntries * P.patch_bytes;
+  P.off_p = (unsigned)off; off += (size_t)P.entries * P.patch_bytes;
+  P.off_epi = (unsigned)off; off += (size_t)kEpiWarps * kEpiTileBytes;
   P.off_tab = (unsigned)off; off += (size_t)kTc2MaxStages * sizeof(Tc2Stage);
   P.off_bar = (unsigned)off; off += bar_bytes;
   P.smem_bytes = (unsigned)(off + 1024);

@@ -44,6 +44,7 @@ struct Tc2Plan {
   int chunks;            // c_in / 64
   int nb, ns;            // base-path stages, all stages
   int ring;              // weight ring depth in stages
+  int entries;           // patch buffers: 2 or 3
   int lead;              // stages by which sub-tile a runs ahead of sub-tile b
   int w_rows;            // channels per weight tile: min(128, c_out)
   int w_stage_bytes;     // w_rows * 128
@@ -54,7 +55,7 @@ struct Tc2Plan {
   int pad8;              // c_p = 8: the weights are repacked into the workspace with whole K steps
   int use_img;           // whole images are loaded by single copies (small images)
   int grid;
-  unsigned off_w, off_p, off_tab, off_bar, smem_bytes;
+  unsigned off_w, off_p, off_epi, off_tab, off_bar, smem_bytes;
   Tc2Stage st[kTc2MaxStages];
 };
 
