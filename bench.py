@@ -376,6 +376,73 @@ def run_block(block, args, peaks, rank):
     return out
 
 
+def run_network_block(args, peaks):
+    """Whole CG-ResNet-18 forward pass (batch 128, 224 x 224, G = 4) at the gate density that gives a
+    2.8x reduction of the network's multiplications, and the same network with every gate open."""
+    import torch
+    from paper_1805_12549_b200 import resnet18 as R
+    batch, reduction = 128, 2.8
+    net = R.CgResNet18(groups=4, cond_mode=args.cond_mode)
+    gated, other = net.macs_per_image()
+    tau = R.density_for_reduction(reduction, 4, gated, other)
+    x = R.synthetic_images("bench_resnet18", batch)
+    net.calibrate(x[:CALIB_IMAGES].contiguous(), tau)
+    inst = net.instance(batch)
+    stream = torch.cuda.current_stream()
+
+    def timed(reps):
+        inst.forward(x)
+        torch.cuda.synchronize()
+        g = capture(lambda: inst.forward(x), args.no_graph)
+        g.replay()
+        torch.cuda.synchronize()
+        inst.stats()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            g.replay()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        _, summary = inst.stats()
+        return e0.elapsed_time(e1) / reps, summary
+
+    reps = 10
+    ms, summ = timed(reps)
+    events = []
+    for _ in range(3):
+        inst.forward(x, events=events)
+    torch.cuda.synchronize()
+    inst.stats()
+    per_op = {}
+    for name, e0, e1 in events:
+        per_op[name] = per_op.get(name, 0.0) + e0.elapsed_time(e1) / 3
+    gated_names = {s.name for s in net.gated_specs}
+    net.set_density(1.0)
+    ms1, summ1 = timed(reps)
+    net.set_density(tau)
+    out = {
+        "workload": "cg_resnet18_forward", "batch": batch, "image": 224, "groups": 4, "dtype": "bf16",
+        "target_flop_reduction": reduction, "target_density": round(tau, 4),
+        "calibration": f"layer by layer on the first {CALIB_IMAGES} images",
+        "ms_per_forward": round(ms, 4), "images_per_s": round(batch / (ms * 1e-3), 1),
+        "ms_per_forward_density1": round(ms1, 4), "images_per_s_density1": round(batch / (ms1 * 1e-3), 1),
+        "speedup_vs_density1": round(ms1 / ms, 3),
+        "flop_reduction": round(summ["flop_reduction"], 3),
+        "gated_layer_density": round(summ["gated_layer_density"], 4),
+        "executed_over_gated": round(summ["executed_macs"] / max(summ["gated_macs"], 1), 3),
+        "gated_tflops": round(2.0 * summ["gated_macs"] / (ms * 1e-3) / 1e12, 1),
+        "dense_tflops_density1": round(2.0 * summ1["dense_macs"] / (ms1 * 1e-3) / 1e12, 1),
+        "launches_per_forward": inst.launches_per_forward(),
+        "ms_gated_layers": round(sum(v for k, v in per_op.items() if k in gated_names), 4),
+        "ms_other_operators": round(sum(v for k, v in per_op.items() if k not in gated_names), 4),
+        "ms_per_operator": {k: round(v, 4) for k, v in per_op.items()},
+        "kernels": {s.name: ["direct", "tcgen05 pixel-major", "tcgen05 channel-major"][inst.convs[s.name].kernel_id]
+                    for s in net.specs},
+    }
+    inst.close()
+    return out
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -490,6 +557,8 @@ def run_ours(args):
         for block in EXTRA_BLOCKS:
             blocks.append(run_block(block, args, peaks, rank))
             torch.cuda.empty_cache()
+        blocks.append(run_network_block(args, peaks))
+        torch.cuda.empty_cache()
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:

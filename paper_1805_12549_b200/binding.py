@@ -24,6 +24,8 @@ EXPORTS = ("cg_conv_create", "cg_conv_workspace_bytes", "cg_conv_forward",
            "cg_conv_host_staging_bytes", "cg_conv_forward_host", "cg_conv_partial_sums",
            "cg_conv_stats", "cg_conv_launches_per_forward", "cg_conv_uses_tensor_cores",
            "cg_conv_kernel_id", "cg_conv_plan_string", "cg_conv_destroy", "cg_status_string", "cg_conv_forward_static")
+# include/cgnet.h: the ungated operators of a whole network
+NET_EXPORTS = ("cg_im2col_bf16", "cg_subsample_bf16", "cg_maxpool_bf16", "cg_avgpool_bf16")
 
 
 class CgConvDesc(C.Structure):
@@ -95,6 +97,15 @@ def lib():
                                              C.POINTER(CgStats), C.c_void_p]
         L.cg_status_string.restype = C.c_char_p
         L.cg_status_string.argtypes = [C.c_int]
+        i = C.c_int
+        L.cg_im2col_bf16.restype = C.c_int
+        L.cg_im2col_bf16.argtypes = [C.c_void_p, C.c_void_p, i, i, i, i, i, i, i, i, C.c_void_p]
+        L.cg_subsample_bf16.restype = C.c_int
+        L.cg_subsample_bf16.argtypes = [C.c_void_p, C.c_void_p, i, i, i, i, i, C.c_void_p]
+        L.cg_maxpool_bf16.restype = C.c_int
+        L.cg_maxpool_bf16.argtypes = [C.c_void_p, C.c_void_p, i, i, i, i, i, i, i, C.c_void_p]
+        L.cg_avgpool_bf16.restype = C.c_int
+        L.cg_avgpool_bf16.argtypes = [C.c_void_p, C.c_void_p, i, i, i, C.c_void_p]
         _lib = L
     return _lib
 
@@ -233,6 +244,30 @@ def cg_conv_plan_string(h) -> str:
     buf = C.create_string_buffer(512)
     lib().cg_conv_plan_string(h, buf, len(buf))
     return buf.value.decode()
+
+
+def cg_im2col_bf16(x, a, k, stride, pad, stream=None):
+    """x [n,h,w,c] -> a [n,h',w',k_pad] (include/cgnet.h)."""
+    n, h, w, c = x.shape
+    _check(lib().cg_im2col_bf16(_ptr(x), _ptr(a), n, h, w, c, k, stride, pad, a.shape[-1],
+                                _stream_ptr(stream)), "cg_im2col_bf16")
+
+
+def cg_subsample_bf16(x, y, stride, stream=None):
+    n, h, w, c = x.shape
+    _check(lib().cg_subsample_bf16(_ptr(x), _ptr(y), n, h, w, c, stride, _stream_ptr(stream)),
+           "cg_subsample_bf16")
+
+
+def cg_maxpool_bf16(x, y, k, stride, pad, stream=None):
+    n, h, w, c = x.shape
+    _check(lib().cg_maxpool_bf16(_ptr(x), _ptr(y), n, h, w, c, k, stride, pad, _stream_ptr(stream)),
+           "cg_maxpool_bf16")
+
+
+def cg_avgpool_bf16(x, y, stream=None):
+    n, h, w, c = x.shape
+    _check(lib().cg_avgpool_bf16(_ptr(x), _ptr(y), n, h * w, c, _stream_ptr(stream)), "cg_avgpool_bf16")
 
 
 class GatedConv:

@@ -11,8 +11,8 @@ from paper_1805_12549_b200 import binding as B
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
-def _declared_symbols():
-    text = open(os.path.join(ROOT, "include", "cgconv.h")).read()
+def _declared_symbols(header="cgconv.h"):
+    text = open(os.path.join(ROOT, "include", header)).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(cg_[a-z0-9_]+)\s*\(", text)))
 
@@ -24,6 +24,34 @@ def test_library_exports_every_declared_symbol():
     assert len(names) >= 11
     for n in names:
         assert hasattr(lib, n), n
+
+
+def test_library_exports_the_network_operators():
+    lib = B.lib()
+    names = _declared_symbols("cgnet.h")
+    assert set(names) == set(B.NET_EXPORTS)
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_network_operators_reject_bad_arguments_before_any_launch():
+    lib = B.lib()
+    buf = (C.c_uint8 * 4096)()
+    base = C.addressof(buf)
+    p = C.c_void_p((base + 15) & ~15)
+    odd = C.c_void_p(p.value + 2)
+    INVALID, ALIGN = 1, 3
+    assert lib.cg_im2col_bf16(None, p, 1, 8, 8, 3, 7, 2, 3, 152, None) == INVALID
+    assert lib.cg_im2col_bf16(p, p, 1, 8, 8, 3, 7, 2, 3, 144, None) == INVALID      # k_pad < 147
+    assert lib.cg_im2col_bf16(p, p, 1, 8, 8, 3, 7, 2, 3, 150, None) == INVALID      # not a multiple of 8
+    assert lib.cg_im2col_bf16(p, p, 1, 2, 2, 3, 7, 2, 0, 152, None) == INVALID      # filter larger than the image
+    assert lib.cg_im2col_bf16(odd, p, 1, 8, 8, 3, 7, 2, 3, 152, None) == ALIGN
+    assert lib.cg_subsample_bf16(p, p, 1, 8, 8, 12, 2, None) == INVALID             # channels not a multiple of 8
+    assert lib.cg_subsample_bf16(p, odd, 1, 8, 8, 16, 2, None) == ALIGN
+    assert lib.cg_maxpool_bf16(p, p, 1, 8, 8, 16, 3, 2, 3, None) == INVALID         # a window of padding only
+    assert lib.cg_maxpool_bf16(p, None, 1, 8, 8, 16, 3, 2, 1, None) == INVALID
+    assert lib.cg_avgpool_bf16(p, p, 0, 49, 16, None) == INVALID
+    assert lib.cg_avgpool_bf16(odd, p, 1, 49, 16, None) == ALIGN
 
 
 def test_status_strings():
