@@ -69,7 +69,8 @@ typedef struct {
   int32_t groups;               /* G = 1/eta (Section 3.1): the base path reads input channels
                                    [0, c_in/G), the conditional path the rest.  G = 1: ungated */
   int32_t in_dtype;             /* cg_dtype of x, w_base, w_cond                               */
-  int32_t out_dtype;            /* cg_dtype of y: F32 for F32, BF16 for BF16, I8 for I8        */
+  int32_t out_dtype;            /* cg_dtype of y, equal to in_dtype (a BF16 layer with I8
+                                   output is not built: CG_ERR_INVALID_ARG)                    */
   float bn_eps;                 /* added inside sqrt(var + eps) of BN1, BN2 and the gate       */
   int32_t relu;                 /* 1: f = ReLU (the paper's choice); 0: identity               */
   int32_t has_residual;         /* 1: `residual` [M,c_out] (out_dtype) is added after the batch
@@ -81,16 +82,17 @@ typedef struct {
                                    x_p (Fig. 5(a)).  1: channel grouping (Section 3.3, Fig. 5(b)):
                                    output group i = channels [i*c_out/G,(i+1)*c_out/G) takes input
                                    group i as x_p and the other groups, in ascending order, as
-                                   x_r; needs c_out % G == 0.  Direct kernels only for now.    */
+                                   x_r; needs c_out % G == 0.  Direct kernels only.            */
   float channel_tau;            /* tau_c of the channel-wise gate (Eq. 4).  0: off.  > 0: per
                                    image, an output channel whose gate fires at fewer than
                                    tau_c * h' * w' positions loses its conditional path (all its
                                    activations take Eq. 1's first case, its mask bits are 0);
                                    a count equal to tau_c*h'*w' keeps the channel (theta(0) = 1);
                                    the comparison is (float)count >= tau_c * (float)(h'*w').
-                                   Floating-point layers, direct kernels, three launches (partial
-                                   sums and counts, decisions, conditional path); needs the
-                                   workspace cg_conv_workspace_bytes reports.                  */
+                                   Floating-point layers, direct kernels only: a memset of the
+                                   counts and two launches (partial sums and counts; decisions
+                                   and conditional path); needs the workspace
+                                   cg_conv_workspace_bytes reports.                            */
 } cg_conv_desc;
 
 /* Per-output-channel parameters: DEVICE pointers to c_out entries, caller-owned.
@@ -137,13 +139,27 @@ typedef struct {
 /* Section 3.1: fixes the layer and picks kernels.  Host work only, plus one small device
  * allocation for the counters (freed by cg_conv_destroy).  `*out` is set on CG_OK only.
  * Errors: CG_ERR_INVALID_ARG (NULL, extents <= 0, c_in % groups != 0, kh != kw, dtype pair not
- * listed above, shift out of range), CG_ERR_UNSUPPORTED (algo = TENSOR on a layer outside
- * its limits: bf16/int8 only, c_in/groups a multiple of 16 bytes of elements, c_out a
- * multiple of 16), CG_ERR_CUDA. */
+ * listed above, shift out of range), CG_ERR_CUDA, and CG_ERR_UNSUPPORTED when a tensor-core
+ * algo is asked for a layer outside the kernels' limits.  Those are: BF16 or I8; no channel
+ * grouping, no channel-wise gate; odd square filter with pad = (k-1)/2; c_in a multiple of 64
+ * (BF16) or 128 (I8);
+ *   pixel-major kernel:   stride 1, or stride 2 for 3x3 filters on even extents; c_out a multiple
+ *                         of 64 (BF16) or 128 (I8); c_in/G equal to 16 or 32 (BF16; 32 or 64 for
+ *                         I8) or a multiple of 64 (128); output width at most 128;
+ *   channel-major kernel: BF16, stride 1, c_out a multiple of 32, c_in/G equal to 8, 16, 32 or a
+ *                         multiple of 64, no row compaction (CG_COND_COMPACT).
+ * AUTO falls back to the direct kernels outside these limits.
+ * A handle is not thread-safe: calls on one handle must not overlap in time on the host
+ * (different handles are independent).  Forward calls of one handle may be queued on different
+ * streams only if the streams are ordered so that they do not run concurrently: the counters and
+ * the workspace are per handle. */
 cg_status cg_conv_create(cg_conv_t* out, const cg_conv_desc* desc);
 
-/* Bytes of device scratch cg_conv_forward needs (may be 0).  Contents need not persist
- * between calls; two forwards that overlap in time must not share one workspace. */
+/* Bytes of device scratch cg_conv_forward needs (may be 0): the partial sums and per-channel
+ * counts of the channel-wise gate (Eq. 4), the compacted row lists of CG_COND_COMPACT (Eq. 1: the
+ * rows where d = 1), or weights repacked for c_in/G = 8.  Contents need not persist between
+ * calls; two forwards that overlap in time must not share one workspace.  The pointer given to
+ * cg_conv_forward must be 256-byte aligned (CG_ERR_ALIGNMENT otherwise). */
 size_t cg_conv_workspace_bytes(cg_conv_t h);
 
 /* Eq. 1-3 and the two batch norms of Section 4 for one batch.
@@ -153,7 +169,8 @@ size_t cg_conv_workspace_bytes(cg_conv_t h);
  *   bn        host struct of device pointers (read during the call, not kept)
  *   delta     [c_out] float, Delta of Eq. 3 in normalised units, +-inf allowed (all shut /
  *             all open); ignored (may be NULL) for I8, which uses bn->q_gate_thr
- *   residual  [M,c_out] out_dtype or NULL (must be NULL unless has_residual)
+ *   residual  [M,c_out] out_dtype or NULL (must be NULL unless has_residual); must not overlap y
+ *             (the kernels write y before they have read all of residual)
  *   y         [n,h',w',c_out] out_dtype
  *   mask_out  d of Section 3.1, one bit per activation: bit (c & 31) of 32-bit word
  *             m*ceil(c_out/32) + (c >> 5), m the pixel row; unused high bits 0.  NULL: not

@@ -13,6 +13,7 @@
 #include <cstring>
 
 #include "common.cuh"
+#include "direct_point.cuh"
 
 namespace cg {
 namespace {
@@ -28,14 +29,6 @@ static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];
 constexpr int kMaxDevices = 64;
 void* g_scratch_addr[kMaxDevices];   // per device, filled on the first call with that device current
 
-template <typename T> __device__ __forceinline__ float ld_f(const T* p);
-template <> __device__ __forceinline__ float ld_f<float>(const float* p) { return *p; }
-template <> __device__ __forceinline__ float ld_f<__nv_bfloat16>(const __nv_bfloat16* p) {
-  return __bfloat162float(*p);
-}
-__device__ __forceinline__ void st_f(float* p, float v) { *p = v; }
-__device__ __forceinline__ void st_f(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
-
 // Prologue: clear the counters left by the previous call and fold the channel constants.
 __global__ void static_prologue_kernel(cg_bn_params bn, const float* delta, float eps, int c_out,
                                        unsigned long long* counters, float* consts) {
@@ -49,25 +42,6 @@ __global__ void static_prologue_kernel(cg_bn_params bn, const float* delta, floa
     consts[3 * c_out + i] = k.a2;
     consts[4 * c_out + i] = k.b2;
   }
-}
-
-template <typename T>
-__device__ __forceinline__ float conv_sum(const LayerDims& L, const T* __restrict__ x,
-                                          const T* __restrict__ w, int n, int ho, int wo, int co,
-                                          int c_lo, int cw) {
-  float acc = 0.f;
-  for (int r = 0; r < L.kh; ++r) {
-    const int hi = ho * L.stride + r - L.pad;
-    if (hi < 0 || hi >= L.h) continue;
-    for (int s = 0; s < L.kw; ++s) {
-      const int wi = wo * L.stride + s - L.pad;
-      if (wi < 0 || wi >= L.w) continue;
-      const T* xp = x + (((long long)n * L.h + hi) * L.w + wi) * L.c_in + c_lo;
-      const T* wp = w + (((long long)co * L.kh + r) * L.kw + s) * cw;
-      for (int ci = 0; ci < cw; ++ci) acc = __fadd_rn(acc, __fmul_rn(ld_f<T>(xp + ci), ld_f<T>(wp + ci)));
-    }
-  }
-  return acc;
 }
 
 // One warp per (pixel row, 32-channel block): base path, gate, conditional path where the gate
@@ -97,18 +71,18 @@ static_gated_conv_kernel(LayerDims L, const T* __restrict__ x, const T* __restri
     const int n = (int)(m / ((long long)L.wo * L.ho));
     bool fire = false;
     if (co < L.c_out) {
-      const float p = conv_sum<T>(L, x, w_base, n, ho, wo, co, 0, L.c_p);
+      const float p = conv_point<T>(L, x, w_base, n, ho, wo, co, 0, L.c_p);
       fire = (p >= c_t[co]);
       float v;
       if (fire) {
-        const float r = conv_sum<T>(L, x, w_cond, n, ho, wo, co, L.c_p, L.c_r);
+        const float r = conv_point<T>(L, x, w_cond, n, ho, wo, co, L.c_p, L.c_r);
         v = __fadd_rn(__fmul_rn(c_a2[co], __fadd_rn(p, r)), c_b2[co]);
       } else {
         v = __fadd_rn(__fmul_rn(c_a1[co], p), c_b1[co]);
       }
-      if (residual) v = __fadd_rn(v, ld_f<T>(residual + m * L.c_out + co));
+      if (residual) v = __fadd_rn(v, Elem<T>::ld(residual + m * L.c_out + co));
       if (L.relu) v = (v > 0.f) ? v : 0.f;
-      st_f(y + m * L.c_out + co, v);
+      st_out(y + m * L.c_out + co, v);
     }
     const unsigned word = __ballot_sync(0xffffffffu, fire);
     if (lane == 0) {

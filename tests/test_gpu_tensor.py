@@ -27,6 +27,7 @@ SHAPES = [
     (O.Shape(2, 14, 14, 256, 64, groups=8), "G = 8, c_p = 32, c_out != c_in"),
     (O.Shape(2, 13, 11, 64, 192, groups=2), "odd extents, G = 2, three column tiles of 64"),
     (O.Shape(2, 9, 9, 64, 64, kh=1, kw=1, pad=0, groups=4), "1x1 kernel"),
+    (O.Shape(14, 56, 56, 64, 128, kh=1, kw=1, pad=0, groups=4), "1x1 kernel 64 -> 128, 392 row tiles: three jobs per CTA"),
     (O.Shape(12, 56, 56, 64, 64, groups=4), "336 row tiles: up to three jobs per CTA, resident weights"),
     (O.Shape(50, 28, 28, 128, 128, groups=4), "350 row tiles: streamed weights, three jobs per CTA"),
     (O.Shape(40, 14, 14, 256, 256, groups=4), "80 row tiles x 2 column tiles, two jobs per CTA"),
@@ -152,6 +153,7 @@ I8_SHAPES = [
     (O.Shape(5, 7, 7, 512, 512, groups=4), "int8 512@7, c_p = 128 bytes, two images per tile"),
     (O.Shape(2, 28, 28, 128, 256, stride=2, groups=4), "int8 stride 2"),
     (O.Shape(30, 28, 28, 128, 128, groups=2), "int8 G = 2, 210 row tiles"),
+    (O.Shape(64, 28, 28, 128, 128, groups=4), "int8 128 -> 128, 448 row tiles: four jobs per CTA"),
 ]
 
 
@@ -267,3 +269,29 @@ def test_dependent_layers_back_to_back_on_one_stream():
         assert torch.equal(y.view(torch.int16), y_ref.view(torch.int16))
     assert g1.conv.stats().device_status == 0 and g2.conv.stats().device_status == 0
     g1.close(); g2.close()
+
+
+def test_misaligned_workspace_is_refused_before_any_launch():
+    """cg_conv_forward checks the workspace pointer (256-byte alignment) on the host."""
+    import torch
+    from paper_1805_12549_b200 import binding as B
+    s = O.Shape(2, 28, 28, 128, 128, groups=4)
+    c = K.make_float_case("tcalign", s, "bf16", density=0.3)
+    g = K.GpuCase(c, algo=TENSOR, cond_mode=3)               # row compaction: the layer needs a workspace
+    need = B.cg_conv_workspace_bytes(g.conv.handle)
+    assert need > 0
+    y0, m0, _ = g.run()
+    buf = torch.zeros(need + 512, dtype=torch.uint8, device="cuda")
+    off = (-buf.data_ptr()) % 256 + 16
+    g.conv.workspace = buf[off:off + need]
+    g.y.fill_(0)
+    with pytest.raises(B.CgError) as e:
+        g.conv.forward(g.x, g.wb, g.wc, g.bn, g.delta, g.y, g.mask, g.res)
+    assert e.value.status == 3                               # CG_ERR_ALIGNMENT
+    torch.cuda.synchronize()
+    assert float(g.y.float().abs().max()) == 0.0             # nothing ran
+    g.conv.workspace = None
+    with pytest.raises(B.CgError) as e:
+        g.conv.forward(g.x, g.wb, g.wc, g.bn, g.delta, g.y, g.mask, g.res)
+    assert e.value.status == 4                               # CG_ERR_WORKSPACE
+    g.close()

@@ -448,3 +448,40 @@ def test_channel_gate_is_per_image():
     for i in range(2):
         one = O.gated_conv(s1, x[i:i + 1], wb, wc, bn, delta, channel_tau=0.45)
         np.testing.assert_array_equal(one.y[0], both.y[i])
+
+
+# --------------------------------------------------------------------------- channel reordering
+def test_reordering_output_channels_only_relabels_the_layer():
+    """A layer whose output channels are gathered by a permutation gives the permuted outputs and
+    mask bits of the original layer, and a consumer whose input channels are gathered the same way
+    (ungated, so that its split does not move) gives its original output."""
+    from paper_1805_12549_b200 import permute, synth
+    s = O.Shape(2, 6, 6, 16, 32, 3, 3, 1, 1, 4)
+    key = ("permute", 1)
+    x = synth.smoothed_noise((key, "x"), s.n, s.h, s.w, s.c_in)
+    wb, wc = synth.kaiming_weights(key, s.c_out, 3, 3, s.c_in, s.groups)
+    bn = synth.bn_params(key, s.c_out)
+    delta = synth.rng(key, "delta").normal(0.3, 0.5, s.c_out).astype(np.float32)
+    ref = O.gated_conv(s, x, wb, wc, bn, delta)
+    d = permute.unpack_mask(ref.mask, s.c_out)
+    np.testing.assert_array_equal(d, O.unpack_mask(ref.mask, s.c_out))
+    perm = permute.order_by_firing_rate(d)
+    assert sorted(perm.tolist()) == list(range(s.c_out))
+    rates = d.mean(0)[perm]
+    assert (np.diff(rates) <= 1e-12).all()
+    wb2, wc2, pc = permute.permute_output_channels(wb, wc, {**bn, "delta": delta}, perm)
+    delta2 = pc.pop("delta")
+    got = O.gated_conv(s, x, wb2, wc2, pc, delta2)
+    np.testing.assert_array_equal(got.y, ref.y[..., perm])
+    np.testing.assert_array_equal(O.unpack_mask(got.mask, s.c_out), d[:, perm])
+    # consumer: an ungated 1x1 layer over the 32 channels
+    s2 = O.Shape(2, 6, 6, 32, 8, 1, 1, 1, 0, 1)
+    w2, _ = synth.kaiming_weights((key, "next"), 8, 1, 1, 32, 1)
+    bn2 = synth.bn_params((key, "next"), 8)
+    shut = np.full(8, np.inf, np.float32)
+    empty = np.zeros((8, 1, 1, 0), np.float32)
+    a = O.gated_conv(s2, ref.y, w2, empty, bn2, shut)
+    w2p, w2c = permute.permute_input_channels(w2, perm, 1)
+    assert w2c.size == 0
+    b = O.gated_conv(s2, got.y, w2p, w2c, bn2, shut)
+    np.testing.assert_allclose(b.y, a.y, rtol=0, atol=1e-5)     # same products, summed in another order
