@@ -32,14 +32,14 @@ METRIC = "gated-conv images/sec at measured gate density"
 UNIT = "images/s"
 
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the layer kernel,
-# from the ncu captures summarised under profiles/.  It is reported only while the kernel sources
-# still hash to what they were when the counters were taken.
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the layer kernel:
+# the mean over the six launches listed in profiles/dram_traffic_layer_kernels.txt.  The y and mask
+# writes of a captured launch are still in the 126 MB L2 when it ends, so they are not in these
+# sums.  Reported only while the kernel sources still hash to what they were when the counters
+# were taken.
 TRAFFIC = {
-    "source_sha": "0e2953bc28412162",
-    # profiles/tc_gated_conv_kernel_c64at32_full.txt and ..._c128at16_full.txt; the y and mask writes
-    # of the captured launch were still in the 126 MB L2 when it ended, so they are not in these sums
-    "bytes_per_launch": {"c64@32": 33736192 + 633088, "c128@16": 17210624 + 256},
+    "source_sha": "f3b9cae6d3bc6ea2",
+    "bytes_per_launch": {"c64@32": 33822000, "c128@16": 17134500},
 }
 
 

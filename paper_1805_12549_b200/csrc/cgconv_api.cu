@@ -119,10 +119,12 @@ cg_status cg_conv_create(cg_conv_t* out, const cg_conv_desc* desc) {
   // runs on the direct kernels
   const bool want_tc = desc->algo != CG_ALGO_DIRECT && !(desc->channel_tau > 0.f);
   // Two tensor-core kernels.  Measured on B200 (batch 64-256 ResNet-18 shapes), the channel-major
-  // kernel is the faster one for 128 output channels and for 256 channels on 8x8 images, where the
-  // pixel-major kernel's whole-image tiles are half padding; elsewhere the pixel-major kernel wins.
+  // kernel is the faster one for 128 output channels, and for 256 channels on 8x8 images (where the
+  // pixel-major kernel's whole-image tiles are half padding) or with 20,000 and more pixels (enough
+  // pixel tiles to fill every SM with both channel tiles); elsewhere the pixel-major kernel wins.
   // Each also takes the layers only it can run.
-  const bool prefer2 = h->L.c_out == 128 || (h->L.c_out == 256 && h->L.ho * h->L.wo <= 64);
+  const bool prefer2 = h->L.c_out == 128 ||
+                       (h->L.c_out == 256 && (h->L.ho * h->L.wo <= 64 || h->L.m >= 20000));
   const bool allow1 = desc->algo != CG_ALGO_TENSOR_CHANNELS, allow2 = desc->algo != CG_ALGO_TENSOR_ROWS;
   bool ok1 = false, ok2 = false;
   if (want_tc && allow2 && (prefer2 || !allow1)) ok2 = cg::tc2_plan(h->L, desc->in_dtype, desc->cond_mode, sms, &h->plan2);

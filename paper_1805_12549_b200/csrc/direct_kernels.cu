@@ -24,7 +24,12 @@ __device__ __forceinline__ int conv_point_i8(const LayerDims& L, const int8_t* _
       if (wi < 0 || wi >= L.w) continue;
       const int8_t* xp = x + (((long long)n * L.h + hi) * L.w + wi) * L.c_in + c_lo;
       const int8_t* wp = w + (((long long)co * L.kh + r) * L.kw + s) * cw;
-      for (int ci = 0; ci < cw; ++ci) acc += (int)xp[ci] * (int)wp[ci];
+      int ci = 0;
+      // four products per instruction where both runs are 4-byte aligned (integer sums do not
+      // depend on the order)
+      if ((((uintptr_t)xp | (uintptr_t)wp) & 3u) == 0)
+        for (; ci + 4 <= cw; ci += 4) acc = __dp4a(*(const int*)(xp + ci), *(const int*)(wp + ci), acc);
+      for (; ci < cw; ++ci) acc += (int)xp[ci] * (int)wp[ci];
     }
   }
   return acc;
