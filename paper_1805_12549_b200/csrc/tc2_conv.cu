@@ -524,13 +524,16 @@ tc2_gated_conv_kernel(const __grid_constant__ CUtensorMap map_r1,
                 ptx::tc_fence_after();
                 if (!dense) {
                   uint32_t f = 0;
+#pragma unroll
                   for (int w = 0; w < kEpiWarps; ++w) f |= *(volatile uint32_t*)&sh->fired[X][w];
                   run = f != 0u;
                 }
-                // (sub-tiles made of padding rows only do not count as skipped work)
-                bool has_rows = false;
-                for (int g = (first_m + jb * stride_m) * rows_per_job + X * P.r, e = g + P.r; g < e && g < rows_all; ++g)
-                  has_rows = has_rows || (g % P.hp) < L.h;
+                // (sub-tiles made of padding rows only do not count as skipped work; a sub-tile
+                // taller than an image's padding always holds a real row)
+                const int gs = (first_m + jb * stride_m) * rows_per_job + X * P.r;
+                bool has_rows = gs < rows_all && P.r > P.hp - L.h;
+                if (!has_rows)
+                  for (int g = gs, e = gs + P.r; g < e && g < rows_all; ++g) has_rows = has_rows || (g % P.hp) < L.h;
                 if (has_rows) { st_sub += 1; if (run) st_sub_run += 1; }
               }
               if (flags & kStageNewChunk) {
