@@ -144,7 +144,7 @@ typedef struct {
  * grouping, no channel-wise gate; odd square filter with pad = (k-1)/2; c_in a multiple of 64
  * (BF16) or 128 (I8);
  *   pixel-major kernel:   stride 1, or stride 2 for 3x3 filters on even extents; c_out a multiple
- *                         of 64 (BF16) or 128 (I8); c_in/G equal to 16 or 32 (BF16; 32 or 64 for
+ *                         of 64 (BF16) or 128 (I8); c_in/G equal to 8, 16 or 32 (BF16; 32 or 64 for
  *                         I8) or a multiple of 64 (128); output width at most 128;
  *   channel-major kernel: BF16, stride 1, c_out a multiple of 32, c_in/G equal to 8, 16, 32 or a
  *                         multiple of 64, no row compaction (CG_COND_COMPACT).

@@ -167,7 +167,7 @@ int cg_conv_launches_per_forward(cg_conv_t h) {
   if (!h) return 0;
   if (h->L.channel_tau > 0.f) return 2;
   if (h->use_tc2) return h->plan2.pad8 ? 2 : 1;
-  return (h->use_tc && h->plan.cond_mode == CG_COND_COMPACT) ? 2 : 1;
+  return (h->use_tc && (h->plan.cond_mode == CG_COND_COMPACT || h->plan.pad8)) ? 2 : 1;
 }
 
 int cg_conv_uses_tensor_cores(cg_conv_t h) { return h ? h->use_tc : 0; }

@@ -721,10 +721,25 @@ __global__ void tc2_repack_kernel(const __nv_bfloat16* __restrict__ wb, const __
 
 }  // namespace
 
-size_t tc2_workspace_bytes(const LayerDims& L, const Tc2Plan& P) {
-  if (!P.valid || !P.pad8) return 0;
+size_t repack8_bytes(const LayerDims& L) {
   const size_t rows = (size_t)L.c_out * L.kh * L.kw;
   return align_up2(rows * 16 * 2, 256) + align_up2(rows * (size_t)L.c_in * 2, 256);
+}
+
+int launch_repack8(const LayerDims& L, const void* w_base, const void* w_cond, void* workspace, const void** wb16,
+                   const void** wcf, cudaStream_t stream) {
+  const size_t rows = (size_t)L.c_out * L.kh * L.kw;
+  __nv_bfloat16* b = static_cast<__nv_bfloat16*>(workspace);
+  __nv_bfloat16* c = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + align_up2(rows * 16 * 2, 256));
+  tc2_repack_kernel<<<64, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(w_base), static_cast<const __nv_bfloat16*>(w_cond), b, c,
+                                            (int)rows, L.c_in);
+  *wb16 = b; *wcf = c;
+  return (int)cudaGetLastError();
+}
+
+size_t tc2_workspace_bytes(const LayerDims& L, const Tc2Plan& P) {
+  if (!P.valid || !P.pad8) return 0;
+  return repack8_bytes(L);
 }
 
 // K stages of a job in the order the MMA issuer consumes them (and the weight producer loads

@@ -70,6 +70,13 @@ struct Tc2Maps {
   int next;
 };
 
+// Weights of a layer with c_in/G = 8 repacked into `workspace` (repack8_bytes) with whole K steps:
+// W_base gets 8 zero channels behind its 8 per tap, W_cond 8 zero channels in front; the layer is
+// then computed as one with 16 base channels and a conditional path over all input channels.
+size_t repack8_bytes(const LayerDims& L);
+int launch_repack8(const LayerDims& L, const void* w_base, const void* w_cond, void* workspace, const void** wb16,
+                   const void** wcf, cudaStream_t stream);
+
 bool tc2_plan(const LayerDims& L, int in_dtype, int cond_mode, int sms, Tc2Plan* plan);
 size_t tc2_workspace_bytes(const LayerDims& L, const Tc2Plan& plan);
 int launch_tc2(const LayerDims& L, const Tc2Plan& plan, Tc2Maps* maps, const void* x,

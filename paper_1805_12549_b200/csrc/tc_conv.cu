@@ -38,6 +38,7 @@
 
 #include "ptx.cuh"
 #include "tc_conv.cuh"
+#include "tc2_conv.cuh"
 
 namespace cg {
 
@@ -95,8 +96,12 @@ __device__ __forceinline__ WTile base_tile(const LayerDims& L, int ck, int bt) {
   return {bt * ck, 0};
 }
 
-__device__ __forceinline__ WTile cond_tile(const LayerDims& L, int ck, int bt) {
+__device__ __forceinline__ WTile cond_tile(const LayerDims& L, int ck, int bt, bool pad8) {
   const int taps = L.kh * L.kw;
+  if (pad8) {                       // repacked weights: every chunk whole, chunk 0 included
+    const int q = bt / taps, t = bt % taps;
+    return {t * L.c_r + ck * q, q};
+  }
   if (L.c_p >= ck) {
     const int q = L.c_p / ck + bt / taps, t = bt % taps;
     return {t * L.c_r + ck * q - L.c_p, q};
@@ -219,6 +224,7 @@ struct MmaIssuer {
   // (r ? 1 : 0) rows + (sx ? 1 : 0) pixels, and plane p is the p-th buffer of the chunk.
   uint32_t f0, f1, f2, c0, c1, c2, row_lo;
   int resident, a0, na /* ring slots [a0, na) */, nb, kp16 /* base K steps per tap */, chunks, base_chunks, base_tiles, kh, kw, planes;
+  bool pad8;
   int as, bs;                            // ring slots and the parities of their "full" barriers
   uint32_t apar, bpar;
   // per phase
@@ -249,7 +255,7 @@ struct MmaIssuer {
       f0 = 0u; f1 = row_lo; f2 = 2u * row_lo;
       c0 = 0u; c1 = 8u; c2 = 16u;
     }
-    resident = P.resident; a0 = slot0; na = slot0 + slots; nb = P.nb; kp16 = L.c_p / (P.ck / 4); chunks = P.chunks;
+    resident = P.resident; a0 = slot0; na = slot0 + slots; nb = P.nb; kp16 = L.c_p / (P.ck / 4); chunks = P.chunks; pad8 = P.pad8 != 0;
     base_chunks = P.base_chunks; base_tiles = P.base_tiles; kh = L.kh; kw = L.kw; planes = P.planes;
     as = slot0; bs = 0; apar = 0; bpar = 0;
     a_first = slot0; b_held = 0; ok = true;
@@ -385,6 +391,8 @@ struct MmaIssuer {
     } else if (!cond) {
       if (kp16 == 1) base_small3<RES, 1>(); else base_small3<RES, 2>();
       nfull = 0;
+    } else if (pad8) {
+      nfull = chunks;               // (repacked weights: zeros multiply the base channels)
     } else {
       if (kp16 == 1) chunk_taps3<RES, 1, 4>(); else chunk_taps3<RES, 2, 4>();
       nfull = chunks - 1;
@@ -399,7 +407,7 @@ struct MmaIssuer {
     } else if (!cond) {
       chunk_taps_any(0, kp16, 4 / kp16);
     } else {
-      chunk_taps_any(kp16, 4, 1);
+      chunk_taps_any(pad8 ? 0 : kp16, 4, 1);
       for (int q = 1; q < chunks && ok; ++q) chunk_taps_any(0, 4, 1);
     }
   }
@@ -514,7 +522,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   if (warp == 2) {
     // K coordinate of every weight tile, for the weight loads
     for (int bt = lane; bt < P.base_tiles + P.cond_tiles; bt += 32)
-      s_wx[bt] = (bt < P.base_tiles ? base_tile(L, P.ck, bt) : cond_tile(L, P.ck, bt - P.base_tiles)).x;
+      s_wx[bt] = (bt < P.base_tiles ? base_tile(L, P.ck, bt) : cond_tile(L, P.ck, bt - P.base_tiles, P.pad8 != 0)).x;
   }
   // Only the barriers, the TMEM address and the tile coordinates are needed before the first
   // copies can be issued: the rest of the set-up (below, epilogue warps) overlaps those copies.
@@ -1164,7 +1172,7 @@ tc_compact_cond_kernel(const __grid_constant__ CUtensorMap map_wc, const __grid_
           if (!ok) break;
           ptx::mbar_expect_tx(&sh->full[st], NT * 128);
           ptx::tma_load_2d(s_stage + (size_t)st * kStageBytes + 128 * 128, &map_wc, &sh->full[st],
-                           cond_tile(L, P.ck, bt).x, tn * NT);
+                           cond_tile(L, P.ck, bt, false).x, tn * NT);
           if (++st == kCpStages) { st = 0; par ^= 1; }
         }
       }
@@ -1218,7 +1226,7 @@ tc_compact_cond_kernel(const __grid_constant__ CUtensorMap map_wc, const __grid_
       int pending = 0;       // stages whose copies are issued but not yet published
       int pub = st;          // next stage to publish
       for (int bt = 0; bt < P.cond_tiles && ok; ++bt) {
-        const WTile w = cond_tile(L, P.ck, bt);
+        const WTile w = cond_tile(L, P.ck, bt, false);
         int t;
         if (L.c_p >= P.ck) t = bt % taps; else t = bt < taps ? bt : (bt - taps) % taps;
         const int hi = ho * L.stride + t / L.kw - L.pad, wi = wo * L.stride + t % L.kw - L.pad;
@@ -1360,10 +1368,17 @@ int sm_count(int dev) {
 
 }  // namespace
 
-bool tc_plan(const LayerDims& L, int in_dtype, int cond_mode, TcPlan* plan) {
+bool tc_plan(const LayerDims& L_in, int in_dtype, int cond_mode, TcPlan* plan) {
   TcPlan P;
   std::memset(&P, 0, sizeof(P));
   *plan = P;
+  // Base slices of 8 channels (bf16) are half a K step: the layer is planned, and later run, as one
+  // with 16 base channels and a conditional path over all input channels (weights repacked).
+  LayerDims L = L_in;
+  if (in_dtype == CG_BF16 && L.c_p == 8 && L.c_r > 0 && !L.grouping) {
+    if (cond_mode == CG_COND_COMPACT) return false;
+    L.c_p = 16; L.c_r = L.c_in; P.pad8 = 1;
+  }
   if (in_dtype != CG_BF16 && in_dtype != CG_I8) return false;
   const int eb = in_dtype == CG_BF16 ? 2 : 1;
   const int ck = 128 / eb;          // channels per 128-byte patch row
@@ -1504,17 +1519,25 @@ bool tc_device_ok(int device) {
 // CG_COND_COMPACT workspace: [row counts, 256 B][row lists: tiles_n x M x u32][row records:
 // tiles_n x M x (NT + 4) words]
 size_t tc_workspace_bytes(const LayerDims& L, const TcPlan& P) {
+  if (P.valid && P.pad8) return repack8_bytes(L);
   if (!P.valid || P.cond_mode != CG_COND_COMPACT) return 0;
   const size_t rows = (size_t)P.tiles_n * (size_t)L.m;
   return 256 + align_up(rows * 4, 256) + rows * (size_t)(P.nt + 4) * 4;
 }
 
-int launch_tc(const LayerDims& L, const TcPlan& P, int in_dtype, TcMaps* maps, const void* x,
+int launch_tc(const LayerDims& L_in, const TcPlan& P, int in_dtype, TcMaps* maps, const void* x,
               const void* w_base, const void* w_cond, const cg_bn_params& bn, const float* delta,
               const void* residual, void* y, uint32_t* mask, void* workspace,
               unsigned long long* counters, cudaStream_t stream) {
   (void)in_dtype;
   if (!P.valid) return (int)cudaErrorInvalidValue;
+  LayerDims L = L_in;
+  if (P.pad8) {
+    if (!workspace) return (int)cudaErrorInvalidValue;
+    const int e = launch_repack8(L_in, w_base, w_cond, workspace, &w_base, &w_cond, stream);
+    if (e != 0) return e;
+    L.c_p = 16; L.c_r = L.c_in;
+  }
   const void* wc_key = w_cond ? w_cond : w_base;
   TcMapSet* ms = nullptr;
   for (int i = 0; i < TcMaps::kEntries; ++i) {

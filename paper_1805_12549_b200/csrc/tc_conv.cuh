@@ -41,6 +41,8 @@ struct TcPlan {
   int stage_rows;       // rows of the y staging tile
   int base_tiles, cond_tiles;   // weight tiles per phase
   int cond_mode;
+  int pad8;             // c_in/G = 8 (bf16): computed as 16 base channels + a conditional path over all
+                        // input channels, with weights repacked into the workspace (tc2_conv.cuh)
   unsigned off_a, off_b, off_y, off_consts, off_mask, off_tables, off_bar, smem_bytes;
 };
 

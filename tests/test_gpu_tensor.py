@@ -35,6 +35,9 @@ SHAPES = [
     (O.Shape(3, 28, 28, 128, 256, stride=2, groups=4), "stride 2, 28->14, c_p = 32"),
     (O.Shape(5, 14, 14, 256, 512, stride=2, groups=4), "stride 2, 14->7, c_p = 64, two images per tile"),
     (O.Shape(2, 12, 20, 64, 64, stride=2, groups=2), "stride 2, odd tile split, G = 2"),
+    (O.Shape(3, 56, 56, 64, 64, groups=8), "G = 8 at 64 channels: c_p = 8 through repacked weights"),
+    (O.Shape(3, 56, 56, 64, 128, stride=2, groups=8), "G = 8, stride 2, c_p = 8"),
+    (O.Shape(2, 14, 14, 128, 64, groups=16), "G = 16 at 128 channels: c_p = 8, two chunks"),
 ]
 
 
