@@ -142,10 +142,10 @@ typedef struct {
  * listed above, shift out of range), CG_ERR_CUDA, and CG_ERR_UNSUPPORTED when a tensor-core
  * algo is asked for a layer outside the kernels' limits.  Those are: BF16 or I8; no channel
  * grouping, no channel-wise gate; odd square filter with pad = (k-1)/2; c_in a multiple of 64
- * (BF16) or 128 (I8);
+ * (BF16), a multiple of 128 or equal to 64 (I8);
  *   pixel-major kernel:   stride 1, or stride 2 for 3x3 filters on even extents; c_out a multiple
- *                         of 64 (BF16) or 128 (I8); c_in/G equal to 8, 16 or 32 (BF16; 32 or 64 for
- *                         I8) or a multiple of 64 (128); output width at most 128;
+ *                         of 64; c_in/G equal to 8, 16 or 32 (BF16; 32 or 64 for I8, at most 32 when
+ *                         c_in = 64) or a multiple of 64 (128); output width at most 128;
  *   channel-major kernel: BF16, stride 1, c_out a multiple of 32, c_in/G equal to 8, 16, 32 or a
  *                         multiple of 64, no row compaction (CG_COND_COMPACT).
  * AUTO falls back to the direct kernels outside these limits.
@@ -157,7 +157,7 @@ cg_status cg_conv_create(cg_conv_t* out, const cg_conv_desc* desc);
 
 /* Bytes of device scratch cg_conv_forward needs (may be 0): the partial sums and per-channel
  * counts of the channel-wise gate (Eq. 4), the compacted row lists of CG_COND_COMPACT (Eq. 1: the
- * rows where d = 1), or weights repacked for c_in/G = 8.  Contents need not persist between
+ * rows where d = 1), or weights repacked with whole K steps (c_in/G = 8; I8 layers with c_in = 64).  Contents need not persist between
  * calls; two forwards that overlap in time must not share one workspace.  The pointer given to
  * cg_conv_forward must be 256-byte aligned (CG_ERR_ALIGNMENT otherwise). */
 size_t cg_conv_workspace_bytes(cg_conv_t h);

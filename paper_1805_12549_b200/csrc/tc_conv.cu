@@ -486,7 +486,10 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   const bool has_cond = P.cond_tiles > 0 && !compact;
   const int cond_first_chunk = L.c_p >= P.ck ? P.base_chunks : 0;
   constexpr int kBlocks = NT / 64;
-  constexpr uint32_t kAllBlocks = (1u << kBlocks) - 1u;
+  // 64-channel column blocks of this tile that hold real output channels (the last tile of a
+  // layer whose c_out is not a multiple of NT holds fewer)
+  const int real_blocks = min(kBlocks, (L.c_out - (int)(blockIdx.x % P.tiles_n) * NT + 63) / 64);
+  const uint32_t kAllBlocks = (1u << real_blocks) - 1u;
   constexpr int kWords = NT / 32;
   constexpr int kNP = NT == 64 ? 4 : 3;      // P accumulators in TMEM
   constexpr int kNR = NT == 64 ? 4 : 1;      // R accumulators in TMEM
@@ -548,9 +551,10 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     for (int c = et; c < NT; c += kEpiThreads) {
       const int cg_ = tile_n * NT + c;
       if (I8) {
-        s_qt[c] = prm.bn.q_gate_thr[cg_];
-        s_qm1[c] = prm.bn.q_mul_base[cg_]; s_qm2[c] = prm.bn.q_mul_full[cg_];
-        s_qo1[c] = prm.bn.q_off_base[cg_]; s_qo2[c] = prm.bn.q_off_full[cg_];
+        const bool real = cg_ < L.c_out;               // (columns behind c_out: never fire, never stored)
+        s_qt[c] = real ? prm.bn.q_gate_thr[cg_] : 0x7fffffff;
+        s_qm1[c] = real ? prm.bn.q_mul_base[cg_] : 0; s_qm2[c] = real ? prm.bn.q_mul_full[cg_] : 0;
+        s_qo1[c] = real ? prm.bn.q_off_base[cg_] : 0ll; s_qo2[c] = real ? prm.bn.q_off_full[cg_] : 0ll;
       } else {
         const ChannelConsts k = fold_channel(prm.bn, prm.delta, L.eps, cg_);
         s_t[c] = k.t; s_k[c] = make_float4(k.a1, k.b1, k.a2, k.b2);
@@ -806,10 +810,10 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
           }
         }
         uint32_t word = (pw[0] | pw[1]) | (pw[2] | pw[3]);
-        if (!valid) word = 0;
+        if (!valid || tile_n * kWords + w >= L.words) word = 0;
         s_words[w] = word;
         st_active += __popc(word);
-        if (valid && prm.mask) g_words[w] = word;
+        if (valid && prm.mask && tile_n * kWords + w < L.words) g_words[w] = word;
         if (__ballot_sync(0xffffffffu, word != 0u)) fired_blocks |= 1u << (w >> 1);
       }
       // 64-channel column blocks with a firing gate, over the warp
@@ -1034,9 +1038,9 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     if (ct == 0 && ok) {
       const unsigned long long k_p = (unsigned long long)taps * L.c_p, k_r = (unsigned long long)taps * L.c_r;
       if (blockIdx.x == 0) atomicAdd(&prm.counters[CNT_CALLS], 1ull);
-      atomicAdd(&prm.counters[CNT_TILES_TOTAL], (unsigned long long)kBlocks * jobs);
+      atomicAdd(&prm.counters[CNT_TILES_TOTAL], (unsigned long long)real_blocks * jobs);
       atomicAdd(&prm.counters[CNT_TILES_SKIPPED],
-                has_cond ? (unsigned long long)kBlocks * jobs - st_blocks_run : 0ull);
+                has_cond ? (unsigned long long)real_blocks * jobs - st_blocks_run : 0ull);
       atomicAdd(&prm.counters[CNT_EXEC_MACS],
                 (unsigned long long)kBM * NT * k_p * jobs + (unsigned long long)kBM * 64ull * st_blocks_run * k_r);
     }
@@ -1379,6 +1383,14 @@ bool tc_plan(const LayerDims& L_in, int in_dtype, int cond_mode, TcPlan* plan) {
     if (cond_mode == CG_COND_COMPACT) return false;
     L.c_p = 16; L.c_r = L.c_in; P.pad8 = 1;
   }
+  // int8 layers with 64 input channels: a pixel is half a 128-byte patch row.  The copies of x
+  // fill the upper half with zeros (out-of-bounds elements of the tensor map), and the weights
+  // are repacked as for 8-channel slices: 32 base channels per tap (zeros behind the real ones), a
+  // conditional path over all 128 (zeros in front of and behind the real ones).
+  if (in_dtype == CG_I8 && L.c_in == 64 && L.c_p <= 32 && L.c_r > 0 && !L.grouping) {
+    if (cond_mode == CG_COND_COMPACT) return false;
+    L.c_in = 128; L.c_p = 32; L.c_r = 128; P.pad8 = 2;
+  }
   if (in_dtype != CG_BF16 && in_dtype != CG_I8) return false;
   const int eb = in_dtype == CG_BF16 ? 2 : 1;
   const int ck = 128 / eb;          // channels per 128-byte patch row
@@ -1392,7 +1404,7 @@ bool tc_plan(const LayerDims& L_in, int in_dtype, int cond_mode, TcPlan* plan) {
   if (s2 && (L.kh != 3 || (L.h & 1) || (L.w & 1))) return false;
   if (L.c_in % ck != 0) return false;
   if (!(L.c_p == kst || L.c_p == 2 * kst || L.c_p % ck == 0)) return false;
-  if (L.c_out % 64 != 0 || (eb == 1 && L.c_out % 128 != 0)) return false;
+  if (L.c_out % 64 != 0) return false;   // (int8: the last 128-channel tile may be half empty)
   const int xpad = s2 ? 1 : L.pad;                  // zero columns/rows shared between patch rows
   if (L.wo + xpad > kBM) return false;
   P.elem_bytes = eb;
@@ -1450,7 +1462,7 @@ bool tc_plan(const LayerDims& L_in, int in_dtype, int cond_mode, TcPlan* plan) {
   const size_t limit = 227 * 1024 - 1024;
   for (int pass = 0; pass < 2; ++pass)
   for (int nt = 128; nt >= (eb == 1 ? 128 : 64); nt >>= 1) {
-    if (L.c_out % nt != 0) continue;
+    if (L.c_out % nt != 0 && eb != 1) continue;
     const size_t fixed = align_up((size_t)(nt * eb / 128) * P.stage_rows * 128, 1024) +
                          align_up((size_t)8 * nt * 4, 128) +
                          align_up((size_t)4 * 128 * (nt / 32) * 4, 128) +
@@ -1493,7 +1505,7 @@ bool tc_plan(const LayerDims& L_in, int in_dtype, int cond_mode, TcPlan* plan) {
     P.off_mask = (unsigned)off; off += align_up((size_t)4 * 128 * (nt / 32) * 4, 128);
     P.off_tables = (unsigned)off; off += align_up((size_t)kMaxWTiles * 4, 128);
     P.off_bar = (unsigned)off; off += align_up(sizeof(Shared), 128);
-    P.nt = nt; P.na = na; P.nb = nb; P.resident = resident; P.tiles_n = L.c_out / nt;
+    P.nt = nt; P.na = na; P.nb = nb; P.resident = resident; P.tiles_n = (L.c_out + nt - 1) / nt;
     // resident weights: the base and the conditional path get their own MMA issuer and their own
     // half of the patch ring
     const bool two = resident && P.cond_tiles > 0 && P.cond_mode != CG_COND_COMPACT;
@@ -1518,7 +1530,30 @@ bool tc_device_ok(int device) {
 
 // CG_COND_COMPACT workspace: [row counts, 256 B][row lists: tiles_n x M x u32][row records:
 // tiles_n x M x (NT + 4) words]
+// int8 weights of a layer with 64 input channels, repacked with whole K steps (see tc_plan):
+// W_base [rows][c_p] -> [rows][32], W_cond [rows][64 - c_p] -> [rows][128] with the real channels at
+// their input-channel positions [c_p, 64); everything else zero.  rows = c_out * taps.
+__global__ void repack_i8_kernel(const int8_t* __restrict__ wb, const int8_t* __restrict__ wc, int8_t* __restrict__ wb32,
+                                 int8_t* __restrict__ wc128, int rows, int c_p) {
+  const int total = rows * 160;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+    const int row = i / 160, c = i - row * 160;
+    if (c < 32) {
+      wb32[(size_t)row * 32 + c] = c < c_p ? wb[(size_t)row * c_p + c] : (int8_t)0;
+    } else {
+      const int cc = c - 32;
+      wc128[(size_t)row * 128 + cc] = (cc >= c_p && cc < 64) ? wc[(size_t)row * (64 - c_p) + cc - c_p] : (int8_t)0;
+    }
+  }
+}
+
+static size_t repack_i8_bytes(const LayerDims& L) {
+  const size_t rows = (size_t)L.c_out * L.kh * L.kw;
+  return align_up(rows * 32, 256) + align_up(rows * 128, 256);
+}
+
 size_t tc_workspace_bytes(const LayerDims& L, const TcPlan& P) {
+  if (P.valid && P.pad8 == 2) return repack_i8_bytes(L);
   if (P.valid && P.pad8) return repack8_bytes(L);
   if (!P.valid || P.cond_mode != CG_COND_COMPACT) return 0;
   const size_t rows = (size_t)P.tiles_n * (size_t)L.m;
@@ -1532,7 +1567,17 @@ int launch_tc(const LayerDims& L_in, const TcPlan& P, int in_dtype, TcMaps* maps
   (void)in_dtype;
   if (!P.valid) return (int)cudaErrorInvalidValue;
   LayerDims L = L_in;
-  if (P.pad8) {
+  if (P.pad8 == 2) {
+    if (!workspace) return (int)cudaErrorInvalidValue;
+    const size_t rows = (size_t)L_in.c_out * L_in.kh * L_in.kw;
+    int8_t* b = static_cast<int8_t*>(workspace);
+    int8_t* c = b + align_up(rows * 32, 256);
+    repack_i8_kernel<<<64, 256, 0, stream>>>(static_cast<const int8_t*>(w_base), static_cast<const int8_t*>(w_cond), b, c,
+                                             (int)rows, L_in.c_p);
+    if (cudaGetLastError() != cudaSuccess) return (int)cudaErrorLaunchFailure;
+    w_base = b; w_cond = c;
+    L.c_in = 128; L.c_p = 32; L.c_r = 128;
+  } else if (P.pad8) {
     if (!workspace) return (int)cudaErrorInvalidValue;
     const int e = launch_repack8(L_in, w_base, w_cond, workspace, &w_base, &w_cond, stream);
     if (e != 0) return e;
@@ -1552,9 +1597,9 @@ int launch_tc(const LayerDims& L_in, const TcPlan& P, int in_dtype, TcMaps* maps
     const cuuint64_t eb = (cuuint64_t)P.elem_bytes;
     const cuuint32_t ck = (cuuint32_t)P.ck;
     if (L.stride == 1) {
-      cuuint64_t dims[4] = {(cuuint64_t)L.c_in, (cuuint64_t)L.w, (cuuint64_t)L.h, (cuuint64_t)L.n};
-      cuuint64_t str[3] = {(cuuint64_t)L.c_in * eb, (cuuint64_t)L.w * L.c_in * eb,
-                           (cuuint64_t)L.h * L.w * L.c_in * eb};
+      const cuuint64_t cx = (cuuint64_t)L_in.c_in;   // (the tensor's own channel count: a box may reach past it)
+      cuuint64_t dims[4] = {cx, (cuuint64_t)L.w, (cuuint64_t)L.h, (cuuint64_t)L.n};
+      cuuint64_t str[3] = {cx * eb, (cuuint64_t)L.w * cx * eb, (cuuint64_t)L.h * L.w * cx * eb};
       cuuint32_t box[4] = {ck, (cuuint32_t)P.wp, (cuuint32_t)P.box_h, (cuuint32_t)P.ni};
       if (!encode(&ms->x[0], P.elem_bytes, const_cast<void*>(x), 4, dims, str, box)) return (int)cudaErrorInvalidValue;
       ms->x[1] = ms->x[2] = ms->x[3] = ms->x[0];
@@ -1562,10 +1607,10 @@ int launch_tc(const LayerDims& L_in, const TcPlan& P, int in_dtype, TcMaps* maps
       // plane 2*ph + pw holds the input pixels (2a + ph, 2b + pw)
       for (int pl = 0; pl < 4; ++pl) {
         const int ph = pl >> 1, pw = pl & 1;
-        const char* base = static_cast<const char*>(x) + ((size_t)ph * L.w + pw) * L.c_in * eb;
-        cuuint64_t dims[4] = {(cuuint64_t)L.c_in, (cuuint64_t)L.w / 2, (cuuint64_t)L.h / 2, (cuuint64_t)L.n};
-        cuuint64_t str[3] = {(cuuint64_t)2 * L.c_in * eb, (cuuint64_t)2 * L.w * L.c_in * eb,
-                             (cuuint64_t)L.h * L.w * L.c_in * eb};
+        const cuuint64_t cx = (cuuint64_t)L_in.c_in;
+        const char* base = static_cast<const char*>(x) + ((size_t)ph * L.w + pw) * cx * eb;
+        cuuint64_t dims[4] = {cx, (cuuint64_t)L.w / 2, (cuuint64_t)L.h / 2, (cuuint64_t)L.n};
+        cuuint64_t str[3] = {(cuuint64_t)2 * cx * eb, (cuuint64_t)2 * L.w * cx * eb, (cuuint64_t)L.h * L.w * cx * eb};
         cuuint32_t box[4] = {ck, (cuuint32_t)P.wp, (cuuint32_t)P.box_h, (cuuint32_t)P.ni};
         if (!encode(&ms->x[pl], P.elem_bytes, const_cast<char*>(base), 4, dims, str, box)) return (int)cudaErrorInvalidValue;
       }

@@ -157,6 +157,11 @@ I8_SHAPES = [
     (O.Shape(2, 28, 28, 128, 256, stride=2, groups=4), "int8 stride 2"),
     (O.Shape(30, 28, 28, 128, 128, groups=2), "int8 G = 2, 210 row tiles"),
     (O.Shape(64, 28, 28, 128, 128, groups=4), "int8 128 -> 128, 448 row tiles: four jobs per CTA"),
+    (O.Shape(3, 56, 56, 64, 64, groups=4), "int8 64@56: 64-byte pixel rows, half-empty column tile"),
+    (O.Shape(2, 32, 32, 64, 64, groups=8), "int8 64@32, G = 8: 8 base channels"),
+    (O.Shape(2, 56, 56, 64, 128, stride=2, groups=4), "int8 64 -> 128 stride 2"),
+    (O.Shape(2, 28, 28, 128, 64, groups=4), "int8 128 -> 64: half-empty column tile"),
+    (O.Shape(2, 14, 14, 256, 192, groups=4), "int8 256 -> 192: one full and one half-empty column tile"),
 ]
 
 
