@@ -96,8 +96,9 @@ __device__ __forceinline__ WTile base_tile(const LayerDims& L, int ck, int bt) {
   return {bt * ck, 0};
 }
 
-__device__ __forceinline__ WTile cond_tile(const LayerDims& L, int ck, int bt, bool pad8) {
+__device__ __forceinline__ WTile cond_tile(const LayerDims& L, int ck, int bt, int pad8) {
   const int taps = L.kh * L.kw;
+  if (pad8 == 2) return {bt * ck, 0};   // int8, 64 input channels: a tile covers two taps of the only chunk
   if (pad8) {                       // repacked weights: every chunk whole, chunk 0 included
     const int q = bt / taps, t = bt % taps;
     return {t * L.c_r + ck * q, q};
@@ -224,7 +225,7 @@ struct MmaIssuer {
   // (r ? 1 : 0) rows + (sx ? 1 : 0) pixels, and plane p is the p-th buffer of the chunk.
   uint32_t f0, f1, f2, c0, c1, c2, row_lo;
   int resident, a0, na /* ring slots [a0, na) */, nb, kp16 /* base K steps per tap */, chunks, base_chunks, base_tiles, kh, kw, planes;
-  bool pad8;
+  int pad8;
   int as, bs;                            // ring slots and the parities of their "full" barriers
   uint32_t apar, bpar;
   // per phase
@@ -255,7 +256,7 @@ struct MmaIssuer {
       f0 = 0u; f1 = row_lo; f2 = 2u * row_lo;
       c0 = 0u; c1 = 8u; c2 = 16u;
     }
-    resident = P.resident; a0 = slot0; na = slot0 + slots; nb = P.nb; kp16 = L.c_p / (P.ck / 4); chunks = P.chunks; pad8 = P.pad8 != 0;
+    resident = P.resident; a0 = slot0; na = slot0 + slots; nb = P.nb; kp16 = L.c_p / (P.ck / 4); chunks = P.chunks; pad8 = P.pad8;
     base_chunks = P.base_chunks; base_tiles = P.base_tiles; kh = L.kh; kw = L.kw; planes = P.planes;
     as = slot0; bs = 0; apar = 0; bpar = 0;
     a_first = slot0; b_held = 0; ok = true;
@@ -391,6 +392,9 @@ struct MmaIssuer {
     } else if (!cond) {
       if (kp16 == 1) base_small3<RES, 1>(); else base_small3<RES, 2>();
       nfull = 0;
+    } else if (pad8 == 2) {
+      base_small3<RES, 2>();        // (int8, 64 input channels: two K steps per tap, two taps per tile)
+      nfull = 0;
     } else if (pad8) {
       nfull = chunks;               // (repacked weights: zeros multiply the base channels)
     } else {
@@ -406,6 +410,8 @@ struct MmaIssuer {
       for (int q = q0; q < q1 && ok; ++q) chunk_taps_any(0, 4, 1);
     } else if (!cond) {
       chunk_taps_any(0, kp16, 4 / kp16);
+    } else if (pad8 == 2) {
+      chunk_taps_any(0, 2, 2);
     } else {
       chunk_taps_any(pad8 ? 0 : kp16, 4, 1);
       for (int q = 1; q < chunks && ok; ++q) chunk_taps_any(0, 4, 1);
@@ -525,7 +531,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   if (warp == 2) {
     // K coordinate of every weight tile, for the weight loads
     for (int bt = lane; bt < P.base_tiles + P.cond_tiles; bt += 32)
-      s_wx[bt] = (bt < P.base_tiles ? base_tile(L, P.ck, bt) : cond_tile(L, P.ck, bt - P.base_tiles, P.pad8 != 0)).x;
+      s_wx[bt] = (bt < P.base_tiles ? base_tile(L, P.ck, bt) : cond_tile(L, P.ck, bt - P.base_tiles, P.pad8)).x;
   }
   // Only the barriers, the TMEM address and the tile coordinates are needed before the first
   // copies can be issued: the rest of the set-up (below, epilogue warps) overlaps those copies.
@@ -1176,7 +1182,7 @@ tc_compact_cond_kernel(const __grid_constant__ CUtensorMap map_wc, const __grid_
           if (!ok) break;
           ptx::mbar_expect_tx(&sh->full[st], NT * 128);
           ptx::tma_load_2d(s_stage + (size_t)st * kStageBytes + 128 * 128, &map_wc, &sh->full[st],
-                           cond_tile(L, P.ck, bt, false).x, tn * NT);
+                           cond_tile(L, P.ck, bt, 0).x, tn * NT);
           if (++st == kCpStages) { st = 0; par ^= 1; }
         }
       }
@@ -1230,7 +1236,7 @@ tc_compact_cond_kernel(const __grid_constant__ CUtensorMap map_wc, const __grid_
       int pending = 0;       // stages whose copies are issued but not yet published
       int pub = st;          // next stage to publish
       for (int bt = 0; bt < P.cond_tiles && ok; ++bt) {
-        const WTile w = cond_tile(L, P.ck, bt, false);
+        const WTile w = cond_tile(L, P.ck, bt, 0);
         int t;
         if (L.c_p >= P.ck) t = bt % taps; else t = bt < taps ? bt : (bt - taps) % taps;
         const int hi = ho * L.stride + t / L.kw - L.pad, wi = wo * L.stride + t % L.kw - L.pad;
@@ -1386,10 +1392,11 @@ bool tc_plan(const LayerDims& L_in, int in_dtype, int cond_mode, TcPlan* plan) {
   // int8 layers with 64 input channels: a pixel is half a 128-byte patch row.  The copies of x
   // fill the upper half with zeros (out-of-bounds elements of the tensor map), and the weights
   // are repacked as for 8-channel slices: 32 base channels per tap (zeros behind the real ones), a
-  // conditional path over all 128 (zeros in front of and behind the real ones).
+  // conditional path over the 64 real channels (zeros in front of the real ones), two taps per
+  // weight tile.
   if (in_dtype == CG_I8 && L.c_in == 64 && L.c_p <= 32 && L.c_r > 0 && !L.grouping) {
     if (cond_mode == CG_COND_COMPACT) return false;
-    L.c_in = 128; L.c_p = 32; L.c_r = 128; P.pad8 = 2;
+    L.c_in = 128; L.c_p = 32; L.c_r = 64; P.pad8 = 2;
   }
   if (in_dtype != CG_BF16 && in_dtype != CG_I8) return false;
   const int eb = in_dtype == CG_BF16 ? 2 : 1;
@@ -1448,6 +1455,7 @@ bool tc_plan(const LayerDims& L_in, int in_dtype, int cond_mode, TcPlan* plan) {
     const int tpt = ck / L.c_p;
     P.base_tiles = (taps + tpt - 1) / tpt;
     P.cond_tiles = L.c_r > 0 ? P.chunks * taps : 0;
+    if (P.pad8 == 2) P.cond_tiles = (taps + 1) / 2;
   }
   P.stage_rows = (int)align_up((size_t)max(kBM, P.wp * P.out_box_h * P.ni), 8);
   P.cond_mode = cond_mode == CG_COND_AUTO ? CG_COND_SKIP_TILES : cond_mode;
@@ -1531,25 +1539,25 @@ bool tc_device_ok(int device) {
 // CG_COND_COMPACT workspace: [row counts, 256 B][row lists: tiles_n x M x u32][row records:
 // tiles_n x M x (NT + 4) words]
 // int8 weights of a layer with 64 input channels, repacked with whole K steps (see tc_plan):
-// W_base [rows][c_p] -> [rows][32], W_cond [rows][64 - c_p] -> [rows][128] with the real channels at
-// their input-channel positions [c_p, 64); everything else zero.  rows = c_out * taps.
+// W_base [rows][c_p] -> [rows][32], W_cond [rows][64 - c_p] -> [rows][64] with the real channels at
+// their input-channel positions [c_p, 64) of 64; everything else zero.  rows = c_out * taps.
 __global__ void repack_i8_kernel(const int8_t* __restrict__ wb, const int8_t* __restrict__ wc, int8_t* __restrict__ wb32,
-                                 int8_t* __restrict__ wc128, int rows, int c_p) {
-  const int total = rows * 160;
+                                 int8_t* __restrict__ wc64, int rows, int c_p) {
+  const int total = rows * 96;
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
-    const int row = i / 160, c = i - row * 160;
+    const int row = i / 96, c = i - row * 96;
     if (c < 32) {
       wb32[(size_t)row * 32 + c] = c < c_p ? wb[(size_t)row * c_p + c] : (int8_t)0;
     } else {
       const int cc = c - 32;
-      wc128[(size_t)row * 128 + cc] = (cc >= c_p && cc < 64) ? wc[(size_t)row * (64 - c_p) + cc - c_p] : (int8_t)0;
+      wc64[(size_t)row * 64 + cc] = cc >= c_p ? wc[(size_t)row * (64 - c_p) + cc - c_p] : (int8_t)0;
     }
   }
 }
 
 static size_t repack_i8_bytes(const LayerDims& L) {
   const size_t rows = (size_t)L.c_out * L.kh * L.kw;
-  return align_up(rows * 32, 256) + align_up(rows * 128, 256);
+  return align_up(rows * 32, 256) + align_up(rows * 64, 256);
 }
 
 size_t tc_workspace_bytes(const LayerDims& L, const TcPlan& P) {
@@ -1576,7 +1584,7 @@ int launch_tc(const LayerDims& L_in, const TcPlan& P, int in_dtype, TcMaps* maps
                                              (int)rows, L_in.c_p);
     if (cudaGetLastError() != cudaSuccess) return (int)cudaErrorLaunchFailure;
     w_base = b; w_cond = c;
-    L.c_in = 128; L.c_p = 32; L.c_r = 128;
+    L.c_in = 128; L.c_p = 32; L.c_r = 64;
   } else if (P.pad8) {
     if (!workspace) return (int)cudaErrorInvalidValue;
     const int e = launch_repack8(L_in, w_base, w_cond, workspace, &w_base, &w_cond, stream);
