@@ -762,6 +762,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     const int quad = warp & 3;
     const int cgi = gate_group ? 0 : (warp - kEpiWarp0 - kGateWarps) >> 2;   // column quarter
     const int col0 = cgi * CW;
+    const bool phantom_cols = (int)(blockIdx.x % P.tiles_n) * NT + col0 >= L.c_out;   // (uniform over the warp)
     const int row = quad * 32 + lane;                      // TMEM lane = patch row i
     const int ct = threadIdx.x - kEpiThread0 - kGateWarps * 32;   // thread index within the combine group
     const int n_loc = P.images_mode ? row / P.ip : 0;
@@ -928,7 +929,9 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         for (int q = 0; q < 4; ++q)
           *(uint4*)(rec + colS + q * 4) = make_uint4(p[q * 4], p[q * 4 + 1], p[q * 4 + 2], p[q * 4 + 3]);
       }
-      if (I8) {
+      if (I8 && phantom_cols) {
+        // (columns behind c_out: nothing to compute, the y store clips them)
+      } else if (I8) {
         // quantised layer: z = acc*mul + off (64-bit), q = (z + 2^(S-1)) >> S, clamp to int8;
         // 32 channels = 32 bytes = two 16-byte pieces of a 128-channel staging row
         uint8_t* st = s_y + (size_t)(colS >> 7) * P.stage_rows * 128 + (size_t)row * 128;
