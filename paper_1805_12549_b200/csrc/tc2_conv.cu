@@ -403,7 +403,15 @@ tc2_gated_conv_kernel(const __grid_constant__ CUtensorMap map_r1,
           const int g0 = (first_m + jb * stride_m) * rows_per_job;
           for (int s = 0; s < ns && ok; ++s) {
             if (!(s_tab[s].flags & kStageNewChunk)) continue;
-            const int chunk = s_tab[s].chunk;
+            int chunk = s_tab[s].chunk;
+            if (L.grouping) {
+              // Channel grouping (Section 3.3): the channel tile lies inside one output group; its
+              // base path reads that group's input chunks, its conditional path the others in
+              // ascending order.  The weight tiles keep their K coordinates.
+              const int bc = L.c_p >> 6, own0 = (tile_c * 128) / (L.c_out / L.groups) * bc;
+              if (s_tab[s].flags & kStageCond) { const int i = chunk - bc; chunk = i < own0 ? i : i + bc; }
+              else chunk += own0;
+            }
             for (int X = 0; X < P.nsub && ok; ++X) {
               int cnt = 0;
               if (lane == 0) {
@@ -812,7 +820,9 @@ bool tc2_plan(const LayerDims& L, int in_dtype, int cond_mode, int sms, Tc2Plan*
   Tc2Plan& P = *plan;
   std::memset(&P, 0, sizeof(P));
   if (in_dtype != CG_BF16) return false;
-  if (L.grouping || L.stride != 1) return false;
+  if (L.stride != 1) return false;
+  // channel grouping: whole 64-channel chunks per input group, 128-channel tiles inside one output group
+  if (L.grouping && (L.c_p % 64 != 0 || (L.c_out / L.groups) % 128 != 0)) return false;
   if (L.kh != L.kw || L.kh != 2 * L.pad + 1) return false;
   if (L.c_in % 64 != 0 || L.c_out % 32 != 0) return false;
   if (!(L.c_p == 8 || L.c_p == 16 || L.c_p == 32 || L.c_p % 64 == 0)) return false;

@@ -607,8 +607,12 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         }
       };
       const int cond_part = P.split_a ? 1 : 0;
+      // Channel grouping (Section 3.3): the column tile lies inside one output group; its base
+      // path reads that group's input chunks, its conditional path the others in ascending order.
+      // The weight tiles keep their K coordinates: only the chunks of x change.
+      const int own0 = L.grouping ? (tile_n * NT) / (L.c_out / L.groups) * P.base_chunks : 0;
       for (int j = 0; j <= jobs && ok; ++j) {
-        if (j < jobs) { load_chunks(j, 0, P.base_chunks, 0); CG_PROF_EV(j, 0); }
+        if (j < jobs) { load_chunks(j, own0, own0 + P.base_chunks, 0); CG_PROF_EV(j, 0); }
         if (j >= 1 && has_cond && ok && !P.share_a) {
           const int jj = j - 1;
           uint32_t blocks = kAllBlocks;
@@ -617,7 +621,12 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
             if (!ok) break;
             blocks = __shfl_sync(0xffffffffu, slot_blocks(sh, jj % kNP), 0);
           }
-          if (blocks) load_chunks(jj, cond_first_chunk, P.chunks, cond_part);
+          if (blocks && L.grouping) {
+            load_chunks(jj, 0, own0, cond_part);
+            load_chunks(jj, own0 + P.base_chunks, P.chunks, cond_part);
+          } else if (blocks) {
+            load_chunks(jj, cond_first_chunk, P.chunks, cond_part);
+          }
         }
       }
     }
@@ -1405,7 +1414,8 @@ bool tc_plan(const LayerDims& L_in, int in_dtype, int cond_mode, TcPlan* plan) {
   const int eb = in_dtype == CG_BF16 ? 2 : 1;
   const int ck = 128 / eb;          // channels per 128-byte patch row
   const int kst = ck / 4;           // channels per MMA K step (32 bytes)
-  if (L.grouping) return false;
+  // channel grouping: whole 128-byte chunks per group, column tiles inside one output group
+  if (L.grouping && (in_dtype != CG_BF16 || L.c_p % ck != 0 || (L.c_out / L.groups) % 64 != 0 || cond_mode == CG_COND_COMPACT)) return false;
   if (L.has_residual && in_dtype != CG_BF16) return false;
   if (L.kh != L.kw || L.kh != 2 * L.pad + 1) return false;
   const bool s2 = L.stride == 2;
@@ -1474,6 +1484,7 @@ bool tc_plan(const LayerDims& L_in, int in_dtype, int cond_mode, TcPlan* plan) {
   for (int pass = 0; pass < 2; ++pass)
   for (int nt = 128; nt >= (eb == 1 ? 128 : 64); nt >>= 1) {
     if (L.c_out % nt != 0 && eb != 1) continue;
+    if (L.grouping && (L.c_out / L.groups) % nt != 0) continue;
     const size_t fixed = align_up((size_t)(nt * eb / 128) * P.stage_rows * 128, 1024) +
                          align_up((size_t)8 * nt * 4, 128) +
                          align_up((size_t)4 * 128 * (nt / 32) * 4, 128) +

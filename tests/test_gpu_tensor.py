@@ -303,3 +303,25 @@ def test_misaligned_workspace_is_refused_before_any_launch():
         g.conv.forward(g.x, g.wb, g.wc, g.bn, g.delta, g.y, g.mask, g.res)
     assert e.value.status == 4                               # CG_ERR_WORKSPACE
     g.close()
+
+
+GROUPED = [
+    (O.Shape(3, 14, 14, 256, 256, groups=4), "256 channels, G = 4: column tiles of 64 inside the groups"),
+    (O.Shape(5, 7, 7, 512, 512, groups=4), "512 channels, G = 4: column tiles of 128"),
+    (O.Shape(2, 14, 14, 256, 512, groups=4), "c_out != c_in"),
+    (O.Shape(2, 28, 28, 128, 128, groups=2), "G = 2 at 128 channels"),
+    (O.Shape(3, 14, 14, 256, 512, stride=2, groups=4), "stride 2"),
+    (O.Shape(2, 14, 14, 512, 512, groups=8), "G = 8 at 512 channels: groups of 64"),
+]
+
+
+@pytest.mark.parametrize("s,why", GROUPED, ids=[w for _, w in GROUPED])
+def test_channel_grouping_on_the_tensor_path(s, why):
+    """Section 3.3: output group i takes input group i as its base path and the other groups, in
+    ascending order, as its conditional path."""
+    c = K.make_float_case("tcgrp", s, "bf16", density=0.3, grouped=True)
+    ref, st, exempt = _run(c)
+    assert abs(st.density - ref.density) < 2e-3 and 0.2 < st.density < 0.4
+    c = K.make_float_case("tcgrp1", s, "bf16", delta=-K.INF, grouped=True)
+    ref, st, exempt = _run(c)
+    assert exempt == 0 and st.active == st.outputs

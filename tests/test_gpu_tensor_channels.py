@@ -199,3 +199,19 @@ def test_default_choice_of_tensor_kernel():
         conv = B.GatedConv(n, h, w, ci, co, k=3, stride=st, pad=1, groups=4, dtype=B.CG_BF16, algo=B.CG_ALGO_TENSOR)
         assert conv.kernel_id == want, conv.plan
         conv.close()
+
+
+GROUPED = [
+    (O.Shape(5, 7, 7, 512, 512, groups=4), "512 channels, G = 4: one 128-channel tile per output group"),
+    (O.Shape(3, 8, 8, 256, 256, groups=2), "256 channels, G = 2"),
+    (O.Shape(2, 14, 14, 256, 512, groups=4), "c_out != c_in"),
+]
+
+
+@pytest.mark.parametrize("s,why", GROUPED, ids=[w for _, w in GROUPED])
+def test_channel_grouping(s, why):
+    """Section 3.3: output group i takes input group i as its base path and the other groups, in
+    ascending order, as its conditional path."""
+    c = K.make_float_case("tc2grp", s, "bf16", density=0.3, grouped=True)
+    ref, st, exempt, _ = _run(c)
+    assert abs(st.density - ref.density) < 2e-3 and 0.2 < st.density < 0.4
