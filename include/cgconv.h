@@ -82,7 +82,9 @@ typedef struct {
                                    x_p (Fig. 5(a)).  1: channel grouping (Section 3.3, Fig. 5(b)):
                                    output group i = channels [i*c_out/G,(i+1)*c_out/G) takes input
                                    group i as x_p and the other groups, in ascending order, as
-                                   x_r; needs c_out % G == 0.  Direct kernels only.            */
+                                   x_r; needs c_out % G == 0.  Tensor-core kernels where an
+                                   input group is whole 64-channel chunks and an output group a
+                                   multiple of 64 (128) channels; direct kernels otherwise.     */
   float channel_tau;            /* tau_c of the channel-wise gate (Eq. 4).  0: off.  > 0: per
                                    image, an output channel whose gate fires at fewer than
                                    tau_c * h' * w' positions loses its conditional path (all its
@@ -140,8 +142,9 @@ typedef struct {
  * allocation for the counters (freed by cg_conv_destroy).  `*out` is set on CG_OK only.
  * Errors: CG_ERR_INVALID_ARG (NULL, extents <= 0, c_in % groups != 0, kh != kw, dtype pair not
  * listed above, shift out of range), CG_ERR_CUDA, and CG_ERR_UNSUPPORTED when a tensor-core
- * algo is asked for a layer outside the kernels' limits.  Those are: BF16 or I8; no channel
- * grouping, no channel-wise gate; odd square filter with pad = (k-1)/2; c_in a multiple of 64
+ * algo is asked for a layer outside the kernels' limits.  Those are: BF16 or I8; no channel-wise
+ * gate; channel grouping only for BF16 with c_in/G a multiple of 64 and c_out/G a multiple of 64
+ * (pixel-major) or 128 (channel-major); odd square filter with pad = (k-1)/2; c_in a multiple of 64
  * (BF16), a multiple of 128 or equal to 64 (I8);
  *   pixel-major kernel:   stride 1, or stride 2 for 3x3 filters on even extents; c_out a multiple
  *                         of 64; c_in/G equal to 8, 16 or 32 (BF16; 32 or 64 for I8, at most 32 when
