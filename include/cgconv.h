@@ -91,9 +91,11 @@ typedef struct {
                                    activations take Eq. 1's first case, its mask bits are 0);
                                    a count equal to tau_c*h'*w' keeps the channel (theta(0) = 1);
                                    the comparison is (float)count >= tau_c * (float)(h'*w').
-                                   Floating-point layers, direct kernels only: a memset of the
-                                   counts and two launches (partial sums and counts; decisions
-                                   and conditional path); needs the workspace
+                                   Floating-point layers.  BF16 layers the pixel-major tensor-core
+                                   kernel can run take two passes of it (base path and gate; the
+                                   whole layer with per-image thresholds) with two small kernels
+                                   in between; other layers run on the direct kernels (a memset of
+                                   the counts and two launches).  Needs the workspace
                                    cg_conv_workspace_bytes reports.                            */
 } cg_conv_desc;
 
@@ -142,8 +144,8 @@ typedef struct {
  * allocation for the counters (freed by cg_conv_destroy).  `*out` is set on CG_OK only.
  * Errors: CG_ERR_INVALID_ARG (NULL, extents <= 0, c_in % groups != 0, kh != kw, dtype pair not
  * listed above, shift out of range), CG_ERR_CUDA, and CG_ERR_UNSUPPORTED when a tensor-core
- * algo is asked for a layer outside the kernels' limits.  Those are: BF16 or I8; no channel-wise
- * gate; channel grouping only for BF16 with c_in/G a multiple of 64 and c_out/G a multiple of 64
+ * algo is asked for a layer outside the kernels' limits.  Those are: BF16 or I8; the channel-wise
+ * gate on the pixel-major kernel only; channel grouping only for BF16 with c_in/G a multiple of 64 and c_out/G a multiple of 64
  * (pixel-major) or 128 (channel-major); odd square filter with pad = (k-1)/2; c_in a multiple of 64
  * (BF16), a multiple of 128 or equal to 64 (I8);
  *   pixel-major kernel:   stride 1, or stride 2 for 3x3 filters on even extents; c_out a multiple

@@ -116,8 +116,9 @@ cg_status cg_conv_create(cg_conv_t* out, const cg_conv_desc* desc) {
   int sms = 0;
   if (!have_device || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess || sms <= 0) sms = 148;
   // the channel-wise gate needs every partial sum of an image before any conditional path: it
-  // runs on the direct kernels
-  const bool want_tc = desc->algo != CG_ALGO_DIRECT && !(desc->channel_tau > 0.f);
+  // runs as two passes of the pixel-major kernel (chan_gate.cu), or on the direct kernels
+  const bool chan = desc->channel_tau > 0.f;
+  const bool want_tc = desc->algo != CG_ALGO_DIRECT;
   // Two tensor-core kernels.  Measured on B200 (batch 64-256 ResNet-18 shapes), the channel-major
   // kernel is the faster one for 128 output channels, and for 256 channels on 8x8 images (where the
   // pixel-major kernel's whole-image tiles are half padding) or with 20,000 and more pixels (enough
@@ -125,11 +126,12 @@ cg_status cg_conv_create(cg_conv_t* out, const cg_conv_desc* desc) {
   // Each also takes the layers only it can run.
   const bool prefer2 = h->L.c_out == 128 ||
                        (h->L.c_out == 256 && (h->L.ho * h->L.wo <= 64 || h->L.m >= 20000));
-  const bool allow1 = desc->algo != CG_ALGO_TENSOR_CHANNELS, allow2 = desc->algo != CG_ALGO_TENSOR_ROWS;
+  const bool allow1 = desc->algo != CG_ALGO_TENSOR_CHANNELS, allow2 = desc->algo != CG_ALGO_TENSOR_ROWS && !chan;
+  const int cond_mode = (chan && desc->cond_mode == CG_COND_COMPACT) ? CG_COND_SKIP_TILES : desc->cond_mode;
   bool ok1 = false, ok2 = false;
-  if (want_tc && allow2 && (prefer2 || !allow1)) ok2 = cg::tc2_plan(h->L, desc->in_dtype, desc->cond_mode, sms, &h->plan2);
-  if (want_tc && allow1 && !ok2) ok1 = cg::tc_plan(h->L, desc->in_dtype, desc->cond_mode, &h->plan);
-  if (want_tc && allow2 && !ok1 && !ok2) ok2 = cg::tc2_plan(h->L, desc->in_dtype, desc->cond_mode, sms, &h->plan2);
+  if (want_tc && allow2 && (prefer2 || !allow1)) ok2 = cg::tc2_plan(h->L, desc->in_dtype, cond_mode, sms, &h->plan2);
+  if (want_tc && allow1 && !ok2) ok1 = cg::tc_plan(h->L, desc->in_dtype, cond_mode, &h->plan);
+  if (want_tc && allow2 && !ok1 && !ok2) ok2 = cg::tc2_plan(h->L, desc->in_dtype, cond_mode, sms, &h->plan2);
   h->use_tc2 = ok2;
   const bool tc_ok = ok1;
   const bool must_tc = desc->algo >= CG_ALGO_TENSOR;
@@ -158,6 +160,7 @@ void cg_conv_destroy(cg_conv_t h) {
 
 size_t cg_conv_workspace_bytes(cg_conv_t h) {
   if (!h) return 0;
+  if (h->L.channel_tau > 0.f && h->use_tc) return cg::tc_channel_gate_workspace_bytes(h->L, h->plan);
   if (h->L.channel_tau > 0.f) return cg::channel_gate_workspace_bytes(h->L);
   if (h->use_tc2) return cg::tc2_workspace_bytes(h->L, h->plan2);
   return h->use_tc ? cg::tc_workspace_bytes(h->L, h->plan) : 0;
@@ -165,7 +168,7 @@ size_t cg_conv_workspace_bytes(cg_conv_t h) {
 
 int cg_conv_launches_per_forward(cg_conv_t h) {
   if (!h) return 0;
-  if (h->L.channel_tau > 0.f) return 2;
+  if (h->L.channel_tau > 0.f) return h->use_tc ? 4 + 2 * (h->plan.pad8 ? 1 : 0) : 2;
   if (h->use_tc2) return h->plan2.pad8 ? 2 : 1;
   return (h->use_tc && (h->plan.cond_mode == CG_COND_COMPACT || h->plan.pad8)) ? 2 : 1;
 }
@@ -192,7 +195,6 @@ int cg_conv_plan_string(cg_conv_t h, char* buf, size_t len) {
 
 int cg_conv_kernel_id(cg_conv_t h) {
   if (!h) return -1;
-  if (h->L.channel_tau > 0.f) return CG_KERNEL_DIRECT;
   return h->use_tc2 ? CG_KERNEL_TENSOR_CHANNEL_MAJOR : (h->use_tc ? CG_KERNEL_TENSOR_PIXEL_MAJOR : CG_KERNEL_DIRECT);
 }
 
@@ -217,7 +219,10 @@ cg_status cg_conv_forward(cg_conv_t h, const void* x, const void* w_base, const 
   if (cur != h->device) return CG_ERR_INVALID_ARG;         // a handle belongs to the device it was created on
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   int err;
-  if (h->use_tc2) {
+  if (h->use_tc && h->L.channel_tau > 0.f) {
+    err = cg::launch_tc_channel_gate(h->L, h->plan, h->desc.in_dtype, &h->maps, x, w_base, w_cond, *bn, delta,
+                                     residual, y, mask_out, workspace, h->counters, stream);
+  } else if (h->use_tc2) {
     err = cg::launch_tc2(h->L, h->plan2, &h->maps2, x, w_base, w_cond, *bn, delta, residual, y,
                          mask_out, workspace, h->counters, stream);
   } else if (h->use_tc) {

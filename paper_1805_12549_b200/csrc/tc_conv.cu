@@ -68,6 +68,11 @@ struct TcParams {
   const __nv_bfloat16* residual;   // optional, same layout as y (bf16 layers)
   uint32_t* mask;
   unsigned long long* counters;
+  // Channel-wise gate (Eq. 4): thresholds per (image, channel), +inf where the channel is switched
+  // off for the image (NULL: the layer's own thresholds); base_only: no conditional path (the
+  // counting pass)
+  const float* t_img;
+  int base_only;
   // CG_COND_COMPACT: per column tile, the pixel rows in which a gate fired, with their partial
   // sums and mask words, for the second (gathered) kernel
   uint32_t* ws_counts;     // [tiles_n] rows listed so far
@@ -489,7 +494,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   const int taps = L.kh * L.kw;
   const bool dense = (P.cond_mode == CG_COND_DENSE);
   const bool compact = (P.cond_mode == CG_COND_COMPACT);   // R is computed by a second kernel
-  const bool has_cond = P.cond_tiles > 0 && !compact;
+  const bool has_cond = P.cond_tiles > 0 && !compact && !prm.base_only;
   const int cond_first_chunk = L.c_p >= P.ck ? P.base_chunks : 0;
   constexpr int kBlocks = NT / 64;
   // 64-channel column blocks of this tile that hold real output channels (the last tile of a
@@ -801,6 +806,8 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       const bool valid = (w_out < L.wo) && (h_loc < rows_here) && (n_loc < P.ni) && (n0 + n_loc < L.n);
       const long long m = ((long long)(n0 + n_loc) * L.ho + (h0 + h_loc)) * L.wo + w_out;
       uint32_t* g_words = prm.mask + m * L.words + tile_n * kWords;
+      // (channel-wise gate: the thresholds of this row's image)
+      const float* t_row = (!I8 && prm.t_img) ? prm.t_img + (size_t)(valid ? n0 + n_loc : 0) * L.c_out + tile_n * NT : nullptr;
       uint32_t* s_words = s_mask + (slot * 128 + row) * kWords;
       uint32_t fired_blocks = 0;
 #pragma unroll
@@ -818,7 +825,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
             pw[q & 3] |= ((int)r[w & 1][q * 4 + 2] >= t4.z ? 1u : 0u) << (q * 4 + 2);
             pw[q & 3] |= ((int)r[w & 1][q * 4 + 3] >= t4.w ? 1u : 0u) << (q * 4 + 3);
           } else {
-            const float4 t4 = *(const float4*)(s_t + w * 32 + q * 4);
+            const float4 t4 = t_row ? __ldg((const float4*)(t_row + w * 32 + q * 4)) : *(const float4*)(s_t + w * 32 + q * 4);
             pw[q & 3] |= (__uint_as_float(r[w & 1][q * 4 + 0]) >= t4.x ? 1u : 0u) << (q * 4 + 0);
             pw[q & 3] |= (__uint_as_float(r[w & 1][q * 4 + 1]) >= t4.y ? 1u : 0u) << (q * 4 + 1);
             pw[q & 3] |= (__uint_as_float(r[w & 1][q * 4 + 2]) >= t4.z ? 1u : 0u) << (q * 4 + 2);
@@ -1585,7 +1592,7 @@ size_t tc_workspace_bytes(const LayerDims& L, const TcPlan& P) {
 int launch_tc(const LayerDims& L_in, const TcPlan& P, int in_dtype, TcMaps* maps, const void* x,
               const void* w_base, const void* w_cond, const cg_bn_params& bn, const float* delta,
               const void* residual, void* y, uint32_t* mask, void* workspace,
-              unsigned long long* counters, cudaStream_t stream) {
+              unsigned long long* counters, cudaStream_t stream, const float* t_img, int base_only) {
   (void)in_dtype;
   if (!P.valid) return (int)cudaErrorInvalidValue;
   LayerDims L = L_in;
@@ -1663,6 +1670,7 @@ int launch_tc(const LayerDims& L_in, const TcPlan& P, int in_dtype, TcMaps* maps
   TcParams prm;
   prm.L = L; prm.P = P; prm.bn = bn; prm.delta = delta; prm.residual = (const __nv_bfloat16*)residual; prm.mask = mask; prm.counters = counters;
   prm.ws_counts = nullptr; prm.ws_list = nullptr; prm.ws_rows = nullptr;
+  prm.t_img = t_img; prm.base_only = base_only;
   const bool compact = P.cond_mode == CG_COND_COMPACT;
   if (compact) {
     if (!workspace) return (int)cudaErrorInvalidValue;

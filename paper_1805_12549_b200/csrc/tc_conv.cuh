@@ -65,6 +65,14 @@ size_t tc_workspace_bytes(const LayerDims& L, const TcPlan& plan);
 int launch_tc(const LayerDims& L, const TcPlan& plan, int in_dtype, TcMaps* maps, const void* x,
               const void* w_base, const void* w_cond, const cg_bn_params& bn, const float* delta,
               const void* residual, void* y, uint32_t* mask, void* workspace,
-              unsigned long long* counters, cudaStream_t stream);
+              unsigned long long* counters, cudaStream_t stream, const float* t_img = nullptr,
+              int base_only = 0);
+
+// Channel-wise gate (Eq. 4) through two passes of the pixel-major kernel (chan_gate.cu).
+size_t tc_channel_gate_workspace_bytes(const LayerDims& L, const TcPlan& plan);
+int launch_tc_channel_gate(const LayerDims& L, const TcPlan& plan, int in_dtype, TcMaps* maps, const void* x,
+                           const void* w_base, const void* w_cond, const cg_bn_params& bn, const float* delta,
+                           const void* residual, void* y, uint32_t* mask, void* workspace,
+                           unsigned long long* counters, cudaStream_t stream);
 
 }  // namespace cg

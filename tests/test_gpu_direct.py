@@ -164,7 +164,7 @@ def test_channel_wise_gate(s, dtype, tau):
     c = K.make_float_case("chgate", s, dtype, density=0.4)
     c.channel_tau = tau
     ref = K.run_oracle(c)
-    g = K.GpuCase(c)            # algo AUTO: the channel-wise gate selects the direct kernels
+    g = K.GpuCase(c, algo=1)    # the direct kernels
     assert not g.conv.uses_tensor_cores
     y, mask, st = g.run()
     K.compare(c, ref, y, mask, st, exact=True)
@@ -192,9 +192,9 @@ def test_channel_wise_gate_limits_and_rejections():
     assert st.active == 0 and st.channels_skipped == st.channels
     g.close()
     assert plain.active > 0
-    # tensor-core kernels and int8 layers do not take the channel-wise gate
+    # the channel-major kernel and int8 layers do not take the channel-wise gate
     with pytest.raises(B.CgError) as e:
-        B.GatedConv(2, 28, 28, 128, 128, algo=B.CG_ALGO_TENSOR, channel_tau=0.2)
+        B.GatedConv(2, 28, 28, 128, 128, algo=B.CG_ALGO_TENSOR_CHANNELS, channel_tau=0.2)
     assert e.value.status == 2
     with pytest.raises(B.CgError) as e:
         B.GatedConv(2, 28, 28, 128, 128, dtype=B.CG_I8, requant_shift=8, channel_tau=0.2)

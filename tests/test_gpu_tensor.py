@@ -325,3 +325,28 @@ def test_channel_grouping_on_the_tensor_path(s, why):
     c = K.make_float_case("tcgrp1", s, "bf16", delta=-K.INF, grouped=True)
     ref, st, exempt = _run(c)
     assert exempt == 0 and st.active == st.outputs
+
+
+CHANNEL_GATE = [
+    (O.Shape(3, 28, 28, 128, 128, groups=4), "128@28"),
+    (O.Shape(3, 14, 14, 256, 256, groups=4), "256@14, two column tiles"),
+    (O.Shape(2, 56, 56, 64, 64, groups=4), "64@56, one patch for both paths"),
+    (O.Shape(3, 28, 28, 128, 256, stride=2, groups=4), "stride 2"),
+    (O.Shape(5, 7, 7, 512, 512, groups=4), "two images per tile: thresholds per image inside a tile"),
+]
+
+
+@pytest.mark.parametrize("s,why", CHANNEL_GATE, ids=[w for _, w in CHANNEL_GATE])
+@pytest.mark.parametrize("tau", [0.3, 0.45])
+def test_channel_wise_gate_on_the_tensor_path(s, why, tau):
+    """Eq. 4 as two passes of the pixel-major kernel: the first counts the plain gate's decisions per
+    (image, channel), the second runs the layer with the switched-off channels' thresholds at +inf."""
+    c = K.make_float_case("tcchan", s, "bf16", density=0.4)
+    c.channel_tau = tau
+    ref, st, exempt = _run(c)
+    assert st.channels == ref.channels == s.n * s.c_out
+    assert st.channels_skipped == ref.channels_skipped
+    assert st.channels_skipped < st.channels
+    if tau > 0.4:
+        assert st.channels_skipped > 0, "the case should drop some channels"
+    assert st.calls == 1 and st.device_status == 0
