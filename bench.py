@@ -440,6 +440,30 @@ def run_network_block(args, peaks):
                     for s in net.specs},
     }
     inst.close()
+    # batch-1 latency (the regime of the paper's accelerator, Table 4): the same network and
+    # calibration, one image, CUDA-graph replay
+    inst1 = net.instance(1)
+    x1 = x[:1].contiguous()
+
+    def latency(reps=20):
+        inst1.forward(x1)
+        torch.cuda.synchronize()
+        g = capture(lambda: inst1.forward(x1), args.no_graph)
+        g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            g.replay()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    out["batch1_latency_ms"] = round(latency(), 4)
+    net.set_density(1.0)
+    out["batch1_latency_ms_density1"] = round(latency(), 4)
+    net.set_density(tau)
+    inst1.close()
     return out
 
 
