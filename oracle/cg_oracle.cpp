@@ -69,6 +69,9 @@ struct cgo_desc {
   int32_t gate_form;    // 0: merged gate of Eq. 3; 1: normalise P first, then compare with Delta
   int32_t grouped;      // 0: Fig. 5(a), base = channels [0,c_in/G); 1: Fig. 5(b), channel grouping
   float channel_tau;    // tau_c of the channel-wise gate (Eq. 4); <= 0: no channel-wise gate
+  const float* delta_high;   // [c_out] upper thresholds of the two-sided gate of Section 3.2,
+                             // s = theta(Delta_h - x) o theta(x - Delta_l), in normalised units
+                             // like Delta; NULL: the one-sided gate theta(x - Delta)
 };
 
 struct cgo_counts {
@@ -240,6 +243,20 @@ int gated_conv_impl(const cgo_desc* d, const float* x, const float* w_base, cons
             const float centred = p - gm[co];
             const float p_hat = centred / sg;
             fire = (p_hat >= delta[co]);
+          }
+          // Two-sided gate (Section 3.2): the activation must also stay below the upper
+          // threshold; theta(0) = 1 on this side too.
+          if (d->delta_high) {
+            const float sg = std::sqrt(gv[co] + d->bn_eps);
+            if (d->gate_form == 0) {
+              const float prod = d->delta_high[co] * sg;
+              const float t_hi = prod + gm[co];
+              fire = fire && (p <= t_hi);
+            } else {
+              const float centred = p - gm[co];
+              const float p_hat = centred / sg;
+              fire = fire && (p_hat <= d->delta_high[co]);
+            }
           }
           fire_all[(size_t)(m * d->c_out + co)] = fire ? 1 : 0;
         }

@@ -37,7 +37,7 @@ class _Desc(C.Structure):
                                          "groups")] + \
                [("bn_eps", C.c_float)] + \
                [(k, C.c_int32) for k in ("relu", "out_bf16", "acc_double", "gate_form", "grouped")] + \
-               [("channel_tau", C.c_float)]
+               [("channel_tau", C.c_float), ("delta_high", C.c_void_p)]
 
 
 class _Counts(C.Structure):
@@ -161,13 +161,17 @@ def fold_params(s: Shape, bn: dict, delta) -> dict:
 
 
 def gated_conv(s: Shape, x, w_base, w_cond, bn: dict, delta, residual=None, *, out_bf16=False,
-               acc_double=False, gate_form=0, grouped=False, channel_tau=0.0) -> Result:
+               acc_double=False, gate_form=0, grouped=False, channel_tau=0.0, delta_high=None) -> Result:
     """Floating-point gated layer.  bn holds gamma, beta, mean_base, var_base, mean_full,
     var_full and optionally gate_mean, gate_var (absent/None: BN1's statistics).
     channel_tau > 0 adds the channel-wise gate of Eq. 4."""
     d = _Desc(s.n, s.h, s.w, s.c_in, s.c_out, s.kh, s.kw, s.stride, s.pad, s.groups, s.bn_eps,
               s.relu, int(out_bf16), int(acc_double), int(gate_form), int(grouped),
-              float(channel_tau))
+              float(channel_tau), None)
+    delta_high = _f32(delta_high)
+    if delta_high is not None:
+        assert delta_high.size == s.c_out
+        d.delta_high = delta_high.ctypes.data     # two-sided gate of Section 3.2
     x = _f32(x)
     w_base = _f32(w_base)
     w_cond = _f32(w_cond)

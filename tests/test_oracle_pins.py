@@ -485,3 +485,60 @@ def test_reordering_output_channels_only_relabels_the_layer():
     assert w2c.size == 0
     b = O.gated_conv(s2, got.y, w2p, w2c, bn2, shut)
     np.testing.assert_allclose(b.y, a.y, rtol=0, atol=1e-5)     # same products, summed in another order
+
+
+# --------------------------------------------------------------------------- two-sided gate
+@pytest.mark.parametrize("s", SHAPES[:3])
+def test_two_sided_gate_keeps_the_band_between_the_thresholds(s):
+    """Section 3.2: s(x, Delta_h, Delta_l) = theta(Delta_h - x) o theta(x - Delta_l).  An
+    activation takes Eq. 1's second case iff its normalised partial sum lies in
+    [Delta_l, Delta_h]; decided here from the library partial sums (away from near-ties)."""
+    x, wb, wc, bn = make_layer(("band", s.c_in, s.h), s)
+    g = synth.rng("band-delta", s.c_in)
+    lo = g.uniform(-0.8, 0.0, s.c_out).astype(np.float32)
+    hi = (lo + g.uniform(0.3, 1.2, s.c_out)).astype(np.float32)
+    res = O.gated_conv(s, x, wb, wc, bn, lo, delta_high=hi)
+    p_ref = lib_conv64(x[..., :s.c_p], wb, s.stride, s.pad)
+    full_ref = lib_conv64(x, np.concatenate([wb, wc], axis=3), s.stride, s.pad)
+    sg = np.sqrt(bn["gate_var"].astype(np.float64) + s.bn_eps)
+    t_lo = lo.astype(np.float64) * sg + bn["gate_mean"].astype(np.float64)
+    t_hi = hi.astype(np.float64) * sg + bn["gate_mean"].astype(np.float64)
+    d_ref = (p_ref >= t_lo) & (p_ref <= t_hi)
+    clear = (np.abs(p_ref - t_lo) > 1e-4) & (np.abs(p_ref - t_hi) > 1e-4)
+    d = O.unpack_mask(res.mask, s.c_out).reshape(p_ref.shape)
+    assert (d == d_ref)[clear].all()
+    y_ref = np.where(d, bn_relu64(full_ref, bn["gamma"], bn["beta"], bn["mean_full"], bn["var_full"], s.bn_eps),
+                     bn_relu64(p_ref, bn["gamma"], bn["beta"], bn["mean_base"], bn["var_base"], s.bn_eps))
+    np.testing.assert_allclose(res.y, y_ref, rtol=1e-5, atol=1e-5)
+    one_sided = O.gated_conv(s, x, wb, wc, bn, lo)
+    assert 0 < res.active < one_sided.active, "the upper threshold must shut some gates"
+    assert res.active == int(d.sum())
+    assert res.cond_macs == s.kh * s.kw * s.c_r * res.active
+
+
+def test_two_sided_gate_limits_and_ties():
+    """Delta_h = +inf is the one-sided gate; Delta_h below Delta_l shuts everything; a partial sum
+    equal to the upper threshold still fires (theta(0) = 1), the next float above does not; the
+    normalise-then-compare form agrees with the merged one away from ties."""
+    s = O.Shape(1, 6, 6, 8, 8, groups=4)
+    x, wb, wc, bn = make_layer(("band2", 1), s)
+    lo = np.full(s.c_out, -0.2, np.float32)
+    one = O.gated_conv(s, x, wb, wc, bn, lo)
+    same = O.gated_conv(s, x, wb, wc, bn, lo, delta_high=np.full(s.c_out, INF, np.float32))
+    np.testing.assert_array_equal(one.mask, same.mask)
+    np.testing.assert_array_equal(one.y, same.y)
+    none = O.gated_conv(s, x, wb, wc, bn, lo, delta_high=np.full(s.c_out, -0.5, np.float32))
+    assert none.active == 0
+    # exact tie at the upper threshold: unit statistics, eps = 0, Delta_h = a partial sum itself
+    s0 = O.Shape(1, 6, 6, 8, 8, groups=4, bn_eps=0.0)
+    bn0 = dict(bn, gate_mean=np.zeros(s.c_out, np.float32), gate_var=np.ones(s.c_out, np.float32))
+    shut = np.full(s.c_out, -INF, np.float32)
+    p = O.gated_conv(s0, x, wb, wc, bn0, shut).p.reshape(-1, s.c_out)
+    hi = p[7].copy()                                   # pixel 7's partial sums as upper thresholds
+    tie = O.gated_conv(s0, x, wb, wc, bn0, shut, delta_high=hi)
+    assert O.unpack_mask(tie.mask, s.c_out)[7].all()
+    below = O.gated_conv(s0, x, wb, wc, bn0, shut, delta_high=np.nextafter(hi, np.float32(-INF)))
+    assert not O.unpack_mask(below.mask, s.c_out)[7].any()
+    merged = O.gated_conv(s, x, wb, wc, bn, lo, delta_high=lo + np.float32(0.7))
+    split = O.gated_conv(s, x, wb, wc, bn, lo, delta_high=lo + np.float32(0.7), gate_form=1)
+    assert (O.unpack_mask(merged.mask, s.c_out) != O.unpack_mask(split.mask, s.c_out)).sum() <= 2
