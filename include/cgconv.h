@@ -119,6 +119,11 @@ typedef struct {
   const int32_t* q_mul_full;
   const int64_t* q_off_base;
   const int64_t* q_off_full;
+  /* Two-sided gate of Section 3.2, s = theta(Delta_h - x) o theta(x - Delta_l), for networks whose
+   * activation saturates on both sides: upper thresholds Delta_h[c] in the same normalised units
+   * as `delta` (which is then Delta_l); a gate fires iff Delta_l <= x^ <= Delta_h, ties included.
+   * NULL: the one-sided gate theta(x - Delta).  Floating-point layers only. */
+  const float* delta_high;
 } cg_bn_params;
 
 /* Counters accumulated by cg_conv_forward since the last cg_conv_stats. */

@@ -40,7 +40,8 @@ class CgConvDesc(C.Structure):
 class CgBnParams(C.Structure):
     _fields_ = [(k, C.c_void_p) for k in ("gamma", "beta", "mean_base", "var_base", "mean_full",
                                           "var_full", "gate_mean", "gate_var", "q_gate_thr",
-                                          "q_mul_base", "q_mul_full", "q_off_base", "q_off_full")]
+                                          "q_mul_base", "q_mul_full", "q_off_base", "q_off_full",
+                                          "delta_high")]
 
 
 class CgStats(C.Structure):

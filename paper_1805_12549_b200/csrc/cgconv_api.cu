@@ -72,6 +72,7 @@ cg_status check_bn(const cg_conv_s* h, const cg_bn_params* bn, const float* delt
   if (h->desc.in_dtype == CG_I8) {
     if (!bn->q_gate_thr || !bn->q_mul_base || !bn->q_mul_full || !bn->q_off_base || !bn->q_off_full)
       return CG_ERR_INVALID_ARG;
+    if (bn->delta_high) return CG_ERR_INVALID_ARG;      // the two-sided gate is defined for floating-point layers
   } else {
     if (!bn->gamma || !bn->beta || !bn->mean_base || !bn->var_base || !bn->mean_full || !bn->var_full)
       return CG_ERR_INVALID_ARG;

@@ -43,6 +43,7 @@ enum CounterSlot {
 // a = gamma/sqrt(var+eps), b = beta - a*mean  (a batch norm at inference is a scale and shift).
 struct ChannelConsts {
   float t, a1, b1, a2, b2;
+  float t2;   // upper threshold of the two-sided gate (Section 3.2); +inf for the one-sided gate
 };
 
 __device__ __forceinline__ ChannelConsts fold_channel(const cg_bn_params& bn, const float* delta,
@@ -52,6 +53,7 @@ __device__ __forceinline__ ChannelConsts fold_channel(const cg_bn_params& bn, co
   const float* gv = bn.gate_var ? bn.gate_var : bn.var_base;
   const float sg = __fsqrt_rn(__fadd_rn(gv[c], eps));
   k.t = __fadd_rn(__fmul_rn(delta[c], sg), gm[c]);
+  k.t2 = bn.delta_high ? __fadd_rn(__fmul_rn(bn.delta_high[c], sg), gm[c]) : __int_as_float(0x7f800000);
   const float g = bn.gamma[c], be = bn.beta[c];
   k.a1 = __fdiv_rn(g, __fsqrt_rn(__fadd_rn(bn.var_base[c], eps)));
   k.b1 = __fsub_rn(be, __fmul_rn(k.a1, bn.mean_base[c]));

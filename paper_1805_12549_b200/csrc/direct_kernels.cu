@@ -95,18 +95,19 @@ direct_gated_conv_kernel(LayerDims L, const TIn* __restrict__ x, const TIn* __re
   // and output channel, the number of firing gates to chan_cnt; 2 = second pass: partial sums
   // read back from p_out, conditional path only where the activation's gate fires AND the
   // channel's count reaches chan_need = tau_c * h' * w'.
-  extern __shared__ float s_consts[];   // 5 * c_out: t, a1, b1, a2, b2
+  extern __shared__ float s_consts[];   // 6 * c_out: t, a1, b1, a2, b2, t2
   __shared__ unsigned long long s_active;
   float* s_t = s_consts;
   float* s_a1 = s_t + L.c_out;
   float* s_b1 = s_a1 + L.c_out;
   float* s_a2 = s_b1 + L.c_out;
   float* s_b2 = s_a2 + L.c_out;
+  float* s_t2 = s_b2 + L.c_out;
   if (threadIdx.x == 0) s_active = 0ull;
   if (!base_only) {
     for (int c = threadIdx.x; c < L.c_out; c += blockDim.x) {
       const ChannelConsts k = fold_channel(bn, delta, L.eps, c);
-      s_t[c] = k.t; s_a1[c] = k.a1; s_b1[c] = k.b1; s_a2[c] = k.a2; s_b2[c] = k.b2;
+      s_t[c] = k.t; s_a1[c] = k.a1; s_b1[c] = k.b1; s_a2[c] = k.a2; s_b2[c] = k.b2; s_t2[c] = k.t2;
     }
   }
   __syncthreads();
@@ -133,9 +134,9 @@ direct_gated_conv_kernel(LayerDims L, const TIn* __restrict__ x, const TIn* __re
         p_out[m * L.c_out + co] = p;
       } else if (chan_pass == 1) {
         p_out[m * L.c_out + co] = p;
-        if (p >= s_t[co]) atomicAdd(&chan_cnt[(long long)n * L.c_out + co], 1);
+        if (p >= s_t[co] && p <= s_t2[co]) atomicAdd(&chan_cnt[(long long)n * L.c_out + co], 1);
       } else {
-        fire = (p >= s_t[co]);   // NaN compares false
+        fire = (p >= s_t[co]) && (p <= s_t2[co]);   // NaN compares false; t2 = +inf unless the gate is two-sided
         if (chan_pass == 2) {
           const bool on = ((float)chan_cnt[(long long)n * L.c_out + co] >= chan_need);
           fire = fire && on;
@@ -244,7 +245,7 @@ int launch_direct(const LayerDims& L, int in_dtype, const void* x, const void* w
   long long blocks = (items + warps_per_block - 1) / warps_per_block;
   const long long cap = 148ll * 8 * 8;
   if (blocks > cap) blocks = cap;
-  const size_t smem = (size_t)5 * L.c_out * sizeof(float);
+  const size_t smem = (size_t)6 * L.c_out * sizeof(float);
   if (in_dtype == CG_F32) {
     direct_gated_conv_kernel<float, float><<<(unsigned)blocks, kThreads, smem, stream>>>(
         L, (const float*)x, (const float*)w_base, (const float*)w_cond, bn, delta,
@@ -284,7 +285,7 @@ int launch_direct_channel_gate(const LayerDims& L, int in_dtype, const void* x, 
   long long blocks = (items + warps_per_block - 1) / warps_per_block;
   const long long cap = 148ll * 8 * 8;
   if (blocks > cap) blocks = cap;
-  const size_t smem = (size_t)5 * L.c_out * sizeof(float);
+  const size_t smem = (size_t)6 * L.c_out * sizeof(float);
   // Eq. 4's threshold on the count, in fp32 like the comparison itself
   const float need = L.channel_tau * (float)(L.ho * L.wo);
   for (int pass = 1; pass <= 2; ++pass) {

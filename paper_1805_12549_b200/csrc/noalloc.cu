@@ -112,7 +112,7 @@ extern "C" cg_status cg_conv_forward_static(const cg_conv_desc* d, const void* x
     return CG_ERR_INVALID_ARG;
   if (d->in_dtype != d->out_dtype || (d->in_dtype != CG_F32 && d->in_dtype != CG_BF16))
     return CG_ERR_UNSUPPORTED;
-  if (d->grouping || d->channel_tau > 0.f) return CG_ERR_UNSUPPORTED;
+  if (d->grouping || d->channel_tau > 0.f || bn->delta_high) return CG_ERR_UNSUPPORTED;
   if (d->c_out > kMaxChannels) return CG_ERR_WORKSPACE;   // would not fit the static scratch
   if (!bn->gamma || !bn->beta || !bn->mean_base || !bn->var_base || !bn->mean_full || !bn->var_full ||
       (bn->gate_mean == nullptr) != (bn->gate_var == nullptr))

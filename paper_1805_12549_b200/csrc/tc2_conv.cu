@@ -123,6 +123,7 @@ __device__ __forceinline__ void set_max_regs_dec() {
 // layout: channels ch0 + 8*ci + lane/4, ci = 0..3, of the warp's 32.
 struct Consts4 {
   float kt[4], ka1[4], kb1[4], ka2[4], kb2[4];
+  float kt2[4];   // upper thresholds of the two-sided gate (Section 3.2), +inf for the one-sided gate
 };
 
 // What an epilogue thread keeps of a sub-tile between its gate pass and its combine pass.  Lane l
@@ -207,7 +208,7 @@ __device__ __forceinline__ void gate_pass(const Tc2Params& prm, Keep& kp, const 
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
           const float a = __uint_as_float((ci >> 1) ? r1[4 * oct + 2 * (ci & 1) + e] : r0[4 * oct + 2 * (ci & 1) + e]);
-          d[e] = a >= kc.kt[ci];                             // Eq. 2: a tie fires, NaN does not
+          d[e] = a >= kc.kt[ci] && a <= kc.kt2[ci];          // Eq. 2 (two-sided: Section 3.2): ties fire, NaN does not
           float v = fmaf(kc.ka1[ci], a, kc.kb1[ci]);         // BN1 of the partial sum (Section 4)
           if (kHasRes) {
             const uint32_t oj = __shfl_sync(0xffffffffu, offs, slot0 + 8 * oct + 2 * (lane & 3) + e);
@@ -602,10 +603,10 @@ tc2_gated_conv_kernel(const __grid_constant__ CUtensorMap map_r1,
     Consts4 kc;
 #pragma unroll
     for (int ci = 0; ci < 4; ++ci) {
-      kc.kt[ci] = 0.f; kc.ka1[ci] = 0.f; kc.kb1[ci] = 0.f; kc.ka2[ci] = 0.f; kc.kb2[ci] = 0.f;
+      kc.kt[ci] = 0.f; kc.ka1[ci] = 0.f; kc.kb1[ci] = 0.f; kc.ka2[ci] = 0.f; kc.kb2[ci] = 0.f; kc.kt2[ci] = 0.f;
       if (ch_valid && jobs > 0) {
         const ChannelConsts k = fold_channel(prm.bn, prm.delta, L.eps, ch0 + 8 * ci + (lane >> 2));
-        kc.kt[ci] = k.t; kc.ka1[ci] = k.a1; kc.kb1[ci] = k.b1; kc.ka2[ci] = k.a2; kc.kb2[ci] = k.b2;
+        kc.kt[ci] = k.t; kc.ka1[ci] = k.a1; kc.kb1[ci] = k.b1; kc.ka2[ci] = k.a2; kc.kb2[ci] = k.b2; kc.kt2[ci] = k.t2;
       }
     }
     const float lo = L.relu ? 0.f : -__int_as_float(0x7f800000);   // f = ReLU, or the identity

@@ -35,6 +35,7 @@
 // copies and MMAs.  Every mbarrier wait is bounded; on expiry the CTA records
 // CG_ERR_DEVICE_TIMEOUT with the id of the wait and leaves.
 #include <cstring>
+#include <type_traits>
 
 #include "ptx.cuh"
 #include "tc_conv.cuh"
@@ -475,6 +476,8 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   // layers reuse the region: threshold, two multipliers (int32), two offsets (int64).
   float* s_t = (float*)(smem + P.off_consts);
   float4* s_k = (float4*)(s_t + NT);                       // per channel {a1, b1, a2, b2}
+  float* s_t2 = s_t + 5 * NT;                              // upper thresholds of the two-sided gate (Section 3.2)
+  const bool two_sided = !I8 && prm.bn.delta_high != nullptr;
   int* s_qt = (int*)s_t;
   int* s_qm1 = s_qt + NT;
   int* s_qm2 = s_qm1 + NT;
@@ -499,8 +502,10 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
   constexpr int kBlocks = NT / 64;
   // 64-channel column blocks of this tile that hold real output channels (the last tile of a
   // layer whose c_out is not a multiple of NT holds fewer)
-  const int real_blocks = min(kBlocks, (L.c_out - (int)(blockIdx.x % P.tiles_n) * NT + 63) / 64);
+  // (bf16 layers: c_out is a multiple of NT, the count is a compile-time constant)
+  const int real_blocks = I8 ? min(kBlocks, (L.c_out - (int)(blockIdx.x % P.tiles_n) * NT + 63) / 64) : kBlocks;
   const uint32_t kAllBlocks = (1u << real_blocks) - 1u;
+  const int words_here = 2 * real_blocks;                  // mask words of this tile that belong to real channels
   constexpr int kWords = NT / 32;
   constexpr int kNP = NT == 64 ? 4 : 3;      // P accumulators in TMEM
   constexpr int kNR = NT == 64 ? 4 : 1;      // R accumulators in TMEM
@@ -568,7 +573,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
         s_qo1[c] = real ? prm.bn.q_off_base[cg_] : 0ll; s_qo2[c] = real ? prm.bn.q_off_full[cg_] : 0ll;
       } else {
         const ChannelConsts k = fold_channel(prm.bn, prm.delta, L.eps, cg_);
-        s_t[c] = k.t; s_k[c] = make_float4(k.a1, k.b1, k.a2, k.b2);
+        s_t[c] = k.t; s_k[c] = make_float4(k.a1, k.b1, k.a2, k.b2); s_t2[c] = k.t2;
       }
     }
     ptx::named_bar_sync(2, kEpiThreads);
@@ -776,7 +781,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     const int quad = warp & 3;
     const int cgi = gate_group ? 0 : (warp - kEpiWarp0 - kGateWarps) >> 2;   // column quarter
     const int col0 = cgi * CW;
-    const bool phantom_cols = (int)(blockIdx.x % P.tiles_n) * NT + col0 >= L.c_out;   // (uniform over the warp)
+    const bool phantom_cols = I8 && (int)(blockIdx.x % P.tiles_n) * NT + col0 >= L.c_out;   // (uniform over the warp)
     const int row = quad * 32 + lane;                      // TMEM lane = patch row i
     const int ct = threadIdx.x - kEpiThread0 - kGateWarps * 32;   // thread index within the combine group
     const int n_loc = P.images_mode ? row / P.ip : 0;
@@ -789,7 +794,11 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     bool ok = true;
 
     // gate of job j: P -> mask words (global + stash), block activity flags
-    auto gate_pass = [&](int j) {
+    // (kExtra: thresholds per image -- the channel-wise gate -- and/or upper thresholds -- the
+    // two-sided gate; the plain gate keeps its own, shorter instruction stream: the gate warps are
+    // on the critical path of the 64-channel layers)
+    auto gate_pass = [&](int j, auto extra_tag) {
+      constexpr bool kExtra = decltype(extra_tag)::value;
       const int slot = j % kNP;
       ok = wait_bar(cx, &sh->base_done[slot], (j / kNP) & 1, 11);
       if (!ok) return;
@@ -807,7 +816,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       const long long m = ((long long)(n0 + n_loc) * L.ho + (h0 + h_loc)) * L.wo + w_out;
       uint32_t* g_words = prm.mask + m * L.words + tile_n * kWords;
       // (channel-wise gate: the thresholds of this row's image)
-      const float* t_row = (!I8 && prm.t_img) ? prm.t_img + (size_t)(valid ? n0 + n_loc : 0) * L.c_out + tile_n * NT : nullptr;
+      const float* t_row = (kExtra && !I8 && prm.t_img) ? prm.t_img + (size_t)(valid ? n0 + n_loc : 0) * L.c_out + tile_n * NT : nullptr;
       uint32_t* s_words = s_mask + (slot * 128 + row) * kWords;
       uint32_t fired_blocks = 0;
 #pragma unroll
@@ -825,7 +834,8 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
             pw[q & 3] |= ((int)r[w & 1][q * 4 + 2] >= t4.z ? 1u : 0u) << (q * 4 + 2);
             pw[q & 3] |= ((int)r[w & 1][q * 4 + 3] >= t4.w ? 1u : 0u) << (q * 4 + 3);
           } else {
-            const float4 t4 = t_row ? __ldg((const float4*)(t_row + w * 32 + q * 4)) : *(const float4*)(s_t + w * 32 + q * 4);
+            float4 t4 = *(const float4*)(s_t + w * 32 + q * 4);
+            if constexpr (kExtra) { if (t_row) t4 = __ldg((const float4*)(t_row + w * 32 + q * 4)); }
             pw[q & 3] |= (__uint_as_float(r[w & 1][q * 4 + 0]) >= t4.x ? 1u : 0u) << (q * 4 + 0);
             pw[q & 3] |= (__uint_as_float(r[w & 1][q * 4 + 1]) >= t4.y ? 1u : 0u) << (q * 4 + 1);
             pw[q & 3] |= (__uint_as_float(r[w & 1][q * 4 + 2]) >= t4.z ? 1u : 0u) << (q * 4 + 2);
@@ -833,10 +843,23 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
           }
         }
         uint32_t word = (pw[0] | pw[1]) | (pw[2] | pw[3]);
-        if (!valid || tile_n * kWords + w >= L.words) word = 0;
+        if (kExtra && two_sided) {
+          // Section 3.2: the gate also needs P <= the upper threshold (ties included)
+          uint32_t ph[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const float4 u4 = *(const float4*)(s_t2 + w * 32 + q * 4);
+            ph[q & 3] |= (__uint_as_float(r[w & 1][q * 4 + 0]) <= u4.x ? 1u : 0u) << (q * 4 + 0);
+            ph[q & 3] |= (__uint_as_float(r[w & 1][q * 4 + 1]) <= u4.y ? 1u : 0u) << (q * 4 + 1);
+            ph[q & 3] |= (__uint_as_float(r[w & 1][q * 4 + 2]) <= u4.z ? 1u : 0u) << (q * 4 + 2);
+            ph[q & 3] |= (__uint_as_float(r[w & 1][q * 4 + 3]) <= u4.w ? 1u : 0u) << (q * 4 + 3);
+          }
+          word &= (ph[0] | ph[1]) | (ph[2] | ph[3]);
+        }
+        if (!valid || w >= words_here) word = 0;
         s_words[w] = word;
         st_active += __popc(word);
-        if (valid && prm.mask && tile_n * kWords + w < L.words) g_words[w] = word;
+        if (valid && prm.mask && w < words_here) g_words[w] = word;
         if (__ballot_sync(0xffffffffu, word != 0u)) fired_blocks |= 1u << (w >> 1);
       }
       // 64-channel column blocks with a firing gate, over the warp
@@ -1044,7 +1067,11 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
     };
 
     if (gate_group) {
-      for (int j = 0; j < jobs && ok; ++j) gate_pass(j);
+      if (prm.t_img || two_sided) {
+        for (int j = 0; j < jobs && ok; ++j) gate_pass(j, std::true_type{});
+      } else {
+        for (int j = 0; j < jobs && ok; ++j) gate_pass(j, std::false_type{});
+      }
     } else {
       for (int j = 0; j < jobs && ok; ++j) combine_pass(j);
       if (ct == 0) ptx::tma_store_wait_all();

@@ -31,6 +31,7 @@ class Case:
     shift: int = 0
     grouped: bool = False
     channel_tau: float = 0.0    # tau_c of the channel-wise gate (Eq. 4); 0 = off
+    delta_high: np.ndarray | None = None   # upper thresholds of the two-sided gate (Section 3.2)
 
 
 def _quantile_delta(p_hat: np.ndarray, density: float) -> float:
@@ -108,7 +109,7 @@ def run_oracle(c: Case, **kw) -> O.Result:
         return O.gated_conv_i8(c.s, c.shift, c.x, c.wb, c.wc, c.bn)
     return O.gated_conv(c.s, c.x, c.wb, c.wc, c.bn, c.delta, c.residual,
                         out_bf16=(c.dtype == "bf16"), grouped=c.grouped,
-                        channel_tau=c.channel_tau, **kw)
+                        channel_tau=c.channel_tau, delta_high=c.delta_high, **kw)
 
 
 # ----------------------------------------------------------------------------- GPU side
@@ -147,6 +148,8 @@ class GpuCase:
             if v is None:
                 continue
             self.params[k] = torch.from_numpy(np.ascontiguousarray(v)).cuda()
+        if c.delta_high is not None:
+            self.params["delta_high"] = torch.from_numpy(np.ascontiguousarray(c.delta_high, np.float32)).cuda()
         self.bn = B.make_bn(self.params)
         self.delta = None if c.delta is None else torch.from_numpy(c.delta).cuda()
         # y, mask and the workspace sit inside larger buffers whose margins hold a known pattern:
@@ -228,6 +231,8 @@ def compare(c: Case, ref: O.Result, y, mask, st, exact=False):
         with np.errstate(invalid="ignore"):
             p_hat = (p - gm) / np.sqrt(gv.astype(np.float64) + s.bn_eps)
             near = np.abs(p_hat - c.delta.astype(np.float64)) < NEAR_TIE
+            if c.delta_high is not None:      # two-sided gate: a tie at either threshold may flip
+                near |= np.abs(p_hat - c.delta_high.astype(np.float64)) < NEAR_TIE
         diff = d_ref != d_gpu
         bad = diff & ~near
         assert not bad.any(), f"{int(bad.sum())} gate decisions differ away from the threshold"

@@ -202,3 +202,18 @@ def test_channel_wise_gate_limits_and_rejections():
     with pytest.raises(B.CgError) as e:
         B.GatedConv(2, 8, 8, 16, 16, channel_tau=-0.1)
     assert e.value.status == 1
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_two_sided_gate_on_the_direct_path(dtype):
+    """Section 3.2 through the C ABI: upper thresholds in cg_bn_params.delta_high; bit-exact."""
+    s = O.Shape(2, 9, 10, 12, 40, groups=4)
+    c = K.make_float_case("band", s, dtype, density=0.5)
+    one_sided = K.run_oracle(c)
+    c.delta_high = (c.delta + np.float32(0.8)).astype(np.float32)
+    ref = K.run_oracle(c)
+    g = K.GpuCase(c, algo=1)
+    y, mask, st = g.run()
+    K.compare(c, ref, y, mask, st, exact=True)
+    assert 0 < ref.active < one_sided.active and st.active == ref.active
+    g.close()

@@ -350,3 +350,21 @@ def test_channel_wise_gate_on_the_tensor_path(s, why, tau):
     if tau > 0.4:
         assert st.channels_skipped > 0, "the case should drop some channels"
     assert st.calls == 1 and st.device_status == 0
+
+
+TWO_SIDED = [
+    (O.Shape(3, 28, 28, 128, 128, groups=4), "128@28"),
+    (O.Shape(3, 14, 14, 256, 256, groups=4), "256@14"),
+    (O.Shape(3, 8, 8, 256, 256, groups=4), "256@8"),
+]
+
+
+@pytest.mark.parametrize("s,why", TWO_SIDED, ids=[w for _, w in TWO_SIDED])
+def test_two_sided_gate(s, why):
+    """Section 3.2: with upper thresholds the gate fires only between Delta_l and Delta_h."""
+    c = K.make_float_case("band", s, "bf16", density=0.5)
+    one_sided = K.run_oracle(c)
+    c.delta_high = (c.delta + np.float32(0.8)).astype(np.float32)
+    ref, st, exempt = _run(c)
+    assert 0 < ref.active < one_sided.active
+    assert st.active == ref.active or exempt > 0

@@ -215,3 +215,21 @@ def test_channel_grouping(s, why):
     c = K.make_float_case("tc2grp", s, "bf16", density=0.3, grouped=True)
     ref, st, exempt, _ = _run(c)
     assert abs(st.density - ref.density) < 2e-3 and 0.2 < st.density < 0.4
+
+
+TWO_SIDED = [
+    (O.Shape(3, 28, 28, 128, 128, groups=4), "128@28"),
+    (O.Shape(3, 14, 14, 256, 256, groups=4), "256@14"),
+    (O.Shape(3, 8, 8, 256, 256, groups=4), "256@8"),
+]
+
+
+@pytest.mark.parametrize("s,why", TWO_SIDED, ids=[w for _, w in TWO_SIDED])
+def test_two_sided_gate(s, why):
+    """Section 3.2: with upper thresholds the gate fires only between Delta_l and Delta_h."""
+    c = K.make_float_case("band", s, "bf16", density=0.5)
+    one_sided = K.run_oracle(c)
+    c.delta_high = (c.delta + np.float32(0.8)).astype(np.float32)
+    ref, st, exempt, _ = _run(c)
+    assert 0 < ref.active < one_sided.active
+    assert st.active == ref.active or exempt > 0
