@@ -74,6 +74,7 @@ struct Shared2 {
   uint32_t tmem_base;
   uint32_t abort_flag;
   uint32_t fired[2][kEpiWarps];   // per sub-tile, per epilogue warp: a gate of a valid pixel fired
+  float t2[128];                  // upper thresholds of the two-sided gate (Section 3.2) of the channel tile
   // copies that make up the patch being loaded: {shared-memory offset, h, n, tensor map}
   uint32_t box_dst[kMaxBoxes];
   int box_h[kMaxBoxes], box_n[kMaxBoxes], box_map[kMaxBoxes];
@@ -123,7 +124,6 @@ __device__ __forceinline__ void set_max_regs_dec() {
 // layout: channels ch0 + 8*ci + lane/4, ci = 0..3, of the warp's 32.
 struct Consts4 {
   float kt[4], ka1[4], kb1[4], ka2[4], kb2[4];
-  float kt2[4];   // upper thresholds of the two-sided gate (Section 3.2), +inf for the one-sided gate
 };
 
 // What an epilogue thread keeps of a sub-tile between its gate pass and its combine pass.  Lane l
@@ -178,8 +178,10 @@ __device__ __forceinline__ uint32_t open_halves(uint32_t v) { return __vcmpeq2(v
 // d = (P >= t).  Where d = 0 the output f(a1*P + b1) is final; where d = 1 the "gate open" mark
 // is written in its place.  A piece goes through the staging tile to y as 16-byte vectors, and
 // the lane that stores a vector reads the eight decisions off it for the pixel's mask word.
-template <bool kHasRes>
-__device__ __forceinline__ void gate_pass(const Tc2Params& prm, Keep& kp, const Consts4& kc, uint32_t t_acc,
+// (kTwoSided: the gate of Section 3.2 with upper thresholds t2[4], read from shared memory per
+// pass so that the plain gate neither keeps them in registers nor compares against them)
+template <bool kHasRes, bool kTwoSided>
+__device__ __forceinline__ void gate_pass(const Tc2Params& prm, Keep& kp, const Consts4& kc, const float* s_t2, uint32_t t_acc,
                                           int gx, int pg, int lane, int word_idx, float lo, __nv_bfloat16* y_q,
                                           const __nv_bfloat16* res_q, uint8_t* s_tile, unsigned long long& st_active,
                                           unsigned long long& st_words, unsigned long long& st_words_on) {
@@ -187,6 +189,11 @@ __device__ __forceinline__ void gate_pass(const Tc2Params& prm, Keep& kp, const 
   const Tc2Plan& P = prm.P;
   const int pieces = P.nmma >> 4;
   pixel_offsets(L, P, gx, pg, lane, kp);
+  float t2[4] = {0.f, 0.f, 0.f, 0.f};
+  if (kTwoSided) {
+#pragma unroll
+    for (int ci = 0; ci < 4; ++ci) t2[ci] = s_t2[8 * ci + (lane >> 2)];
+  }
   bool fired = false;
 #pragma unroll 1
   for (int q = 0; q < 4; ++q) {
@@ -208,7 +215,8 @@ __device__ __forceinline__ void gate_pass(const Tc2Params& prm, Keep& kp, const 
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
           const float a = __uint_as_float((ci >> 1) ? r1[4 * oct + 2 * (ci & 1) + e] : r0[4 * oct + 2 * (ci & 1) + e]);
-          d[e] = a >= kc.kt[ci] && a <= kc.kt2[ci];          // Eq. 2 (two-sided: Section 3.2): ties fire, NaN does not
+          d[e] = a >= kc.kt[ci];                             // Eq. 2: a tie fires, NaN does not
+          if (kTwoSided) d[e] = d[e] && a <= t2[ci];         // Section 3.2: and stays below the upper threshold
           float v = fmaf(kc.ka1[ci], a, kc.kb1[ci]);         // BN1 of the partial sum (Section 4)
           if (kHasRes) {
             const uint32_t oj = __shfl_sync(0xffffffffu, offs, slot0 + 8 * oct + 2 * (lane & 3) + e);
@@ -603,13 +611,16 @@ tc2_gated_conv_kernel(const __grid_constant__ CUtensorMap map_r1,
     Consts4 kc;
 #pragma unroll
     for (int ci = 0; ci < 4; ++ci) {
-      kc.kt[ci] = 0.f; kc.ka1[ci] = 0.f; kc.kb1[ci] = 0.f; kc.ka2[ci] = 0.f; kc.kb2[ci] = 0.f; kc.kt2[ci] = 0.f;
+      kc.kt[ci] = 0.f; kc.ka1[ci] = 0.f; kc.kb1[ci] = 0.f; kc.ka2[ci] = 0.f; kc.kb2[ci] = 0.f;
       if (ch_valid && jobs > 0) {
         const ChannelConsts k = fold_channel(prm.bn, prm.delta, L.eps, ch0 + 8 * ci + (lane >> 2));
-        kc.kt[ci] = k.t; kc.ka1[ci] = k.a1; kc.kb1[ci] = k.b1; kc.ka2[ci] = k.a2; kc.kb2[ci] = k.b2; kc.kt2[ci] = k.t2;
+        kc.kt[ci] = k.t; kc.ka1[ci] = k.a1; kc.kb1[ci] = k.b1; kc.ka2[ci] = k.a2; kc.kb2[ci] = k.b2;
+        sh->t2[quad * 32 + 8 * ci + (lane >> 2)] = k.t2;   // (the four warps of a quadrant write the same values)
       }
     }
     const float lo = L.relu ? 0.f : -__int_as_float(0x7f800000);   // f = ReLU, or the identity
+    const bool two_sided = prm.bn.delta_high != nullptr;
+    __syncwarp();                                                  // (sh->t2 is read by the warp's own lanes only)
     const uint32_t t_lane = tmem + ((uint32_t)(quad * 32) << 16);
     const int word_idx = tile_c * 4 + quad;
     __nv_bfloat16* y_q = prm.y + ch0;
@@ -634,8 +645,12 @@ tc2_gated_conv_kernel(const __grid_constant__ CUtensorMap map_r1,
         Keep kx = X ? keep1 : keep0;
         if (ch_valid) {
           if (!comb)
-            gate_pass<kHasRes>(prm, kx, kc, t_acc, g0 + X * P.r, pg, lane, word_idx, lo, y_q, res_q, s_tile, st_active,
-                               st_words, st_words_on);
+            if (two_sided)
+              gate_pass<kHasRes, true>(prm, kx, kc, sh->t2 + quad * 32, t_acc, g0 + X * P.r, pg, lane, word_idx, lo, y_q, res_q,
+                                       s_tile, st_active, st_words, st_words_on);
+            else
+              gate_pass<kHasRes, false>(prm, kx, kc, nullptr, t_acc, g0 + X * P.r, pg, lane, word_idx, lo, y_q, res_q,
+                                        s_tile, st_active, st_words, st_words_on);
           else
             combine_pass<kHasRes>(prm, kx, kc, t_acc, pg, lane, lo, y_q, res_q, s_tile);
         }

@@ -621,6 +621,7 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
       // path reads that group's input chunks, its conditional path the others in ascending order.
       // The weight tiles keep their K coordinates: only the chunks of x change.
       const int own0 = L.grouping ? (tile_n * NT) / (L.c_out / L.groups) * P.base_chunks : 0;
+      const int cond_lo = L.grouping ? own0 + P.base_chunks : cond_first_chunk;   // first chunk behind the base chunks
       for (int j = 0; j <= jobs && ok; ++j) {
         if (j < jobs) { load_chunks(j, own0, own0 + P.base_chunks, 0); CG_PROF_EV(j, 0); }
         if (j >= 1 && has_cond && ok && !P.share_a) {
@@ -631,11 +632,11 @@ tc_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x,
             if (!ok) break;
             blocks = __shfl_sync(0xffffffffu, slot_blocks(sh, jj % kNP), 0);
           }
-          if (blocks && L.grouping) {
-            load_chunks(jj, 0, own0, cond_part);
-            load_chunks(jj, own0 + P.base_chunks, P.chunks, cond_part);
-          } else if (blocks) {
-            load_chunks(jj, cond_first_chunk, P.chunks, cond_part);
+          if (blocks) {
+            // (one call site: the chunks in front of the tile's own group, then those behind it)
+#pragma unroll 1
+            for (int part2 = L.grouping ? 0 : 1; part2 < 2 && ok; ++part2)
+              load_chunks(jj, part2 ? cond_lo : 0, part2 ? P.chunks : own0, cond_part);
           }
         }
       }
