@@ -27,6 +27,8 @@ SHAPES = [
     (O.Shape(2, 14, 14, 256, 64, groups=8), "G = 8, c_p = 32, c_out != c_in"),
     (O.Shape(2, 13, 11, 64, 192, groups=2), "odd extents, G = 2, three column tiles of 64"),
     (O.Shape(2, 9, 9, 64, 64, kh=1, kw=1, pad=0, groups=4), "1x1 kernel"),
+    (O.Shape(1, 5, 127, 64, 64, groups=4), "widest rows the kernel takes: 127 pixels + 1 pad column = one 128-row tile"),
+    (O.Shape(1, 3, 3, 64, 64, groups=4), "one 3x3 image: a single, mostly empty tile"),
     (O.Shape(14, 56, 56, 64, 128, kh=1, kw=1, pad=0, groups=4), "1x1 kernel 64 -> 128, 392 row tiles: three jobs per CTA"),
     (O.Shape(12, 56, 56, 64, 64, groups=4), "336 row tiles: up to three jobs per CTA, resident weights"),
     (O.Shape(50, 28, 28, 128, 128, groups=4), "350 row tiles: streamed weights, three jobs per CTA"),

@@ -33,6 +33,9 @@ SHAPES = [
     (O.Shape(256, 4, 4, 128, 128, groups=4), "many small images per pixel tile"),
     (O.Shape(3, 56, 56, 64, 64, groups=8), "G = 8 at 64 channels: c_p = 8, weights repacked into the workspace"),
     (O.Shape(2, 17, 9, 64, 128, groups=8), "c_p = 8, odd extents, 128 output channels"),
+    (O.Shape(1, 6, 200, 64, 64, groups=4), "one image, 200 pixels wide: a sub-tile is a single row"),
+    (O.Shape(1, 3, 3, 64, 32, groups=4), "one 3x3 image, 32 output channels: a single job"),
+    (O.Shape(2, 10, 10, 512, 128, groups=2), "c_p = 256: four base chunks, 72 K stages"),
 ]
 
 
