@@ -392,21 +392,22 @@ struct MmaIssuer {
   //   chunk 0 and then the remaining chunks.
   template <bool RES>
   __device__ __forceinline__ void phase3(bool cond) {
-    int nfull;   // whole chunks (four K steps per tap) after the first, partial one
+    int nfull;        // whole chunks (four K steps per tap) after the first, partial one
+    int small = 0;    // K steps per tap of a phase that runs on tiles of several taps (one call site each)
+    int partial = 0;  // first K step of a conditional path that starts behind the base channels of chunk 0
     if (kp16 >= 4) {
       nfull = cond ? chunks - base_chunks : base_chunks;
     } else if (!cond) {
-      if (kp16 == 1) base_small3<RES, 1>(); else base_small3<RES, 2>();
-      nfull = 0;
+      small = kp16; nfull = 0;
     } else if (pad8 == 2) {
-      base_small3<RES, 2>();        // (int8, 64 input channels: two K steps per tap, two taps per tile)
-      nfull = 0;
+      small = 2; nfull = 0;         // (int8, 64 input channels: two K steps per tap, two taps per tile)
     } else if (pad8) {
       nfull = chunks;               // (repacked weights: zeros multiply the base channels)
     } else {
-      if (kp16 == 1) chunk_taps3<RES, 1, 4>(); else chunk_taps3<RES, 2, 4>();
-      nfull = chunks - 1;
+      partial = kp16; nfull = chunks - 1;
     }
+    if (small == 1) base_small3<RES, 1>(); else if (small == 2) base_small3<RES, 2>();
+    if (partial == 1) chunk_taps3<RES, 1, 4>(); else if (partial == 2) chunk_taps3<RES, 2, 4>();
 #pragma unroll 1
     for (int q = 0; q < nfull && ok; ++q) chunk_taps3<RES, 0, 4>();
   }
