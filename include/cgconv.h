@@ -49,8 +49,10 @@ typedef enum {
   CG_ALGO_DIRECT = 1, /* CUDA-core direct convolution: any shape, sums in the order (r,s,c_in) */
   CG_ALGO_TENSOR = 2, /* tcgen05 implicit GEMM; CG_ERR_UNSUPPORTED at create if not eligible */
   CG_ALGO_TENSOR_ROWS = 3,     /* the pixel-major tcgen05 kernel only (pixels on the MMA's M side) */
-  CG_ALGO_TENSOR_CHANNELS = 4  /* the channel-major tcgen05 kernel only (output channels on the M side).
-                                  AUTO and TENSOR pick between the two by layer shape. */
+  CG_ALGO_TENSOR_CHANNELS = 4, /* the channel-major tcgen05 kernel only (output channels on the M side) */
+  CG_ALGO_TENSOR_STACKED = 5   /* the tap-stacked tcgen05 kernel only (64 -> 64 channel layers: the three
+                                  taps of a filter row share one MMA).
+                                  AUTO and TENSOR pick between the three by layer shape. */
 } cg_algo;
 
 /* How the tensor-core path treats the conditional path (Eq. 1, second case). */
@@ -157,7 +159,9 @@ typedef struct {
  *                         of 64; c_in/G equal to 8, 16 or 32 (BF16; 32 or 64 for I8, at most 32 when
  *                         c_in = 64) or a multiple of 64 (128); output width at most 128;
  *   channel-major kernel: BF16, stride 1, c_out a multiple of 32, c_in/G equal to 8, 16, 32 or a
- *                         multiple of 64, no row compaction (CG_COND_COMPACT).
+ *                         multiple of 64, no row compaction (CG_COND_COMPACT);
+ *   tap-stacked kernel:   BF16, 3x3, stride 1, pad 1, c_in = c_out = 64, c_in/G a multiple of 16, image
+ *                         width 8, 16 or 32, no channel grouping, no channel-wise gate, no row compaction.
  * AUTO falls back to the direct kernels outside these limits.
  * A handle is not thread-safe: calls on one handle must not overlap in time on the host
  * (different handles are independent).  Forward calls of one handle may be queued on different
@@ -221,12 +225,14 @@ int cg_conv_launches_per_forward(cg_conv_t h);
 int cg_conv_uses_tensor_cores(cg_conv_t h);
 
 /* Which kernel family runs this layer (Section 3.1's two convolutions, gate and combine fused
- * in all three): the CUDA-core direct kernels, the tcgen05 kernel with pixels on the MMA's M
- * side, or the tcgen05 kernel with output channels on the M side and pixels on the N side. */
+ * in all of them): the CUDA-core direct kernels, the tcgen05 kernel with pixels on the MMA's M
+ * side, the tcgen05 kernel with output channels on the M side and pixels on the N side, or the
+ * tcgen05 kernel with pixels on the M side and (horizontal tap, output channel) on the N side. */
 typedef enum {
   CG_KERNEL_DIRECT = 0,
   CG_KERNEL_TENSOR_PIXEL_MAJOR = 1,
-  CG_KERNEL_TENSOR_CHANNEL_MAJOR = 2
+  CG_KERNEL_TENSOR_CHANNEL_MAJOR = 2,
+  CG_KERNEL_TENSOR_TAP_STACKED = 3
 } cg_kernel_id;
 int cg_conv_kernel_id(cg_conv_t h);
 

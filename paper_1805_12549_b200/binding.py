@@ -17,7 +17,9 @@ from . import build as _build
 CG_OK = 0
 CG_F32, CG_BF16, CG_I8 = 0, 1, 2
 CG_ALGO_AUTO, CG_ALGO_DIRECT, CG_ALGO_TENSOR, CG_ALGO_TENSOR_ROWS, CG_ALGO_TENSOR_CHANNELS = 0, 1, 2, 3, 4
+CG_ALGO_TENSOR_STACKED = 5
 CG_KERNEL_DIRECT, CG_KERNEL_TENSOR_PIXEL_MAJOR, CG_KERNEL_TENSOR_CHANNEL_MAJOR = 0, 1, 2
+CG_KERNEL_TENSOR_TAP_STACKED = 3
 CG_COND_AUTO, CG_COND_DENSE, CG_COND_SKIP_TILES, CG_COND_COMPACT = 0, 1, 2, 3
 
 EXPORTS = ("cg_conv_create", "cg_conv_workspace_bytes", "cg_conv_forward",

@@ -7,6 +7,7 @@
 #include "common.cuh"
 #include "tc_conv.cuh"
 #include "tc2_conv.cuh"
+#include "tc3_conv.cuh"
 
 struct cg_conv_s {
   cg_conv_desc desc;
@@ -19,6 +20,9 @@ struct cg_conv_s {
   int use_tc2;                    // channel-major tensor-core kernel (tc2_conv.cu)
   cg::Tc2Plan plan2;
   cg::Tc2Maps maps2;
+  int use_tc3;                    // tap-stacked tensor-core kernel (tc3_conv.cu)
+  cg::Tc3Plan plan3;
+  cg::Tc3Maps maps3;
 };
 
 namespace {
@@ -41,7 +45,7 @@ cg_status check_desc(const cg_conv_desc* d) {
   if (d->in_dtype == CG_I8 && (d->requant_shift < 1 || d->requant_shift > 31)) return CG_ERR_INVALID_ARG;
   if (d->in_dtype == CG_I8 && d->has_residual) return CG_ERR_INVALID_ARG;
   if (!(d->bn_eps >= 0.f)) return CG_ERR_INVALID_ARG;
-  if (d->algo < CG_ALGO_AUTO || d->algo > CG_ALGO_TENSOR_CHANNELS) return CG_ERR_INVALID_ARG;
+  if (d->algo < CG_ALGO_AUTO || d->algo > CG_ALGO_TENSOR_STACKED) return CG_ERR_INVALID_ARG;
   if (d->cond_mode < CG_COND_AUTO || d->cond_mode > CG_COND_COMPACT) return CG_ERR_INVALID_ARG;
   if (d->grouping != 0 && d->grouping != 1) return CG_ERR_INVALID_ARG;
   if (d->grouping && d->c_out % d->groups != 0) return CG_ERR_INVALID_ARG;
@@ -111,6 +115,7 @@ cg_status cg_conv_create(cg_conv_t* out, const cg_conv_desc* desc) {
   h->counters = nullptr;
   std::memset(&h->maps, 0, sizeof(h->maps));
   std::memset(&h->maps2, 0, sizeof(h->maps2));
+  std::memset(&h->maps3, 0, sizeof(h->maps3));
   // (which kernels apply is decided before the device is needed, so that an ineligible layer is
   // reported as such on any machine)
   const bool have_device = cudaGetDevice(&h->device) == cudaSuccess;
@@ -127,21 +132,26 @@ cg_status cg_conv_create(cg_conv_t* out, const cg_conv_desc* desc) {
   // Each also takes the layers only it can run.
   const bool prefer2 = h->L.c_out == 128 ||
                        (h->L.c_out == 256 && (h->L.ho * h->L.wo <= 64 || h->L.m >= 20000));
-  const bool allow1 = desc->algo != CG_ALGO_TENSOR_CHANNELS, allow2 = desc->algo != CG_ALGO_TENSOR_ROWS && !chan;
+  // A third kernel takes the 64 -> 64 channel layers it can run (measured faster than both others).
+  const bool only3 = desc->algo == CG_ALGO_TENSOR_STACKED;
+  const bool allow1 = desc->algo != CG_ALGO_TENSOR_CHANNELS && !only3;
+  const bool allow2 = desc->algo != CG_ALGO_TENSOR_ROWS && !chan && !only3;
+  const bool allow3 = desc->algo == CG_ALGO_AUTO || desc->algo == CG_ALGO_TENSOR || only3;
   const int cond_mode = (chan && desc->cond_mode == CG_COND_COMPACT) ? CG_COND_SKIP_TILES : desc->cond_mode;
   bool ok1 = false, ok2 = false;
-  if (want_tc && allow2 && (prefer2 || !allow1)) ok2 = cg::tc2_plan(h->L, desc->in_dtype, cond_mode, sms, &h->plan2);
-  if (want_tc && allow1 && !ok2) ok1 = cg::tc_plan(h->L, desc->in_dtype, cond_mode, &h->plan);
-  if (want_tc && allow2 && !ok1 && !ok2) ok2 = cg::tc2_plan(h->L, desc->in_dtype, cond_mode, sms, &h->plan2);
+  h->use_tc3 = want_tc && allow3 && cg::tc3_plan(h->L, desc->in_dtype, cond_mode, sms, &h->plan3);
+  if (!h->use_tc3 && want_tc && allow2 && (prefer2 || !allow1)) ok2 = cg::tc2_plan(h->L, desc->in_dtype, cond_mode, sms, &h->plan2);
+  if (want_tc && allow1 && !ok2 && !h->use_tc3) ok1 = cg::tc_plan(h->L, desc->in_dtype, cond_mode, &h->plan);
+  if (want_tc && allow2 && !ok1 && !ok2 && !h->use_tc3) ok2 = cg::tc2_plan(h->L, desc->in_dtype, cond_mode, sms, &h->plan2);
   h->use_tc2 = ok2;
   const bool tc_ok = ok1;
   const bool must_tc = desc->algo >= CG_ALGO_TENSOR;
-  if (must_tc && !tc_ok && !h->use_tc2) { delete h; return CG_ERR_UNSUPPORTED; }
+  if (must_tc && !tc_ok && !h->use_tc2 && !h->use_tc3) { delete h; return CG_ERR_UNSUPPORTED; }
   if (!have_device) { delete h; return CG_ERR_CUDA; }
-  h->use_tc = tc_ok || h->use_tc2;
+  h->use_tc = tc_ok || h->use_tc2 || h->use_tc3;
   if (h->use_tc && !cg::tc_device_ok(h->device)) {
     if (must_tc) { delete h; return CG_ERR_UNSUPPORTED; }
-    h->use_tc = 0; h->use_tc2 = 0;
+    h->use_tc = 0; h->use_tc2 = 0; h->use_tc3 = 0;
   }
   if (cudaMalloc(&h->counters, cg::CNT_SLOTS * sizeof(unsigned long long)) != cudaSuccess) {
     delete h; return CG_ERR_CUDA;
@@ -164,6 +174,7 @@ size_t cg_conv_workspace_bytes(cg_conv_t h) {
   if (h->L.channel_tau > 0.f && h->use_tc) return cg::tc_channel_gate_workspace_bytes(h->L, h->plan);
   if (h->L.channel_tau > 0.f) return cg::channel_gate_workspace_bytes(h->L);
   if (h->use_tc2) return cg::tc2_workspace_bytes(h->L, h->plan2);
+  if (h->use_tc3) return 0;
   return h->use_tc ? cg::tc_workspace_bytes(h->L, h->plan) : 0;
 }
 
@@ -171,6 +182,7 @@ int cg_conv_launches_per_forward(cg_conv_t h) {
   if (!h) return 0;
   if (h->L.channel_tau > 0.f) return h->use_tc ? 4 + 2 * (h->plan.pad8 ? 1 : 0) : 2;
   if (h->use_tc2) return h->plan2.pad8 ? 2 : 1;
+  if (h->use_tc3) return 1;
   return (h->use_tc && (h->plan.cond_mode == CG_COND_COMPACT || h->plan.pad8)) ? 2 : 1;
 }
 
@@ -185,6 +197,13 @@ int cg_conv_plan_string(cg_conv_t h, char* buf, size_t len) {
                          "(%d pixels, MMA N=%d), %d K stages (%d base), weight ring %d, lead %d, grid %d",
                          P.tiles_c, P.jobs_m, P.nsub, P.r, P.np, P.nmma, P.ns, P.nb, P.ring, P.lead, P.grid);
   }
+  if (h->use_tc3) {
+    const cg::Tc3Plan& P = h->plan3;
+    return std::snprintf(buf, len,
+                         "tap-stacked tcgen05: %d jobs of %d image rows (128 pixels x 192 stacked columns), %d base K step(s) "
+                         "of 4, resident weights, grid %d",
+                         P.jobs, P.rows, P.kp, P.grid);
+  }
   if (h->use_tc) {
     const cg::TcPlan& P = h->plan;
     return std::snprintf(buf, len,
@@ -196,6 +215,7 @@ int cg_conv_plan_string(cg_conv_t h, char* buf, size_t len) {
 
 int cg_conv_kernel_id(cg_conv_t h) {
   if (!h) return -1;
+  if (h->use_tc3) return CG_KERNEL_TENSOR_TAP_STACKED;
   return h->use_tc2 ? CG_KERNEL_TENSOR_CHANNEL_MAJOR : (h->use_tc ? CG_KERNEL_TENSOR_PIXEL_MAJOR : CG_KERNEL_DIRECT);
 }
 
@@ -223,6 +243,9 @@ cg_status cg_conv_forward(cg_conv_t h, const void* x, const void* w_base, const 
   if (h->use_tc && h->L.channel_tau > 0.f) {
     err = cg::launch_tc_channel_gate(h->L, h->plan, h->desc.in_dtype, &h->maps, x, w_base, w_cond, *bn, delta,
                                      residual, y, mask_out, workspace, h->counters, stream);
+  } else if (h->use_tc3) {
+    err = cg::launch_tc3(h->L, h->plan3, &h->maps3, x, w_base, w_cond, *bn, delta, residual, y, mask_out,
+                         h->counters, stream);
   } else if (h->use_tc2) {
     err = cg::launch_tc2(h->L, h->plan2, &h->maps2, x, w_base, w_cond, *bn, delta, residual, y,
                          mask_out, workspace, h->counters, stream);
