@@ -37,6 +37,8 @@ UNIT = "images/s"
 # writes of a captured launch are still in the 126 MB L2 when it ends, so they are not in these
 # sums.  Reported only while the kernel sources still hash to what they were when the counters
 # were taken.
+KERNEL_NAMES = ["direct", "tcgen05 pixel-major", "tcgen05 channel-major", "tcgen05 tap-stacked"]
+
 TRAFFIC = {
     "source_sha": "0695bff4182f201b",
     "bytes_per_launch": {"c64@32": 33915136, "c128@16": 17145344},
@@ -304,7 +306,7 @@ def layer_record(lb, d_ms, st, peaks):
     t_hbm = lb.algorithmic_bytes / (peaks["hbm_gbs"] * 1e9)
     rec = {
         "layer": lb.shape.name, "us": round(d_ms * 1e3, 2), "density": round(st.density, 4),
-        "kernel": ["direct", "tcgen05 pixel-major", "tcgen05 channel-major"][lb.conv.kernel_id],
+        "kernel": KERNEL_NAMES[lb.conv.kernel_id],
         "gated_tflops": round(el_flops / (d_ms * 1e-3) / 1e12, 1),
         "gbs": round(lb.algorithmic_bytes / (d_ms * 1e-3) / 1e9, 1),
         "roof_us": round(max(t_tensor, t_hbm) * 1e6, 2),
@@ -436,7 +438,7 @@ def run_network_block(args, peaks):
         "ms_gated_layers": round(sum(v for k, v in per_op.items() if k in gated_names), 4),
         "ms_other_operators": round(sum(v for k, v in per_op.items() if k not in gated_names), 4),
         "ms_per_operator": {k: round(v, 4) for k, v in per_op.items()},
-        "kernels": {s.name: ["direct", "tcgen05 pixel-major", "tcgen05 channel-major"][inst.convs[s.name].kernel_id]
+        "kernels": {s.name: KERNEL_NAMES[inst.convs[s.name].kernel_id]
                     for s in net.specs},
     }
     inst.close()

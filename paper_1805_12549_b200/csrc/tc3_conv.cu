@@ -16,19 +16,19 @@
 //
 // Per job (128 / W output rows of one image), following Section 3.1 and Eq. 1-3:
 //   base path    raw P = the three D_s over the base channels (TMEM columns [0,192));
-//   gate         8 warps: P = shifted sum of raw P, written back to TMEM as 64 columns (a ring of two)
-//                so that raw P is free for the next job at once; d = (P >= t[c]) (and P <= t2[c] for
-//                the two-sided gate of Section 3.2) -> mask words;
-//   conditional  raw R over the remaining channels (TMEM columns [192,384)), skipped if no gate of the
-//                job fired (CG_COND_SKIP_TILES);
-//   combine      8 warps: R = shifted sum of raw R; y = f(BN1(P)) or f(BN2(P+R)) by mask bit, staged
-//                in shared memory (two tiles) and written by one TMA store.
+//   conditional  raw R over the remaining channels (TMEM columns [192,384)), issued right behind the
+//                base path; with CG_COND_SKIP_TILES only once the gate is known, and not at all if no
+//                gate of the job fired;
+//   epilogue     16 warps (TMEM lane quadrant x 16 channels), all on the same job: raw P -> registers
+//                (raw P is free for the next job at once), P = shifted sum, d = (P >= t[c]) (and
+//                P <= t2[c] for the two-sided gate of Section 3.2) -> mask bits; raw R -> registers,
+//                R = shifted sum; y = f(BN1(P)) or f(BN2(P+R)) by mask bit, staged in shared memory
+//                (a ring of three tiles) and written by one TMA store.  P never leaves the registers.
 // Weights are resident in shared memory: every CTA builds the three 192-row tiles itself with plain
 // loads (row (s,c) = the 64 input channels of tap (r,s): base channels first, as in x).
 //
-// Warp roles: 0 = patch producer, 1 = MMA issuer (owns TMEM), 2-3 = help with the weights,
-// 4-11 = gate group (TMEM lane quadrant x half of the channels), 12-19 = combine group (same
-// split).  Every mbarrier wait is bounded; on expiry the CTA records CG_ERR_DEVICE_TIMEOUT with the
+// Warp roles: 0 = patch producer, 1 = MMA issuer (owns TMEM), 2 = y and mask stores, 4-19 =
+// epilogue; warps 2-19 build the weight tiles first.  Every mbarrier wait is bounded; on expiry the CTA records CG_ERR_DEVICE_TIMEOUT with the
 // id of the wait and leaves.
 #include <cstring>
 
@@ -40,16 +40,16 @@ namespace cg {
 namespace {
 
 constexpr int kT3Threads = 640;
-constexpr int kGateWarp0 = 4, kGateWarps = 8;
-constexpr int kCombWarp0 = 12, kCombWarps = 8;
-constexpr int kEpiThreads = (kGateWarps + kCombWarps) * 32;
-constexpr int kCombThreads = kCombWarps * 32;
+constexpr int kStoreWarp = 2;
+constexpr int kEpiWarp0 = 4, kEpiWarps = 16;
+constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kLoaderWarps = 18;                 // warps 2-19 build the weight tiles
 constexpr int kNA = 4;                           // patch buffers
 constexpr int kPatchBytes = 192 * 128;           // 128 pixel slots + two image rows of at most 32 pixels
 constexpr int kWTileBytes = 192 * 128;           // one filter row: 3 taps x 64 output channels
 constexpr int kStageBytes = 128 * 128;           // y staging tile
-constexpr uint32_t kColRawP = 0, kColRawR = 192, kColFin = 384;   // TMEM columns
+constexpr int kNY = 3;                           // staging tiles
+constexpr uint32_t kColRawP = 0, kColRawR = 192;   // TMEM columns
 constexpr int kSpinLimit = 1 << 21;
 constexpr long long kWaitCycles = 2000000000ll;
 
@@ -57,10 +57,10 @@ constexpr long long kWaitCycles = 2000000000ll;
 constexpr unsigned kOffW = 0;
 constexpr unsigned kOffA = kOffW + 3 * kWTileBytes;
 constexpr unsigned kOffY = kOffA + kNA * kPatchBytes;
-constexpr unsigned kOffMask = kOffY + 2 * kStageBytes;        // [2][128][2] mask words
-constexpr unsigned kOffConsts = kOffMask + 2 * 128 * 2 * 4;   // t[64], t2[64], {a1,b1,a2,b2}[64]
+constexpr unsigned kOffMask = kOffY + kNY * kStageBytes;       // [kNY][128][4] mask bits, 16 per epilogue warp
+constexpr unsigned kOffConsts = kOffMask + kNY * 128 * 4 * 2;   // t[64], t2[64], {a1,b1,a2,b2}[64]
 constexpr unsigned kOffBar = kOffConsts + 64 * 4 * 2 + 64 * 16;
-constexpr unsigned kSmemUsed = kOffBar + 256;
+constexpr unsigned kSmemUsed = kOffBar + 512;
 
 struct Tc3Params {
   LayerDims L;
@@ -78,12 +78,13 @@ struct Shared3 {
   uint64_t a_full[kNA], a_empty[kNA];
   uint64_t w_ready;
   uint64_t rawp_full, rawp_free, rawr_full, rawr_free;
-  uint64_t fin_full[2], fin_free[2];
+  uint64_t y_full[kNY], y_free[kNY];   // staging tiles (with the mask bits) of a job
+  uint64_t gate_done[2];           // CG_COND_SKIP_TILES: the job's gate has been evaluated (by job parity)
   uint32_t tmem_base;
   uint32_t abort_flag;
-  uint32_t fired[2][kGateWarps];   // per P slot, per gate warp: a gate of its rows and channels fired
+  uint32_t fired[2][kEpiWarps];    // by job parity, per epilogue warp: a gate of its rows and channels fired
 };
-static_assert(sizeof(Shared3) <= 256, "barrier block");
+static_assert(sizeof(Shared3) <= 512, "barrier block");
 
 // Bounded wait (the loop lives in one out-of-line copy).  Each poll parks the thread in hardware for
 // a short time; the wait gives up after about a second, or within a few polls once another wait of
@@ -136,8 +137,12 @@ __device__ __forceinline__ void issue_rows(uint32_t lead, uint32_t desc_hi, uint
 __device__ __forceinline__ float stacked_sum(uint32_t d0, uint32_t d1, uint32_t d2, bool first_col, bool last_col) {
   const float a = __uint_as_float(__shfl_up_sync(0xffffffffu, d0, 1));
   const float b = __uint_as_float(__shfl_down_sync(0xffffffffu, d2, 1));
-  return (__uint_as_float(d1) + (first_col ? 0.f : a)) + (last_col ? 0.f : b);
+  float v = __uint_as_float(d1);
+  if (!first_col) v += a;   // (predicated adds: what wraps around the image edge is dropped, not multiplied by 0)
+  if (!last_col) v += b;
+  return v;
 }
+
 
 __global__ void __launch_bounds__(kT3Threads, 1)
 tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
@@ -150,7 +155,7 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
   uint8_t* s_w = smem + kOffW;
   uint8_t* s_a = smem + kOffA;
   uint8_t* s_y = smem + kOffY;
-  uint32_t* s_mask = (uint32_t*)(smem + kOffMask);
+  unsigned short* s_bits = (unsigned short*)(smem + kOffMask);
   float* s_t = (float*)(smem + kOffConsts);
   float* s_t2 = s_t + 64;
   float4* s_k = (float4*)(s_t2 + 64);
@@ -169,21 +174,22 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
     n0 = t / P.tiles_per_image;
     h0 = (t - n0 * P.tiles_per_image) * P.rows;
   };
-  auto any_fired = [&](int f) {
-    const volatile uint32_t* w = sh->fired[f];
-    uint32_t b = 0;
+  auto any_fired = [&](int b) {
+    const volatile uint32_t* w = sh->fired[b];
+    uint32_t v = 0;
 #pragma unroll
-    for (int i = 0; i < kGateWarps; ++i) b |= w[i];
-    return b != 0u;
+    for (int i = 0; i < kEpiWarps; ++i) v |= w[i];
+    return v != 0u;
   };
 
   // ---------------------------------------------------------------- setup
   if (threadIdx.x == 0) {
     for (int i = 0; i < kNA; ++i) { ptx::mbar_init(&sh->a_full[i], 1); ptx::mbar_init(&sh->a_empty[i], 1); }
     ptx::mbar_init(&sh->w_ready, kLoaderWarps);
-    ptx::mbar_init(&sh->rawp_full, 1); ptx::mbar_init(&sh->rawp_free, kGateWarps);
-    ptx::mbar_init(&sh->rawr_full, 1); ptx::mbar_init(&sh->rawr_free, kCombWarps);
-    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&sh->fin_full[i], kGateWarps); ptx::mbar_init(&sh->fin_free[i], kCombWarps); }
+    ptx::mbar_init(&sh->rawp_full, 1); ptx::mbar_init(&sh->rawp_free, kEpiWarps);
+    ptx::mbar_init(&sh->rawr_full, 1); ptx::mbar_init(&sh->rawr_free, kEpiWarps);
+    ptx::mbar_init(&sh->gate_done[0], kEpiWarps); ptx::mbar_init(&sh->gate_done[1], kEpiWarps);
+    for (int i = 0; i < kNY; ++i) { ptx::mbar_init(&sh->y_full[i], kEpiWarps); ptx::mbar_init(&sh->y_free[i], 1); }
     sh->abort_flag = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&map_x); ptx::prefetch_tensormap(&map_y);
@@ -223,8 +229,8 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
     __syncwarp();
     if (lane == 0) ptx::mbar_arrive(&sh->w_ready);
   }
-  if (warp >= kGateWarp0) {
-    const int et = (int)threadIdx.x - kGateWarp0 * 32;
+  if (warp >= kEpiWarp0) {
+    const int et = (int)threadIdx.x - kEpiWarp0 * 32;
     if (et < 64) {
       const ChannelConsts k = fold_channel(prm.bn, prm.delta, L.eps, et);
       s_t[et] = k.t; s_t2[et] = k.t2; s_k[et] = make_float4(k.a1, k.b1, k.a2, k.b2);
@@ -248,15 +254,18 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
     }
   } else if (warp == 1) {
     // ============================================================ MMA issuer
-    // (the whole warp, convergent; lane 0 issues)   order: base(0) | base(1) cond(0) | base(2) cond(1) ...
+    // (the whole warp, convergent; lane 0 issues)   order: base(0) cond(0) | base(1) cond(1) | ...;
+    // with CG_COND_SKIP_TILES the conditional path of a job waits for its gate, so the base path of
+    // the next job goes first: base(0) | base(1) cond(0) | base(2) cond(1) | ...
     const uint32_t lead = lane == 0 ? 1u : 0u;
     const uint32_t desc_hi = (uint32_t)(ptx::smem_desc(0, 1024, 2) >> 32);
     const uint32_t a_base_lo = (ptx::smem_u32(s_a) >> 4) | 0x10000u;
     const uint32_t b_lo = (ptx::smem_u32(s_w) >> 4) | 0x10000u;
     const uint32_t row_lo = (uint32_t)W * 8u;
+    const int skew = dense ? 0 : 1;
     uint32_t r_use = 0;
     bool ok = jobs > 0 && wait3(sh, prm.counters, &sh->w_ready, 0, 2);
-    for (int s = 0; s <= jobs && ok; ++s) {
+    for (int s = 0; s < jobs + skew && ok; ++s) {
       if (s < jobs) {
         const int slot = s % kNA;
         ok = wait3(sh, prm.counters, &sh->a_full[slot], (s / kNA) & 1, 3);
@@ -273,13 +282,14 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
         ptx::umma_commit_if(lead, &sh->rawp_full);
         if (!has_cond) ptx::umma_commit_if(lead, &sh->a_empty[slot]);
       }
-      if (s >= 1 && has_cond) {
-        const int jj = s - 1, f = jj & 1, slot = jj % kNA;
+      const int jj = s - skew;
+      if (jj >= 0 && has_cond) {
+        const int b = jj & 1, slot = jj % kNA;
         bool run = true;
         if (!dense) {
-          ok = wait3(sh, prm.counters, &sh->fin_full[f], (jj >> 1) & 1, 5);
+          ok = wait3(sh, prm.counters, &sh->gate_done[b], (jj >> 1) & 1, 5);
           if (!ok) break;
-          run = any_fired(f);
+          run = any_fired(b);
         }
         if (run) {
           ok = wait3(sh, prm.counters, &sh->rawr_free, (r_use & 1) ^ 1, 6);
@@ -299,206 +309,210 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
         }
       }
     }
-  } else if (warp >= kGateWarp0) {
-    // ============================================================ epilogue (16 warps)
-    const bool gate_group = warp < kCombWarp0;
+  } else if (warp == kStoreWarp) {
+    // ============================================================ store warp
+    // Writes what the epilogue leaves in shared memory: the y tile (one TMA store) and the mask
+    // words of the job's 128 rows (four rows per lane, each from the bits of four epilogue warps).
+    // A tile goes back to the epilogue one job late, when the wait for its store to have read it
+    // no longer blocks.
+    unsigned long long st_rows = 0, st_rows_active = 0;
+    bool ok = true;
+    int b = 0, u = 0;   // j % kNY, j / kNY
+    for (int j = 0; j < jobs && ok; ++j) {
+      ok = wait3(sh, prm.counters, &sh->y_full[b], u & 1, 11);
+      if (!ok) break;
+      int n0, h0;
+      job_origin(j, n0, h0);
+      if (lane == 0) {
+        ptx::tma_store_4d(&map_y, s_y + (size_t)b * kStageBytes, 0, 0, h0, n0);
+        ptx::tma_store_commit();
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int i = k * 32 + lane;
+        const int h_loc = i / W, col = i - h_loc * W;
+        const bool valid = h0 + h_loc < H;
+        const uint2 w2 = *(const uint2*)&s_bits[(b * 128 + i) * 4];
+        if (valid && prm.mask) {
+          const long long m = ((long long)n0 * H + (h0 + h_loc)) * W + col;
+          prm.mask[m * 2] = w2.x; prm.mask[m * 2 + 1] = w2.y;
+        }
+        st_rows += valid ? 1 : 0;
+        st_rows_active += (w2.x | w2.y) != 0u ? 1 : 0;
+      }
+      // the tile (and the bits) of the job before: its store has read them
+      if (lane == 0) ptx::tma_store_wait_read_but_one();
+      __syncwarp();
+      if (j >= 1 && lane == 0) ptx::mbar_arrive(&sh->y_free[b == 0 ? kNY - 1 : b - 1]);
+      if (++b == kNY) { b = 0; ++u; }
+    }
+    if (lane == 0) ptx::tma_store_wait_all();
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      st_rows += __shfl_xor_sync(0xffffffffu, st_rows, o);
+      st_rows_active += __shfl_xor_sync(0xffffffffu, st_rows_active, o);
+    }
+    if (lane == 0 && ok) {
+      atomicAdd(&prm.counters[CNT_ROWS_TOTAL], st_rows);
+      atomicAdd(&prm.counters[CNT_ROWS_ACTIVE], st_rows_active);
+    }
+  } else if (warp >= kEpiWarp0) {
+    // ============================================================ epilogue (16 warps, all on the same job)
     const int quad = warp & 3;                                   // TMEM lane quadrant
-    const int half = ((warp - kGateWarp0) >> 2) & 1;             // channels [32*half, 32*half + 32) = one mask word
+    const int cgp = (warp - kEpiWarp0) >> 2;                     // channels [16*cgp, 16*cgp + 16)
+    const int cb = cgp * 16;
     const int i = quad * 32 + lane;                              // pixel slot = TMEM lane
     const int h_loc = i / W, col = i - h_loc * W;
     const bool first_col = col == 0, last_col = col == W - 1;
     const uint32_t t_lane = tmem + ((uint32_t)(quad * 32) << 16);
-    const int ct = (int)threadIdx.x - kCombWarp0 * 32;           // thread index within the combine group
-    unsigned long long st_active = 0, st_rows = 0;
+    const int et = (int)threadIdx.x - kEpiWarp0 * 32;            // thread index within the group
+    unsigned long long st_active = 0;
     uint32_t r_use = 0;
     bool ok = true;
-
-    if (gate_group) {
-      for (int j = 0; j < jobs && ok; ++j) {
-        const int f = j & 1;
-        ok = wait3(sh, prm.counters, &sh->rawp_full, j & 1, 7);
-        if (!ok) break;
+    int b = 0, u = 0;   // j % kNY, j / kNY
+    for (int j = 0; j < jobs && ok; ++j, b = (b + 1 == kNY ? 0 : b + 1), u += (b == 0 ? 1 : 0)) {
+      uint8_t* buf = s_y + (size_t)b * kStageBytes;
+      int n0, h0;
+      job_origin(j, n0, h0);
+      const bool valid = h0 + h_loc < H;
+      const long long m = ((long long)n0 * H + (h0 + h_loc)) * W + col;
+      // residual values (the shortcut of a residual block, added before the activation): fetched early
+      uint4 res[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
+      const bool has_res = prm.residual != nullptr && valid;
+      if (has_res) {
+        const uint4* rp = (const uint4*)(prm.residual + m * 64 + cb);
+        res[0] = __ldg(rp); res[1] = __ldg(rp + 1);
+      }
+      ok = wait3(sh, prm.counters, &sh->rawp_full, j & 1, 7);
+      if (!ok) break;
+      uint32_t p[16];
+      uint32_t bits = 0;
+      {
         ptx::tc_fence_after();
-        int n0, h0;
-        job_origin(j, n0, h0);
-        const bool valid = h0 + h_loc < H;
-        const long long m = ((long long)n0 * H + (h0 + h_loc)) * W + col;
-        uint32_t word = 0;
-#pragma unroll
-        for (int piece = 0; piece < 2; ++piece) {
-          const int cb = half * 32 + piece * 16;
-          uint32_t d0[16], d1[16], d2[16];
-          ptx::tmem_ld_nowait<16>(t_lane + kColRawP + (uint32_t)cb, d0);
-          ptx::tmem_ld_nowait<16>(t_lane + kColRawP + 64u + (uint32_t)cb, d1);
-          ptx::tmem_ld_nowait<16>(t_lane + kColRawP + 128u + (uint32_t)cb, d2);
-          ptx::tmem_ld_wait<16>(d0);
-          ptx::tmem_ld_wait<16>(d1);
-          ptx::tmem_ld_wait<16>(d2);
-          if (piece == 1) {
-            // raw P has been read: the base path of the next job may overwrite it
-            ptx::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&sh->rawp_free);
-          }
-          uint32_t p[16];
-#pragma unroll
-          for (int c = 0; c < 16; ++c) p[c] = __float_as_uint(stacked_sum(d0[c], d1[c], d2[c], first_col, last_col));
-          if (piece == 0) {
-            // the combine group must be done with this P slot's previous job
-            ok = wait3(sh, prm.counters, &sh->fin_free[f], ((j >> 1) & 1) ^ 1, 8);
-            if (!ok) break;
-          }
-          ptx::tmem_st16(t_lane + kColFin + (uint32_t)(f * 64 + cb), p);
-          // four partial words, so that the bit inserts do not form one dependent chain
-          uint32_t pw[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const float4 t4 = *(const float4*)(s_t + cb + q * 4);
-            pw[q] |= (__uint_as_float(p[q * 4 + 0]) >= t4.x ? 1u : 0u) << (q * 4 + 0);
-            pw[q] |= (__uint_as_float(p[q * 4 + 1]) >= t4.y ? 1u : 0u) << (q * 4 + 1);
-            pw[q] |= (__uint_as_float(p[q * 4 + 2]) >= t4.z ? 1u : 0u) << (q * 4 + 2);
-            pw[q] |= (__uint_as_float(p[q * 4 + 3]) >= t4.w ? 1u : 0u) << (q * 4 + 3);
-          }
-          uint32_t bits = (pw[0] | pw[1]) | (pw[2] | pw[3]);
-          if (two_sided) {
-            // Section 3.2: the gate also needs P <= the upper threshold (ties included)
-            uint32_t ph[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const float4 u4 = *(const float4*)(s_t2 + cb + q * 4);
-              ph[q] |= (__uint_as_float(p[q * 4 + 0]) <= u4.x ? 1u : 0u) << (q * 4 + 0);
-              ph[q] |= (__uint_as_float(p[q * 4 + 1]) <= u4.y ? 1u : 0u) << (q * 4 + 1);
-              ph[q] |= (__uint_as_float(p[q * 4 + 2]) <= u4.z ? 1u : 0u) << (q * 4 + 2);
-              ph[q] |= (__uint_as_float(p[q * 4 + 3]) <= u4.w ? 1u : 0u) << (q * 4 + 3);
-            }
-            bits &= (ph[0] | ph[1]) | (ph[2] | ph[3]);
-          }
-          word |= bits << (piece * 16);
-        }
-        if (!ok) break;
-        ptx::tmem_st_wait();
-        if (!valid) word = 0;
-        s_mask[(f * 128 + i) * 2 + half] = word;
-        if (valid && prm.mask) prm.mask[m * 2 + half] = word;
-        st_active += __popc(word);
-        const uint32_t any = __ballot_sync(0xffffffffu, word != 0u);
-        const uint32_t rows_valid = __ballot_sync(0xffffffffu, valid);
-        if (lane == 0) {
-          sh->fired[f][warp - kGateWarp0] = any;
-          if (half == 0) st_rows += __popc(rows_valid);
-        }
+        uint32_t d0[16], d1[16], d2[16];
+        ptx::tmem_ld_nowait<16>(t_lane + kColRawP + (uint32_t)cb, d0);
+        ptx::tmem_ld_nowait<16>(t_lane + kColRawP + 64u + (uint32_t)cb, d1);
+        ptx::tmem_ld_nowait<16>(t_lane + kColRawP + 128u + (uint32_t)cb, d2);
+        // (while the loads are in flight) the store warp must be done with this staging tile and its bits
+        ok = wait3(sh, prm.counters, &sh->y_free[b], (u & 1) ^ 1, 10);
+        ptx::tmem_ld_wait<16>(d0);
+        ptx::tmem_ld_wait<16>(d1);
+        ptx::tmem_ld_wait<16>(d2);
+        // raw P is in registers: the base path of the next job may overwrite it
         ptx::tc_fence_before();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&sh->fin_full[f]);
+        if (lane == 0) ptx::mbar_arrive(&sh->rawp_free);
+#pragma unroll
+        for (int c = 0; c < 16; ++c) p[c] = __float_as_uint(stacked_sum(d0[c], d1[c], d2[c], first_col, last_col));
+        // Eq. 2-3 with the batch norm folded into the threshold: d = (P >= t), a compare and a
+        // predicated bit insert per channel (a NaN sum does not fire); four partial words, so that the
+        // inserts do not form one dependent chain
+        uint32_t pw[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float4 t4 = *(const float4*)(s_t + cb + q * 4);
+          if (__uint_as_float(p[q * 4 + 0]) >= t4.x) pw[q] |= 1u << (q * 4 + 0);
+          if (__uint_as_float(p[q * 4 + 1]) >= t4.y) pw[q] |= 1u << (q * 4 + 1);
+          if (__uint_as_float(p[q * 4 + 2]) >= t4.z) pw[q] |= 1u << (q * 4 + 2);
+          if (__uint_as_float(p[q * 4 + 3]) >= t4.w) pw[q] |= 1u << (q * 4 + 3);
+        }
+        bits = (pw[0] | pw[1]) | (pw[2] | pw[3]);
+        if (two_sided) {
+          // Section 3.2: the gate also needs P <= the upper threshold (ties included)
+          uint32_t ph[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float4 u4 = *(const float4*)(s_t2 + cb + q * 4);
+            if (__uint_as_float(p[q * 4 + 0]) <= u4.x) ph[q] |= 1u << (q * 4 + 0);
+            if (__uint_as_float(p[q * 4 + 1]) <= u4.y) ph[q] |= 1u << (q * 4 + 1);
+            if (__uint_as_float(p[q * 4 + 2]) <= u4.z) ph[q] |= 1u << (q * 4 + 2);
+            if (__uint_as_float(p[q * 4 + 3]) <= u4.w) ph[q] |= 1u << (q * 4 + 3);
+          }
+          bits &= (ph[0] | ph[1]) | (ph[2] | ph[3]);
+        }
+        if (!valid) bits = 0;
+        if (!ok) break;
+        s_bits[(b * 128 + i) * 4 + cgp] = (unsigned short)bits;
+        st_active += __popc(bits);
       }
-    } else {
-      for (int j = 0; j < jobs; ++j) {
-        const int f = j & 1;
-        uint8_t* buf = s_y + (size_t)(j & 1) * kStageBytes;
-        // A wait that gives up must not keep its warp from the group barrier below, where the sibling
-        // warps are going to arrive: the decision to leave is taken after it, from the CTA-wide flag.
-        ok = wait3(sh, prm.counters, &sh->fin_full[f], (j >> 1) & 1, 9);
-        const bool run = ok && has_cond && (dense || any_fired(f));
-        if (run) ok = wait3(sh, prm.counters, &sh->rawr_full, r_use & 1, 10);
-        int n0, h0;
-        job_origin(j, n0, h0);
-        if (ok) {
+      const uint32_t warp_any = __ballot_sync(0xffffffffu, bits != 0u);
+      bool run = has_cond;
+      if (!dense && has_cond) {
+        // the issuer (and this group) must know whether any gate of the job fired
+        if (lane == 0) sh->fired[j & 1][warp - kEpiWarp0] = warp_any;
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&sh->gate_done[j & 1]);
+        ok = wait3(sh, prm.counters, &sh->gate_done[j & 1], (j >> 1) & 1, 8);
+        if (!ok) break;
+        run = any_fired(j & 1);
+      }
+      // R is read only where the conditional path ran and a gate of these rows and channels fired
+      const bool have_r = run && warp_any != 0u;
+      uint32_t rr[16];
+#pragma unroll
+      for (int c = 0; c < 16; ++c) rr[c] = 0u;
+      if (run) {
+        ok = wait3(sh, prm.counters, &sh->rawr_full, r_use & 1, 9);
+        if (!ok) break;
+        {
           ptx::tc_fence_after();
-          const uint32_t wv = s_mask[(f * 128 + i) * 2 + half];
-          if (half == 0) {
-            const uint32_t other = s_mask[(f * 128 + i) * 2 + 1];
-            const uint32_t act = __ballot_sync(0xffffffffu, (wv | other) != 0u);
-            if (lane == 0) st_rows += __popc(act);
+          if (have_r) {
+            uint32_t e0[16], e1[16], e2[16];
+            ptx::tmem_ld_nowait<16>(t_lane + kColRawR + (uint32_t)cb, e0);
+            ptx::tmem_ld_nowait<16>(t_lane + kColRawR + 64u + (uint32_t)cb, e1);
+            ptx::tmem_ld_nowait<16>(t_lane + kColRawR + 128u + (uint32_t)cb, e2);
+            ptx::tmem_ld_wait<16>(e0);
+            ptx::tmem_ld_wait<16>(e1);
+            ptx::tmem_ld_wait<16>(e2);
+#pragma unroll
+            for (int c = 0; c < 16; ++c) rr[c] = __float_as_uint(stacked_sum(e0[c], e1[c], e2[c], first_col, last_col));
           }
-          const bool valid = h0 + h_loc < H;
-          const __nv_bfloat16* res_row = nullptr;
-          if (prm.residual && valid)
-            res_row = prm.residual + (((long long)n0 * H + (h0 + h_loc)) * W + col) * 64 + half * 32;
-          uint8_t* st = buf + (size_t)i * 128;
-#pragma unroll
-          for (int piece = 0; piece < 2; ++piece) {
-            const int cb = half * 32 + piece * 16;
-            const uint32_t bits = (wv >> (piece * 16)) & 0xffffu;
-            // R is read only where the conditional path ran and a gate of these rows and channels fired
-            const bool have_r = run && __ballot_sync(0xffffffffu, bits != 0u) != 0u;
-            uint32_t p[16], rr[16];
-            ptx::tmem_ld_nowait<16>(t_lane + kColFin + (uint32_t)(f * 64 + cb), p);
-            if (have_r) {
-              uint32_t e0[16], e1[16], e2[16];
-              ptx::tmem_ld_nowait<16>(t_lane + kColRawR + (uint32_t)cb, e0);
-              ptx::tmem_ld_nowait<16>(t_lane + kColRawR + 64u + (uint32_t)cb, e1);
-              ptx::tmem_ld_nowait<16>(t_lane + kColRawR + 128u + (uint32_t)cb, e2);
-              ptx::tmem_ld_wait<16>(e0);
-              ptx::tmem_ld_wait<16>(e1);
-              ptx::tmem_ld_wait<16>(e2);
-#pragma unroll
-              for (int c = 0; c < 16; ++c) rr[c] = __float_as_uint(stacked_sum(e0[c], e1[c], e2[c], first_col, last_col));
-            } else {
-#pragma unroll
-              for (int c = 0; c < 16; ++c) rr[c] = 0u;
-            }
-            ptx::tmem_ld_wait<16>(p);
-            if (piece == 1) {
-              // both accumulators have been read
-              ptx::tc_fence_before();
-              __syncwarp();
-              if (lane == 0) {
-                ptx::mbar_arrive(&sh->fin_free[f]);
-                if (run) ptx::mbar_arrive(&sh->rawr_free);
-              }
-            }
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-              uint4 res4 = make_uint4(0u, 0u, 0u, 0u);
-              if (res_row) res4 = __ldg((const uint4*)(res_row + piece * 16 + q * 8));
-              const uint32_t resw[4] = {res4.x, res4.y, res4.z, res4.w};
-              uint32_t packed[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const int jx = q * 8 + e * 2;
-                const float4 k0 = s_k[cb + jx], k1 = s_k[cb + jx + 1];
-                const bool f0 = (bits >> jx) & 1u, f1 = (bits >> (jx + 1)) & 1u;
-                const float p0 = __uint_as_float(p[jx]), p1 = __uint_as_float(p[jx + 1]);
-                // Eq. 1: the full sum P+R where the gate fired, the partial sum elsewhere, each under
-                // the batch norm of its path (Section 4) as one fused multiply-add
-                float v0 = f0 ? fmaf(k0.z, p0 + __uint_as_float(rr[jx]), k0.w) : fmaf(k0.x, p0, k0.y);
-                float v1 = f1 ? fmaf(k1.z, p1 + __uint_as_float(rr[jx + 1]), k1.w) : fmaf(k1.x, p1, k1.y);
-                if (res_row) {
-                  v0 += __uint_as_float(resw[e] << 16);
-                  v1 += __uint_as_float(resw[e] & 0xffff0000u);
-                }
-                if (L.relu) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
-                const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
-                packed[e] = *(const uint32_t*)&h2;
-              }
-              const int c16 = (cb >> 3) + q;
-              *(uint4*)(st + ((c16 ^ (i & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-            }
-          }
-          if (run) ++r_use;
-        }
-        ptx::fence_proxy_async();
-        // the store of the job before last (the other staging tile was this job's) has long finished
-        // reading; after the barrier every warp may overwrite that tile
-        if (ct == 0) ptx::tma_store_wait_read();
-        ptx::named_bar_sync(1, kCombThreads);
-        if (*(volatile uint32_t*)&sh->abort_flag) { ok = false; break; }
-        if (ct == 0) {
-          ptx::tma_store_4d(&map_y, buf, 0, 0, h0, n0);
-          ptx::tma_store_commit();
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&sh->rawr_free);
+          ++r_use;
         }
       }
-      if (ct == 0) ptx::tma_store_wait_all();
+      {
+        uint8_t* st = buf + (size_t)i * 128;   // (128-byte swizzle: 16-byte piece c16 of row i at c16 ^ (i & 7))
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const uint32_t resw[4] = {res[q].x, res[q].y, res[q].z, res[q].w};
+          uint32_t packed[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int jx = q * 8 + e * 2;
+            const float4 k0 = s_k[cb + jx], k1 = s_k[cb + jx + 1];
+            const bool f0 = (bits >> jx) & 1u, f1 = (bits >> (jx + 1)) & 1u;
+            const float p0 = __uint_as_float(p[jx]), p1 = __uint_as_float(p[jx + 1]);
+            // Eq. 1: the full sum P+R where the gate fired, the partial sum elsewhere, each under the
+            // batch norm of its path (Section 4) as one fused multiply-add
+            const float o0 = fmaf(k0.z, p0 + __uint_as_float(rr[jx]), k0.w), c0 = fmaf(k0.x, p0, k0.y);
+            const float o1 = fmaf(k1.z, p1 + __uint_as_float(rr[jx + 1]), k1.w), c1 = fmaf(k1.x, p1, k1.y);
+            float v0 = f0 ? o0 : c0;
+            float v1 = f1 ? o1 : c1;
+            if (has_res) {
+              v0 += __uint_as_float(resw[e] << 16);
+              v1 += __uint_as_float(resw[e] & 0xffff0000u);
+            }
+            if (L.relu) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
+            packed[e] = *(const uint32_t*)&h2;
+          }
+          const int c16 = (cb >> 3) + q;
+          *(uint4*)(st + ((c16 ^ (i & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        }
+      }
+      ptx::fence_proxy_async();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&sh->y_full[b]);
     }
 
     // counters of this CTA
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) st_active += __shfl_xor_sync(0xffffffffu, st_active, o);
-    if (lane == 0 && ok) {
-      if (gate_group) atomicAdd(&prm.counters[CNT_ACTIVE], st_active);
-      if (half == 0) atomicAdd(&prm.counters[gate_group ? CNT_ROWS_TOTAL : CNT_ROWS_ACTIVE], st_rows);
-    }
-    if (!gate_group && ct == 0 && ok) {
+    if (lane == 0 && ok) atomicAdd(&prm.counters[CNT_ACTIVE], st_active);
+    if (et == 0 && ok) {
       const unsigned long long k_p = 9ull * L.c_p, k_r = 9ull * L.c_r;
       if (blockIdx.x == 0) atomicAdd(&prm.counters[CNT_CALLS], 1ull);
       atomicAdd(&prm.counters[CNT_TILES_TOTAL], (unsigned long long)jobs);
@@ -572,7 +586,10 @@ bool tc3_plan(const LayerDims& L, int in_dtype, int cond_mode, int sms, Tc3Plan*
   if (jobs > 0x7fffffffll) return false;
   P.jobs = (int)jobs;
   P.kp = L.c_p / 16;
-  P.cond_mode = cond_mode == CG_COND_AUTO ? CG_COND_SKIP_TILES : cond_mode;
+  // CG_COND_AUTO: the conditional path is issued right behind the base path.  A job is 128 pixels x
+  // 64 channels: at any useful density some gate of it fires, and waiting for the gate before the
+  // conditional MMAs serialises the job (measured: 1.6x the time).
+  P.cond_mode = cond_mode == CG_COND_SKIP_TILES ? CG_COND_SKIP_TILES : CG_COND_DENSE;
   P.grid = (int)(jobs < sms ? jobs : sms);
   P.valid = 1;
   *plan = P;

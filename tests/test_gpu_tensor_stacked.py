@@ -57,7 +57,7 @@ def test_parity_at_30_percent(s, why):
 def test_delta_limits(s, why, dv):
     """All gates open: the ordinary layer.  All gates shut: base path only, no conditional MMAs."""
     c = K.make_float_case("stlim", s, "bf16", delta=dv)
-    ref, st, exempt, _ = _run(c)
+    ref, st, exempt, _ = _run(c, cond_mode=SKIP)
     assert exempt == 0
     if dv < 0:
         assert st.active == st.outputs and st.tiles_skipped == 0
