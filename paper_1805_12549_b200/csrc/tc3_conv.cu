@@ -27,8 +27,8 @@
 // Weights are resident in shared memory: every CTA builds the three 192-row tiles itself with plain
 // loads (row (s,c) = the 64 input channels of tap (r,s): base channels first, as in x).
 //
-// Warp roles: 0 = patch producer, 1 = MMA issuer (owns TMEM), 2 = y and mask stores, 4-19 =
-// epilogue; warps 2-19 build the weight tiles first.  Every mbarrier wait is bounded; on expiry the CTA records CG_ERR_DEVICE_TIMEOUT with the
+// Warp roles: 0 = patch producer, 1 = MMA issuer of the base path (owns TMEM), 2 = y and mask stores,
+// 3 = MMA issuer of the conditional path, 4-19 = epilogue; warps 2-19 build the weight tiles first.  Every mbarrier wait is bounded; on expiry the CTA records CG_ERR_DEVICE_TIMEOUT with the
 // id of the wait and leaves.
 #include <cstring>
 
@@ -41,6 +41,7 @@ namespace {
 
 constexpr int kT3Threads = 640;
 constexpr int kStoreWarp = 2;
+constexpr int kCondWarp = 3;                     // second MMA issuer (conditional path)
 constexpr int kEpiWarp0 = 4, kEpiWarps = 16;
 constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kLoaderWarps = 18;                 // warps 2-19 build the weight tiles
@@ -184,7 +185,8 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
 
   // ---------------------------------------------------------------- setup
   if (threadIdx.x == 0) {
-    for (int i = 0; i < kNA; ++i) { ptx::mbar_init(&sh->a_full[i], 1); ptx::mbar_init(&sh->a_empty[i], 1); }
+    // (a patch is released by both issuers: each one's commit covers only its own MMAs)
+    for (int i = 0; i < kNA; ++i) { ptx::mbar_init(&sh->a_full[i], 1); ptx::mbar_init(&sh->a_empty[i], has_cond ? 2 : 1); }
     ptx::mbar_init(&sh->w_ready, kLoaderWarps);
     ptx::mbar_init(&sh->rawp_full, 1); ptx::mbar_init(&sh->rawp_free, kEpiWarps);
     ptx::mbar_init(&sh->rawr_full, 1); ptx::mbar_init(&sh->rawr_free, kEpiWarps);
@@ -252,24 +254,23 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
         ptx::tma_load_4d(s_a + (size_t)slot * kPatchBytes, &map_x, &sh->a_full[slot], 0, 0, h0 - 1, n0);
       }
     }
-  } else if (warp == 1) {
-    // ============================================================ MMA issuer
-    // (the whole warp, convergent; lane 0 issues)   order: base(0) cond(0) | base(1) cond(1) | ...;
-    // with CG_COND_SKIP_TILES the conditional path of a job waits for its gate, so the base path of
-    // the next job goes first: base(0) | base(1) cond(0) | base(2) cond(1) | ...
+  } else if (warp == 1 || warp == kCondWarp) {
+    // ============================================================ MMA issuers
+    // Warp 1 issues the base path of every job, warp 3 the conditional path: the two write different
+    // accumulators, and a tcgen05.mma keeps the issuing warp's scheduler busy for about as long as the
+    // MMA runs, so the two paths sit on different schedulers.  (Each warp whole and convergent; lane 0
+    // issues.)  With CG_COND_SKIP_TILES the conditional path of a job waits for its gate.
     const uint32_t lead = lane == 0 ? 1u : 0u;
     const uint32_t desc_hi = (uint32_t)(ptx::smem_desc(0, 1024, 2) >> 32);
     const uint32_t a_base_lo = (ptx::smem_u32(s_a) >> 4) | 0x10000u;
     const uint32_t b_lo = (ptx::smem_u32(s_w) >> 4) | 0x10000u;
     const uint32_t row_lo = (uint32_t)W * 8u;
-    const int skew = dense ? 0 : 1;
-    uint32_t r_use = 0;
-    bool ok = jobs > 0 && wait3(sh, prm.counters, &sh->w_ready, 0, 2);
-    for (int s = 0; s < jobs + skew && ok; ++s) {
-      if (s < jobs) {
-        const int slot = s % kNA;
-        ok = wait3(sh, prm.counters, &sh->a_full[slot], (s / kNA) & 1, 3);
-        ok = ok && wait3(sh, prm.counters, &sh->rawp_free, (s & 1) ^ 1, 4);
+    bool ok = wait3(sh, prm.counters, &sh->w_ready, 0, 2);
+    if (warp == 1) {
+      for (int j = 0; j < jobs && ok; ++j) {
+        const int slot = j % kNA;
+        ok = wait3(sh, prm.counters, &sh->a_full[slot], (j / kNA) & 1, 3);
+        ok = ok && wait3(sh, prm.counters, &sh->rawp_free, (j & 1) ^ 1, 4);
         if (!ok) break;
         ptx::tc_fence_after();
         const uint32_t a_lo = a_base_lo + (uint32_t)slot * (kPatchBytes >> 4);
@@ -280,19 +281,21 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
           default: issue_rows<0, 4>(lead, desc_hi, a_lo, b_lo, row_lo, tmem + kColRawP); break;
         }
         ptx::umma_commit_if(lead, &sh->rawp_full);
-        if (!has_cond) ptx::umma_commit_if(lead, &sh->a_empty[slot]);
+        ptx::umma_commit_if(lead, &sh->a_empty[slot]);
       }
-      const int jj = s - skew;
-      if (jj >= 0 && has_cond) {
-        const int b = jj & 1, slot = jj % kNA;
+    } else if (has_cond) {
+      uint32_t r_use = 0;
+      for (int j = 0; j < jobs && ok; ++j) {
+        const int slot = j % kNA;
         bool run = true;
         if (!dense) {
-          ok = wait3(sh, prm.counters, &sh->gate_done[b], (jj >> 1) & 1, 5);
+          ok = wait3(sh, prm.counters, &sh->gate_done[j & 1], (j >> 1) & 1, 5);
           if (!ok) break;
-          run = any_fired(b);
+          run = any_fired(j & 1);
         }
         if (run) {
-          ok = wait3(sh, prm.counters, &sh->rawr_free, (r_use & 1) ^ 1, 6);
+          ok = wait3(sh, prm.counters, &sh->a_full[slot], (j / kNA) & 1, 12);
+          ok = ok && wait3(sh, prm.counters, &sh->rawr_free, (r_use & 1) ^ 1, 6);
           if (!ok) break;
           ptx::tc_fence_after();
           const uint32_t a_lo = a_base_lo + (uint32_t)slot * (kPatchBytes >> 4);
