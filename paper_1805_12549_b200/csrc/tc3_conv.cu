@@ -11,10 +11,12 @@
 //     D_0[i-1] + D_1[i] + D_2[i+1],
 // where the first term is dropped in image column 0 and the last in column W-1 (the zero padding):
 // the epilogue takes the neighbours' values by warp shuffles.  A job needs 12 MMAs of N = 192
-// instead of 36 of N = 64, a tile is 128 REAL pixels (no pad columns on the M side), and a TMEM lane
-// quadrant holds whole image rows when W divides 32, so no value crosses a warp.
+// instead of 36 of N = 64 and a tile is up to 128 REAL pixels (no pad columns on the M side).  When W
+// divides 32 a TMEM lane quadrant holds whole image rows and no value crosses a warp; otherwise the
+// first and last lane of a warp get their neighbour's value from the adjacent quadrant's warp through
+// shared memory (one named barrier among the four warps that share a channel group, per path).
 //
-// Per job (128 / W output rows of one image), following Section 3.1 and Eq. 1-3:
+// Per job (floor(128 / W) output rows of one image), following Section 3.1 and Eq. 1-3:
 //   base path    raw P = the three D_s over the base channels (TMEM columns [0,192));
 //   conditional  raw R over the remaining channels (TMEM columns [192,384)), issued right behind the
 //                base path; with CG_COND_SKIP_TILES only once the gate is known, and not at all if no
@@ -45,8 +47,7 @@ constexpr int kCondWarp = 3;                     // second MMA issuer (condition
 constexpr int kEpiWarp0 = 4, kEpiWarps = 16;
 constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kLoaderWarps = 18;                 // warps 2-19 build the weight tiles
-constexpr int kNA = 4;                           // patch buffers
-constexpr int kPatchBytes = 192 * 128;           // 128 pixel slots + two image rows of at most 32 pixels
+constexpr int kMaxNA = 4;                        // patch buffers, at most
 constexpr int kWTileBytes = 192 * 128;           // one filter row: 3 taps x 64 output channels
 constexpr int kStageBytes = 128 * 128;           // y staging tile
 constexpr int kNY = 3;                           // staging tiles
@@ -56,12 +57,13 @@ constexpr long long kWaitCycles = 2000000000ll;
 
 // shared-memory map (offsets from a 1024-byte-aligned base)
 constexpr unsigned kOffW = 0;
-constexpr unsigned kOffA = kOffW + 3 * kWTileBytes;
-constexpr unsigned kOffY = kOffA + kNA * kPatchBytes;
+constexpr unsigned kOffY = kOffW + 3 * kWTileBytes;
 constexpr unsigned kOffMask = kOffY + kNY * kStageBytes;       // [kNY][128][4] mask bits, 16 per epilogue warp
 constexpr unsigned kOffConsts = kOffMask + kNY * 128 * 4 * 2;   // t[64], t2[64], {a1,b1,a2,b2}[64]
 constexpr unsigned kOffBar = kOffConsts + 64 * 4 * 2 + 64 * 16;
-constexpr unsigned kSmemUsed = kOffBar + 512;
+constexpr unsigned kOffXch = kOffBar + 512;   // [2 paths][2 directions][4 quadrants][4 channel groups][16] floats
+constexpr unsigned kOffA = (kOffXch + 4096 + 1023) / 1024 * 1024;   // patch buffers: the rest
+constexpr unsigned kPatchArea = 227 * 1024 - 1024 - kOffA;
 
 struct Tc3Params {
   LayerDims L;
@@ -76,7 +78,7 @@ struct Tc3Params {
 };
 
 struct Shared3 {
-  uint64_t a_full[kNA], a_empty[kNA];
+  uint64_t a_full[kMaxNA], a_empty[kMaxNA];
   uint64_t w_ready;
   uint64_t rawp_full, rawp_free, rawr_full, rawr_free;
   uint64_t y_full[kNY], y_free[kNY];   // staging tiles (with the mask bits) of a job
@@ -135,16 +137,20 @@ __device__ __forceinline__ void issue_rows(uint32_t lead, uint32_t desc_hi, uint
 }
 
 // One output value from the three stacked partial sums of its pixel slot and the neighbours'.
-__device__ __forceinline__ float stacked_sum(uint32_t d0, uint32_t d1, uint32_t d2, bool first_col, bool last_col) {
+// (no_a / no_b: the slot has no left / right neighbour in its image row, or the neighbour sits in another warp)
+__device__ __forceinline__ float stacked_sum(uint32_t d0, uint32_t d1, uint32_t d2, bool no_a, bool no_b) {
   const float a = __uint_as_float(__shfl_up_sync(0xffffffffu, d0, 1));
   const float b = __uint_as_float(__shfl_down_sync(0xffffffffu, d2, 1));
   float v = __uint_as_float(d1);
-  if (!first_col) v += a;   // (predicated adds: what wraps around the image edge is dropped, not multiplied by 0)
-  if (!last_col) v += b;
+  if (!no_a) v += a;   // (predicated adds: what wraps around the image edge is dropped, not multiplied by 0)
+  if (!no_b) v += b;
   return v;
 }
 
 
+// kXch: the image width does not divide 32 (two instances, so that the common widths carry none of
+// the exchange code)
+template <bool kXch>
 __global__ void __launch_bounds__(kT3Threads, 1)
 tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
                       const __grid_constant__ Tc3Params prm) {
@@ -169,6 +175,9 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
   const bool has_cond = L.c_r > 0;
   const bool two_sided = prm.bn.delta_high != nullptr;
   const uint32_t patch_tx = (uint32_t)((P.rows + 2) * W) * 128u;
+  const int na = P.na;
+  const uint32_t patch_bytes = (uint32_t)P.patch_bytes;
+  float* s_xch = (float*)(smem + kOffXch);
 
   auto job_origin = [&](int j, int& n0, int& h0) {
     const int t = (int)blockIdx.x + j * (int)gridDim.x;
@@ -186,7 +195,7 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
   // ---------------------------------------------------------------- setup
   if (threadIdx.x == 0) {
     // (a patch is released by both issuers: each one's commit covers only its own MMAs)
-    for (int i = 0; i < kNA; ++i) { ptx::mbar_init(&sh->a_full[i], 1); ptx::mbar_init(&sh->a_empty[i], has_cond ? 2 : 1); }
+    for (int i = 0; i < kMaxNA; ++i) { ptx::mbar_init(&sh->a_full[i], 1); ptx::mbar_init(&sh->a_empty[i], has_cond ? 2 : 1); }
     ptx::mbar_init(&sh->w_ready, kLoaderWarps);
     ptx::mbar_init(&sh->rawp_full, 1); ptx::mbar_init(&sh->rawp_free, kEpiWarps);
     ptx::mbar_init(&sh->rawr_full, 1); ptx::mbar_init(&sh->rawr_free, kEpiWarps);
@@ -244,14 +253,14 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
     // ============================================================ patch producer
     bool ok = true;
     for (int j = 0; j < jobs && ok; ++j) {
-      const int slot = j % kNA;
-      ok = wait3(sh, prm.counters, &sh->a_empty[slot], ((j / kNA) & 1) ^ 1, 1);
+      const int slot = j % na;
+      ok = wait3(sh, prm.counters, &sh->a_empty[slot], ((j / na) & 1) ^ 1, 1);
       if (!ok) break;
       int n0, h0;
       job_origin(j, n0, h0);
       if (lane == 0) {
         ptx::mbar_expect_tx(&sh->a_full[slot], patch_tx);
-        ptx::tma_load_4d(s_a + (size_t)slot * kPatchBytes, &map_x, &sh->a_full[slot], 0, 0, h0 - 1, n0);
+        ptx::tma_load_4d(s_a + (size_t)slot * patch_bytes, &map_x, &sh->a_full[slot], 0, 0, h0 - 1, n0);
       }
     }
   } else if (warp == 1 || warp == kCondWarp) {
@@ -268,12 +277,12 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
     bool ok = wait3(sh, prm.counters, &sh->w_ready, 0, 2);
     if (warp == 1) {
       for (int j = 0; j < jobs && ok; ++j) {
-        const int slot = j % kNA;
-        ok = wait3(sh, prm.counters, &sh->a_full[slot], (j / kNA) & 1, 3);
+        const int slot = j % na;
+        ok = wait3(sh, prm.counters, &sh->a_full[slot], (j / na) & 1, 3);
         ok = ok && wait3(sh, prm.counters, &sh->rawp_free, (j & 1) ^ 1, 4);
         if (!ok) break;
         ptx::tc_fence_after();
-        const uint32_t a_lo = a_base_lo + (uint32_t)slot * (kPatchBytes >> 4);
+        const uint32_t a_lo = a_base_lo + (uint32_t)slot * (patch_bytes >> 4);
         switch (P.kp) {
           case 1: issue_rows<0, 1>(lead, desc_hi, a_lo, b_lo, row_lo, tmem + kColRawP); break;
           case 2: issue_rows<0, 2>(lead, desc_hi, a_lo, b_lo, row_lo, tmem + kColRawP); break;
@@ -286,7 +295,7 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
     } else if (has_cond) {
       uint32_t r_use = 0;
       for (int j = 0; j < jobs && ok; ++j) {
-        const int slot = j % kNA;
+        const int slot = j % na;
         bool run = true;
         if (!dense) {
           ok = wait3(sh, prm.counters, &sh->gate_done[j & 1], (j >> 1) & 1, 5);
@@ -294,11 +303,11 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
           run = any_fired(j & 1);
         }
         if (run) {
-          ok = wait3(sh, prm.counters, &sh->a_full[slot], (j / kNA) & 1, 12);
+          ok = wait3(sh, prm.counters, &sh->a_full[slot], (j / na) & 1, 12);
           ok = ok && wait3(sh, prm.counters, &sh->rawr_free, (r_use & 1) ^ 1, 6);
           if (!ok) break;
           ptx::tc_fence_after();
-          const uint32_t a_lo = a_base_lo + (uint32_t)slot * (kPatchBytes >> 4);
+          const uint32_t a_lo = a_base_lo + (uint32_t)slot * (patch_bytes >> 4);
           switch (P.kp) {
             case 1: issue_rows<1, 4>(lead, desc_hi, a_lo, b_lo, row_lo, tmem + kColRawR); break;
             case 2: issue_rows<2, 4>(lead, desc_hi, a_lo, b_lo, row_lo, tmem + kColRawR); break;
@@ -334,7 +343,7 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
       for (int k = 0; k < 4; ++k) {
         const int i = k * 32 + lane;
         const int h_loc = i / W, col = i - h_loc * W;
-        const bool valid = h0 + h_loc < H;
+        const bool valid = h_loc < P.rows && h0 + h_loc < H;
         const uint2 w2 = *(const uint2*)&s_bits[(b * 128 + i) * 4];
         if (valid && prm.mask) {
           const long long m = ((long long)n0 * H + (h0 + h_loc)) * W + col;
@@ -367,6 +376,14 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
     const int i = quad * 32 + lane;                              // pixel slot = TMEM lane
     const int h_loc = i / W, col = i - h_loc * W;
     const bool first_col = col == 0, last_col = col == W - 1;
+    // W does not divide 32: a warp's first and last lane may have their row neighbour in another warp
+    constexpr bool xch = kXch;
+    const bool no_a = first_col || (xch && lane == 0), no_b = last_col || (xch && lane == 31);
+    const bool fix_a = xch && lane == 0 && !first_col, fix_b = xch && lane == 31 && !last_col && quad < 3;
+    // exchange cells, 16 floats each: [path][direction][quadrant][group]; direction 0 = D_0 of the
+    // quadrant's last slot (for the next quadrant's first lane), 1 = D_2 of its first slot
+    float* x_cell = s_xch + (quad * 4 + cgp) * 16;
+    constexpr int kXDir = 256, kXPath = 512, kXQuad = 64;   // strides in floats
     const uint32_t t_lane = tmem + ((uint32_t)(quad * 32) << 16);
     const int et = (int)threadIdx.x - kEpiWarp0 * 32;            // thread index within the group
     unsigned long long st_active = 0;
@@ -377,7 +394,7 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
       uint8_t* buf = s_y + (size_t)b * kStageBytes;
       int n0, h0;
       job_origin(j, n0, h0);
-      const bool valid = h0 + h_loc < H;
+      const bool valid = h_loc < P.rows && h0 + h_loc < H;
       const long long m = ((long long)n0 * H + (h0 + h_loc)) * W + col;
       // residual values (the shortcut of a residual block, added before the activation): fetched early
       uint4 res[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
@@ -405,8 +422,27 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
         ptx::tc_fence_before();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&sh->rawp_free);
+        if (xch) {
+          if (lane == 31) {
 #pragma unroll
-        for (int c = 0; c < 16; ++c) p[c] = __float_as_uint(stacked_sum(d0[c], d1[c], d2[c], first_col, last_col));
+            for (int c = 0; c < 16; ++c) x_cell[c] = __uint_as_float(d0[c]);
+          }
+          if (lane == 0) {
+#pragma unroll
+            for (int c = 0; c < 16; ++c) x_cell[kXDir + c] = __uint_as_float(d2[c]);
+          }
+          ptx::named_bar_sync(3 + cgp, 128);
+        }
+#pragma unroll
+        for (int c = 0; c < 16; ++c) p[c] = __float_as_uint(stacked_sum(d0[c], d1[c], d2[c], no_a, no_b));
+        if (fix_a) {
+#pragma unroll
+          for (int c = 0; c < 16; ++c) p[c] = __float_as_uint(__uint_as_float(p[c]) + x_cell[c - kXQuad]);
+        }
+        if (fix_b) {
+#pragma unroll
+          for (int c = 0; c < 16; ++c) p[c] = __float_as_uint(__uint_as_float(p[c]) + x_cell[kXDir + kXQuad + c]);
+        }
         // Eq. 2-3 with the batch norm folded into the threshold: d = (P >= t), a compare and a
         // predicated bit insert per channel (a NaN sum does not fire); four partial words, so that the
         // inserts do not form one dependent chain
@@ -450,10 +486,11 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
         run = any_fired(j & 1);
       }
       // R is read only where the conditional path ran and a gate of these rows and channels fired
-      const bool have_r = run && warp_any != 0u;
+      const bool have_r = run && (warp_any != 0u || xch);   // (with the exchange, the neighbours need this warp's R)
       uint32_t rr[16];
 #pragma unroll
       for (int c = 0; c < 16; ++c) rr[c] = 0u;
+      if (xch && !run) ptx::named_bar_sync(3 + cgp, 128);
       if (run) {
         ok = wait3(sh, prm.counters, &sh->rawr_full, r_use & 1, 9);
         if (!ok) break;
@@ -467,8 +504,29 @@ tc3_gated_conv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
             ptx::tmem_ld_wait<16>(e0);
             ptx::tmem_ld_wait<16>(e1);
             ptx::tmem_ld_wait<16>(e2);
+            if (xch) {
+              // (second half of the exchange cells; the barrier also orders this job's reads of the
+              // first half before the next job's writes)
+              if (lane == 31) {
 #pragma unroll
-            for (int c = 0; c < 16; ++c) rr[c] = __float_as_uint(stacked_sum(e0[c], e1[c], e2[c], first_col, last_col));
+                for (int c = 0; c < 16; ++c) x_cell[kXPath + c] = __uint_as_float(e0[c]);
+              }
+              if (lane == 0) {
+#pragma unroll
+                for (int c = 0; c < 16; ++c) x_cell[kXPath + kXDir + c] = __uint_as_float(e2[c]);
+              }
+              ptx::named_bar_sync(3 + cgp, 128);
+            }
+#pragma unroll
+            for (int c = 0; c < 16; ++c) rr[c] = __float_as_uint(stacked_sum(e0[c], e1[c], e2[c], no_a, no_b));
+            if (fix_a) {
+#pragma unroll
+              for (int c = 0; c < 16; ++c) rr[c] = __float_as_uint(__uint_as_float(rr[c]) + x_cell[kXPath - kXQuad + c]);
+            }
+            if (fix_b) {
+#pragma unroll
+              for (int c = 0; c < 16; ++c) rr[c] = __float_as_uint(__uint_as_float(rr[c]) + x_cell[kXPath + kXDir + kXQuad + c]);
+            }
           }
           ptx::tc_fence_before();
           __syncwarp();
@@ -582,8 +640,15 @@ bool tc3_plan(const LayerDims& L, int in_dtype, int cond_mode, int sms, Tc3Plan*
   if (L.grouping && L.groups > 1) return false;
   if (L.channel_tau > 0.f) return false;
   if (cond_mode == CG_COND_COMPACT) return false;
-  if (L.w != 8 && L.w != 16 && L.w != 32) return false;   // a TMEM lane quadrant holds whole image rows
+  if (L.w > 128) return false;                             // a job is at least one whole image row
   P.rows = 128 / L.w;
+  P.xch = (32 % L.w) != 0;                                  // image rows do not line up with the warps
+  // a patch: the job's rows plus one above and one below, and what the last filter row's 128-slot
+  // window reaches behind them
+  P.patch_bytes = (int)(((size_t)(128 + 2 * L.w) * 128 + 1023) / 1024 * 1024);
+  P.na = (int)(kPatchArea / (unsigned)P.patch_bytes);
+  if (P.na > kMaxNA) P.na = kMaxNA;
+  if (P.na < 2) return false;
   P.tiles_per_image = (L.h + P.rows - 1) / P.rows;
   const long long jobs = (long long)L.n * P.tiles_per_image;
   if (jobs > 0x7fffffffll) return false;
@@ -622,16 +687,17 @@ int launch_tc3(const LayerDims& L, const Tc3Plan& P, Tc3Maps* maps, const void* 
   prm.w_cond = static_cast<const __nv_bfloat16*>(w_cond);
   prm.residual = static_cast<const __nv_bfloat16*>(residual);
   prm.mask = mask; prm.counters = counters;
-  static bool attr_set[64] = {};   // (the attribute is per device)
+  static bool attr_set[64][2] = {};   // (the attribute is per device and kernel instance)
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return (int)cudaErrorInvalidDevice;
-  if (!attr_set[dev]) {
-    const cudaError_t e = cudaFuncSetAttribute(tc3_gated_conv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               227 * 1024);
+  typedef void (*Kernel)(CUtensorMap, CUtensorMap, Tc3Params);
+  const Kernel kernel = P.xch ? (Kernel)tc3_gated_conv_kernel<true> : (Kernel)tc3_gated_conv_kernel<false>;
+  if (!attr_set[dev][P.xch ? 1 : 0]) {
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return (int)e;
-    attr_set[dev] = true;
+    attr_set[dev][P.xch ? 1 : 0] = true;
   }
-  static_assert(kSmemUsed + 1024 <= 227 * 1024, "shared memory");
+  static_assert(kPatchArea >= 2 * (128 + 2 * 128) * 128, "shared memory");
   // The same (maximum) amount of dynamic shared memory as the other layer kernels, so that
   // consecutive layers never reconfigure the SM; a programmatic dependent launch: the CTAs set up
   // barriers and TMEM while the previous kernel in the stream drains, and wait for it
@@ -647,7 +713,7 @@ int launch_tc3(const LayerDims& L, const Tc3Plan& P, Tc3Maps* maps, const void* 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  const cudaError_t e = cudaLaunchKernelEx(&cfg, tc3_gated_conv_kernel, ms->x, ms->y, prm);
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, ms->x, ms->y, prm);
   if (e != cudaSuccess) return (int)e;
   return (int)cudaGetLastError();
 }

@@ -1,5 +1,5 @@
 // Tap-stacked tensor-core path of the channel-gated layer (tc3_conv.cu): plan and launcher.
-// For 3x3, stride-1 bf16 layers with 64 input and 64 output channels.
+// For 3x3, stride-1 bf16 layers with 64 input and 64 output channels, images up to 128 pixels wide.
 #pragma once
 
 #include <cuda.h>
@@ -10,7 +10,9 @@ namespace cg {
 
 struct Tc3Plan {
   int valid;
-  int rows;              // output rows per job: 128 / w
+  int rows;              // output rows per job: floor(128 / w)
+  int xch;               // 1: w does not divide 32, neighbouring warps exchange their edge values
+  int patch_bytes, na;   // input patch buffer and how many of them
   int tiles_per_image;   // ceil(h / rows)
   int jobs;              // n * tiles_per_image
   int kp;                // K steps (16 channels) of the base path: c_p / 16

@@ -24,7 +24,17 @@ SHAPES = [
     (O.Shape(1, 1, 8, 64, 64, groups=2), "a single image row of 8 pixels"),
     (O.Shape(40, 32, 32, 64, 64, groups=2), "several jobs per CTA"),
     (O.Shape(2, 32, 32, 64, 64, groups=4, relu=0), "identity activation"),
+    (O.Shape(2, 56, 56, 64, 64, groups=4), "56x56: two rows per job, row ends inside warps, neighbours across warps"),
+    (O.Shape(2, 28, 28, 64, 64, groups=2), "28x28: four rows per job, 112 of 128 slots"),
+    (O.Shape(3, 14, 14, 64, 64, groups=4), "14x14: nine rows per job, the image is two ragged jobs"),
+    (O.Shape(3, 7, 7, 64, 64, groups=2), "7x7: the job's box is taller than the image"),
+    (O.Shape(2, 9, 13, 64, 64, groups=4), "9x13: odd extents"),
+    (O.Shape(1, 5, 64, 64, 64, groups=4), "64 wide: two full rows per job, 5 rows"),
+    (O.Shape(1, 3, 128, 64, 64, groups=2), "128 wide: one row per job, two patch buffers"),
+    (O.Shape(1, 4, 100, 64, 64, groups=4), "100 wide: one row per job, 28 idle slots"),
+    (O.Shape(2, 6, 33, 64, 64, groups=4), "33 wide: every warp boundary falls inside a row"),
 ]
+WIDE = [x for x in SHAPES if x[0].w in (56, 14, 33)]
 
 
 def _run(c, cond_mode=0, with_mask=True):
@@ -52,7 +62,7 @@ def test_parity_at_30_percent(s, why):
         assert (ref.y < 0).any()
 
 
-@pytest.mark.parametrize("s,why", SHAPES[:6], ids=[w for _, w in SHAPES[:6]])
+@pytest.mark.parametrize("s,why", SHAPES[:6] + WIDE, ids=[w for _, w in SHAPES[:6] + WIDE])
 @pytest.mark.parametrize("dv", [-K.INF, K.INF])
 def test_delta_limits(s, why, dv):
     """All gates open: the ordinary layer.  All gates shut: base path only, no conditional MMAs."""
@@ -65,7 +75,7 @@ def test_delta_limits(s, why, dv):
         assert st.active == 0 and st.tiles_skipped == st.tiles_total > 0
 
 
-@pytest.mark.parametrize("s,why", SHAPES[:4], ids=[w for _, w in SHAPES[:4]])
+@pytest.mark.parametrize("s,why", SHAPES[:4] + WIDE, ids=[w for _, w in SHAPES[:4] + WIDE])
 def test_dense_mode_matches_skip_mode(s, why):
     c = K.make_float_case("stdense", s, "bf16", density=0.1, rho=0.7)
     ref, st_d, _, _ = _run(c, cond_mode=DENSE)
@@ -129,16 +139,16 @@ def test_nan_input_does_not_fire():
     np.testing.assert_array_equal(d_gpu[ok], d_ref[ok])
 
 
-@pytest.mark.parametrize("s,why", [SHAPES[0], SHAPES[3], SHAPES[4]], ids=[SHAPES[0][1], SHAPES[3][1], SHAPES[4][1]])
+@pytest.mark.parametrize("s,why", [SHAPES[0], SHAPES[3], SHAPES[4]] + WIDE, ids=[w for _, w in [SHAPES[0], SHAPES[3], SHAPES[4]] + WIDE])
 def test_residual_input(s, why):
     c = K.make_float_case("stres", s, "bf16", density=0.3, residual=True)
     ref, st, exempt, _ = _run(c)
     assert abs(st.density - ref.density) < 2e-3
 
 
-def test_two_sided_gate():
+@pytest.mark.parametrize("s", [O.Shape(3, 32, 32, 64, 64, groups=4), O.Shape(2, 56, 56, 64, 64, groups=4)], ids=["32x32", "56x56"])
+def test_two_sided_gate(s):
     """Section 3.2: the gate fires only between the two thresholds."""
-    s = O.Shape(3, 32, 32, 64, 64, groups=4)
     c = K.make_float_case("st2s", s, "bf16", density=0.3)
     c.delta_high = (c.delta + np.float32(0.8)).astype(np.float32)
     ref, st, exempt, _ = _run(c)
@@ -157,11 +167,13 @@ def test_two_calls_accumulate_and_are_deterministic():
     g.close()
 
 
-def test_full_size_layer_on_sampled_images():
-    """The 64-channel layer of the CIFAR workload at benchmark batch; images are independent, so the
-    oracle checks a sample of them one by one."""
+@pytest.mark.parametrize("workload,layer", [("cifar", "c64@32"), ("imagenet", "c64@56")])
+def test_full_size_layer_on_sampled_images(workload, layer):
+    """The 64-channel layers of the two benchmark workloads at benchmark batch; images are independent,
+    so the oracle checks a sample of them one by one."""
     from paper_1805_12549_b200 import synth
-    ls = {l.name: l for l in synth.cifar_resnet18_layers(256, 4)}["c64@32"]
+    layers = synth.imagenet_resnet18_layers(64, 4) if workload == "imagenet" else synth.cifar_resnet18_layers(256, 4)
+    ls = {l.name: l for l in layers}[layer]
     s = O.Shape(ls.n, ls.hw, ls.hw, ls.c_in, ls.c_out, stride=ls.stride, groups=4)
     c = K.make_float_case("stfull", s, "bf16", density=0.3, calib_images=2)
     g = K.GpuCase(c)              # the default choice for this layer
@@ -179,7 +191,7 @@ def test_full_size_layer_on_sampled_images():
 
 def test_layers_outside_the_kernel_are_refused():
     from paper_1805_12549_b200 import binding as B
-    for kw in (dict(w=56, h=56), dict(c_out=128), dict(groups=8), dict(k=1, pad=0), dict(stride=2)):
+    for kw in (dict(w=130, h=8), dict(c_out=128), dict(groups=8), dict(k=1, pad=0), dict(stride=2)):
         a = dict(n=2, h=32, w=32, c_in=64, c_out=64, k=3, stride=1, pad=1, groups=4)
         a.update(kw)
         with pytest.raises(B.CgError):
