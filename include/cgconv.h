@@ -161,7 +161,8 @@ typedef struct {
  *   channel-major kernel: BF16, stride 1, c_out a multiple of 32, c_in/G equal to 8, 16, 32 or a
  *                         multiple of 64, no row compaction (CG_COND_COMPACT);
  *   tap-stacked kernel:   BF16, 3x3, stride 1, pad 1, c_in = c_out = 64, c_in/G a multiple of 16, image
- *                         width 8, 16 or 32, no channel grouping, no channel-wise gate, no row compaction.
+ *                         width at most 128, no channel grouping, no channel-wise gate, no row compaction
+ *                         (AUTO and TENSOR choose it when the width divides 32).
  * AUTO falls back to the direct kernels outside these limits.
  * A handle is not thread-safe: calls on one handle must not overlap in time on the host
  * (different handles are independent).  Forward calls of one handle may be queued on different

@@ -195,9 +195,9 @@ def test_full_size_layers_on_sampled_images(workload, layer):
 
 def test_default_choice_of_tensor_kernel():
     """CG_ALGO_TENSOR picks the channel-major kernel for 128 output channels, the tap-stacked kernel for
-    64 -> 64 channel 3x3 layers and the pixel-major kernel for stride-2 layers."""
+    64 -> 64 channel 3x3 layers whose width divides 32 and the pixel-major kernel elsewhere."""
     from paper_1805_12549_b200 import binding as B
-    for shape, want in (((4, 28, 28, 128, 128, 1), 2), ((4, 56, 56, 64, 64, 1), 3), ((4, 28, 28, 128, 256, 2), 1)):
+    for shape, want in (((4, 28, 28, 128, 128, 1), 2), ((4, 56, 56, 64, 64, 1), 1), ((4, 32, 32, 64, 64, 1), 3), ((4, 28, 28, 128, 256, 2), 1)):
         n, h, w, ci, co, st = shape
         conv = B.GatedConv(n, h, w, ci, co, k=3, stride=st, pad=1, groups=4, dtype=B.CG_BF16, algo=B.CG_ALGO_TENSOR)
         assert conv.kernel_id == want, conv.plan
