@@ -40,8 +40,8 @@ UNIT = "images/s"
 KERNEL_NAMES = ["direct", "tcgen05 pixel-major", "tcgen05 channel-major", "tcgen05 tap-stacked"]
 
 TRAFFIC = {
-    "source_sha": "0695bff4182f201b",
-    "bytes_per_launch": {"c64@32": 33915136, "c128@16": 17145344},
+    "source_sha": "25f6222633311712",
+    "bytes_per_launch": {"c64@32": 33790250, "c128@16": 17143296, "c256@8": 9645397, "c512@4": 9110314},
 }
 
 
