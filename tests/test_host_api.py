@@ -101,6 +101,25 @@ def test_tensor_algo_rejects_ineligible_layers():
         assert B.lib().cg_conv_create(C.byref(h), C.byref(d)) == 2           # CG_ERR_UNSUPPORTED
 
 
+def test_tap_stacked_algo_eligibility_is_decided_on_the_host():
+    """CG_ALGO_TENSOR_STACKED: 3x3, stride 1, pad 1, bf16, 64 -> 64 channels, c_in/G a multiple of 16,
+    width at most 128, no grouping, no channel-wise gate, no row compaction.  Layers outside report
+    CG_ERR_UNSUPPORTED before any device is needed; a layer inside gets as far as the device."""
+    import torch
+    h = C.c_void_p()
+    ok = dict(algo=B.CG_ALGO_TENSOR_STACKED, in_dtype=B.CG_BF16, out_dtype=B.CG_BF16, c_in=64, c_out=64,
+              h=32, w=32, groups=4)
+    for kw in (dict(w=129), dict(c_out=128), dict(c_in=128), dict(groups=8), dict(kh=1, kw=1, pad=0),
+               dict(stride=2), dict(cond_mode=3), dict(channel_tau=0.5), dict(grouping=1),
+               dict(in_dtype=B.CG_I8, out_dtype=B.CG_I8, requant_shift=8)):
+        d = _desc(**{**ok, **kw})
+        assert B.lib().cg_conv_create(C.byref(h), C.byref(d)) == 2, kw       # CG_ERR_UNSUPPORTED
+    if not torch.cuda.is_available():
+        for kw in (dict(), dict(w=56, h=56), dict(groups=1), dict(groups=2), dict(w=128, h=3)):
+            d = _desc(**{**ok, **kw})
+            assert B.lib().cg_conv_create(C.byref(h), C.byref(d)) == 5, kw   # CG_ERR_CUDA: eligible, no device
+
+
 def test_null_handle_calls_are_safe():
     lib = B.lib()
     assert lib.cg_conv_workspace_bytes(None) == 0
